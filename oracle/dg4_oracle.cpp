@@ -1,0 +1,303 @@
+/*
+ * CPU checker for the sparse-attention layer over an And-Inverter Graph.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, host-only restatement of what
+ * the layer computes, used by the test-suite, by the smoke check and as the timed
+ * CPU baseline of the benchmark.  It shares no code with the CUDA library and the
+ * library never calls it.
+ *
+ * All floating point is fp64.  Every function is the textbook definition written
+ * as direct loops; there is no tiling, fusion or reordering.  OpenMP is used only
+ * as "parallel for over independent nodes".
+ *
+ * What follows what:
+ *   orc_levels            Eq. 1 (logic level: 0 for a primary input, else 1 + max over fan-ins)
+ *   orc_neighbourhood     Sec. 3.2, definition of cone_k(v): all u with a path u -> v of length <= k,
+ *                         v included (the size bound 2^(k+1)-1 counts v); Sec. 3.5: these are the
+ *                         virtual edges the sparse attention is restricted to
+ *   orc_attention         Sec. 3.5: multi-head attention restricted to that set; dot-product score and
+ *                         softmax per destination (the paper leaves the score function to a figure;
+ *                         the dot-product reading is this library's stated choice)
+ *   orc_project           the dense projections of the Transformer block kept around the attention
+ *   orc_layer_parallel    QKV projection -> attention -> output projection (+ residual), all nodes at once
+ *   orc_layer_levelised   the same layer applied level by level in topological order, each level
+ *                         reading the rows already updated for earlier levels (Sec. 1 and Sec. 3.4:
+ *                         each gate is computed once, in strict level order)
+ *   orc_level_buckets / orc_class_order   index arrays of the graph-prep pass, from their definitions
+ *
+ * Pins (tests that do not restate these loops): dense masked softmax attention by a library routine on
+ * tiny graphs; boolean adjacency powers for the neighbourhoods; closed forms (self-only node returns its
+ * V row, equal scores give the mean, scores {0, ln 3} give weights 1/4 and 3/4, complete binary in-tree
+ * gives 3 / 7 members); invariants (weights sum to 1, neighbour-order invariance, convex hull);
+ * levelised == parallel replayed bucket by bucket.
+ * The paper prints no worked numerical example, so no printed value pins the numbers: parity of the
+ * numerical values is pinned only by those definitions and invariants.
+ */
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <set>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+extern "C" {
+
+/* Round an fp64 value to the nearest bfloat16 (8 significant bits, ties to even), returned as fp64.
+ * Used only where a tensor is *stored* in bfloat16 by the layer's interface. */
+double orc_round_bf16(double x) {
+    if (x == 0.0 || !std::isfinite(x)) return x;
+    int e = std::ilogb(x);                 /* x = m * 2^e, 1 <= |m| < 2 */
+    if (e < -126) e = -126;                /* below the smallest normal: fixed quantum */
+    double q = std::ldexp(1.0, e - 7);     /* spacing of bfloat16 numbers in this binade */
+    double r = std::nearbyint(x / q) * q;  /* default rounding mode: to nearest, ties to even */
+    if (std::fabs(r) > 3.3895313892515355e38) r = std::copysign(INFINITY, x);
+    return r;
+}
+
+void orc_round_bf16_array(const double* in, double* out, int64_t cnt) {
+    for (int64_t i = 0; i < cnt; ++i) out[i] = orc_round_bf16(in[i]);
+}
+
+double orc_round_f32(double x) { return (double)(float)x; }
+
+static inline double store_round(double x, int rounding) {
+    if (rounding == 1) return orc_round_bf16(x);
+    if (rounding == 2) return orc_round_f32(x);
+    return x;
+}
+
+/* Eq. 1.  Nodes are visited in id order, which must be a topological order (every source id < its
+ * destination id); returns -1 if it is not. */
+int orc_levels(int n, const int32_t* row_ptr, const int32_t* col_idx, int32_t* level) {
+    for (int v = 0; v < n; ++v) {
+        int lv = 0;
+        for (int e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            int u = col_idx[e];
+            if (u < 0 || u >= v) return -1;
+            lv = std::max(lv, level[u] + 1);
+        }
+        level[v] = lv;
+    }
+    return 0;
+}
+
+/* cone_k(v) as a list: v first, then the other members in ascending id.  Call with nbr_idx == NULL to
+ * get only nbr_ptr (sizes).  Returns the total number of entries. */
+int64_t orc_neighbourhood(int n, const int32_t* row_ptr, const int32_t* col_idx, int hops,
+                          int32_t* nbr_ptr, int32_t* nbr_idx) {
+    int64_t total = 0;
+    for (int v = 0; v < n; ++v) {
+        std::set<int> cone;              /* members other than v */
+        std::set<int> frontier = {v};
+        for (int step = 0; step < hops; ++step) {
+            std::set<int> next;
+            for (int w : frontier)
+                for (int e = row_ptr[w]; e < row_ptr[w + 1]; ++e) next.insert(col_idx[e]);
+            for (int u : next) cone.insert(u);
+            frontier = next;
+        }
+        cone.erase(v);                   /* a DAG never puts v here; kept for safety */
+        nbr_ptr[v] = (int32_t)total;
+        if (nbr_idx) {
+            nbr_idx[total] = v;
+            int64_t k = total + 1;
+            for (int u : cone) nbr_idx[k++] = u;
+        }
+        total += 1 + (int64_t)cone.size();
+    }
+    nbr_ptr[n] = (int32_t)total;
+    return total;
+}
+
+/* Level buckets: nodes ordered by (level, id).  level_ptr has n_levels + 1 entries. */
+int orc_level_buckets(int n, const int32_t* level, int n_levels, int32_t* level_ptr, int32_t* level_nodes) {
+    std::vector<int32_t> order(n);
+    for (int v = 0; v < n; ++v) order[v] = v;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return level[a] < level[b]; });
+    for (int v = 0; v < n; ++v) level_nodes[v] = order[v];
+    /* level_ptr[l] = number of nodes whose level is below l = first position in the sorted order
+     * whose level is >= l */
+    std::vector<int32_t> sorted_level(n);
+    for (int i = 0; i < n; ++i) sorted_level[i] = level[order[i]];
+    for (int l = 0; l <= n_levels; ++l)
+        level_ptr[l] = (int32_t)(std::lower_bound(sorted_level.begin(), sorted_level.end(), l) - sorted_level.begin());
+    return 0;
+}
+
+/* Degree-class order inside segments.  The nodes are given as a sequence seq[0..n) cut into n_seg
+ * consecutive segments seg_ptr[s]..seg_ptr[s+1].  Inside each segment the nodes are reordered by
+ * (class, id) where class(v) = nbr_ptr[v+1] - nbr_ptr[v] (1..max_class).
+ * class_ptr[s*(max_class+1) + c] = position in `perm` where class c+1 of segment s starts
+ * (c = 0..max_class-1); entry c = max_class is the end of the segment. */
+int orc_class_order(int n, const int32_t* seq, int n_seg, const int32_t* seg_ptr, const int32_t* nbr_ptr,
+                    int max_class, int32_t* perm, int32_t* class_ptr) {
+    (void)n;
+    for (int s = 0; s < n_seg; ++s) {
+        int lo = seg_ptr[s], hi = seg_ptr[s + 1];
+        std::vector<int32_t> nodes(seq + lo, seq + hi);
+        auto cls = [&](int v) { return nbr_ptr[v + 1] - nbr_ptr[v]; };
+        std::sort(nodes.begin(), nodes.end(), [&](int a, int b) {
+            if (cls(a) != cls(b)) return cls(a) < cls(b);
+            return a < b;
+        });
+        for (int i = lo; i < hi; ++i) perm[i] = nodes[i - lo];
+        for (int c = 0; c <= max_class; ++c) {
+            int cnt = 0;
+            for (int v : nodes) cnt += (cls(v) < c + 1);
+            class_ptr[(int64_t)s * (max_class + 1) + c] = lo + cnt;
+        }
+    }
+    return 0;
+}
+
+/* One node, one head of the restricted attention.  q: d_head values; krows[j], vrows[j]: the head's
+ * slice of neighbour j's key / value row.  alpha (optional) receives the softmax weights. */
+static void attend_one(int d_head, double scale, const double* q, int cnt,
+                       const double* const* krows, const double* const* vrows, double* out, double* alpha) {
+    std::vector<double> s(cnt), a(cnt);
+    for (int j = 0; j < cnt; ++j) {
+        double dot = 0.0;
+        for (int c = 0; c < d_head; ++c) dot += q[c] * krows[j][c];
+        s[j] = scale * dot;
+    }
+    double m = s[0];
+    for (int j = 1; j < cnt; ++j) m = std::max(m, s[j]);
+    double z = 0.0;
+    for (int j = 0; j < cnt; ++j) { a[j] = std::exp(s[j] - m); z += a[j]; }
+    for (int j = 0; j < cnt; ++j) a[j] /= z;
+    for (int c = 0; c < d_head; ++c) {
+        double acc = 0.0;
+        for (int j = 0; j < cnt; ++j) acc += a[j] * vrows[j][c];
+        out[c] = acc;
+    }
+    if (alpha) for (int j = 0; j < cnt; ++j) alpha[j] = a[j];
+}
+
+/* Attention of every node over its neighbour list.  Q, O: [n, d]; K, V: [n_kv, d] row-major,
+ * d = heads * d_head; neighbour ids index K and V.  alpha (optional): [nbr_ptr[n], heads]. */
+void orc_attention(int n, int d, int heads, double scale, const double* Q, const double* K, const double* V,
+                   const int32_t* nbr_ptr, const int32_t* nbr_idx, double* O, double* alpha) {
+    int dh = d / heads;
+#pragma omp parallel for schedule(static)
+    for (int v = 0; v < n; ++v) {
+        int lo = nbr_ptr[v], cnt = nbr_ptr[v + 1] - lo;
+        std::vector<const double*> kr(cnt), vr(cnt);
+        std::vector<double> a(cnt);
+        for (int h = 0; h < heads; ++h) {
+            for (int j = 0; j < cnt; ++j) {
+                int64_t u = nbr_idx[lo + j];
+                kr[j] = K + u * d + h * dh;
+                vr[j] = V + u * d + h * dh;
+            }
+            attend_one(dh, scale, Q + (int64_t)v * d + h * dh, cnt, kr.data(), vr.data(),
+                       O + (int64_t)v * d + h * dh, alpha ? a.data() : nullptr);
+            if (alpha) for (int j = 0; j < cnt; ++j) alpha[(int64_t)(lo + j) * heads + h] = a[j];
+        }
+    }
+}
+
+static void project_row(int d_in, int d_out, const double* x, const double* W, const double* r, double* y) {
+    for (int o = 0; o < d_out; ++o) {
+        double acc = 0.0;
+        for (int c = 0; c < d_in; ++c) acc += x[c] * W[(int64_t)o * d_in + c];
+        if (r) acc += r[o];
+        y[o] = acc;
+    }
+}
+
+/* Y[n, d_out] = X[n, d_in] * W[d_out, d_in]^T  (+ R[n, d_out] if R != NULL). */
+void orc_project(int n, int d_in, int d_out, const double* X, const double* W, const double* R, double* Y) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < n; ++i)
+        project_row(d_in, d_out, X + (int64_t)i * d_in, W, R ? R + (int64_t)i * d_out : nullptr,
+                    Y + (int64_t)i * d_out);
+}
+
+static void round_all(double* a, int64_t cnt, int rounding) {
+    if (!rounding) return;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < cnt; ++i) a[i] = store_round(a[i], rounding);
+}
+
+/* All-nodes-parallel layer.  W_qkv: [3d, d] (rows 0..d-1 -> Q, d..2d-1 -> K, 2d..3d-1 -> V), W_o: [d, d].
+ * rounding: 0 none, 1 = every stored tensor (Q, K, V, O, H_out) rounded to bfloat16, 2 = to fp32. */
+void orc_layer_parallel(int n, int d, int heads, double scale, const double* X, const double* W_qkv,
+                        const double* W_o, int residual, const int32_t* nbr_ptr, const int32_t* nbr_idx,
+                        int rounding, double* H_out) {
+    int64_t nd = (int64_t)n * d;
+    std::vector<double> Q(nd), K(nd), V(nd), O(nd);
+    orc_project(n, d, d, X, W_qkv, nullptr, Q.data());
+    orc_project(n, d, d, X, W_qkv + (int64_t)d * d, nullptr, K.data());
+    orc_project(n, d, d, X, W_qkv + (int64_t)2 * d * d, nullptr, V.data());
+    round_all(Q.data(), nd, rounding); round_all(K.data(), nd, rounding); round_all(V.data(), nd, rounding);
+    orc_attention(n, d, heads, scale, Q.data(), K.data(), V.data(), nbr_ptr, nbr_idx, O.data(), nullptr);
+    round_all(O.data(), nd, rounding);
+    orc_project(n, d, d, O.data(), W_o, residual ? X : nullptr, H_out);
+    round_all(H_out, nd, rounding);
+}
+
+/* Levelised layer, in place on H.  Buckets l = 0..n_levels-1 are processed in order; a node v of bucket l
+ * takes its query and its own key/value from its current (not yet updated) row, and the key/value of every
+ * other neighbour u from u's row as already updated in this sweep (u lies on a strictly lower level).
+ * Nodes of one bucket do not read one another, so their new rows are committed together. */
+void orc_layer_levelised(int n, int d, int heads, double scale, double* H, const double* W_qkv,
+                         const double* W_o, int residual, const int32_t* nbr_ptr, const int32_t* nbr_idx,
+                         int n_levels, const int32_t* level_ptr, const int32_t* level_nodes, int rounding) {
+    (void)n;
+    int dh = d / heads;
+    const double* Wq = W_qkv;
+    const double* Wk = W_qkv + (int64_t)d * d;
+    const double* Wv = W_qkv + (int64_t)2 * d * d;
+    for (int l = 0; l < n_levels; ++l) {
+        int lo = level_ptr[l], hi = level_ptr[l + 1];
+        std::vector<double> fresh((int64_t)(hi - lo) * d);
+#pragma omp parallel for schedule(static)
+        for (int i = lo; i < hi; ++i) {
+            int v = level_nodes[i];
+            int b = nbr_ptr[v], cnt = nbr_ptr[v + 1] - b;
+            std::vector<double> q(d), kk((int64_t)cnt * d), vv((int64_t)cnt * d), o(d);
+            project_row(d, d, H + (int64_t)v * d, Wq, nullptr, q.data());
+            for (int j = 0; j < cnt; ++j) {
+                int64_t u = nbr_idx[b + j];
+                project_row(d, d, H + u * d, Wk, nullptr, kk.data() + (int64_t)j * d);
+                project_row(d, d, H + u * d, Wv, nullptr, vv.data() + (int64_t)j * d);
+            }
+            for (int c = 0; c < d; ++c) q[c] = store_round(q[c], rounding);
+            for (int64_t c = 0; c < (int64_t)cnt * d; ++c) {
+                kk[c] = store_round(kk[c], rounding);
+                vv[c] = store_round(vv[c], rounding);
+            }
+            std::vector<const double*> kr(cnt), vr(cnt);
+            for (int h = 0; h < heads; ++h) {
+                for (int j = 0; j < cnt; ++j) {
+                    kr[j] = kk.data() + (int64_t)j * d + h * dh;
+                    vr[j] = vv.data() + (int64_t)j * d + h * dh;
+                }
+                attend_one(dh, scale, q.data() + h * dh, cnt, kr.data(), vr.data(), o.data() + h * dh, nullptr);
+            }
+            for (int c = 0; c < d; ++c) o[c] = store_round(o[c], rounding);
+            double* dst = fresh.data() + (int64_t)(i - lo) * d;
+            project_row(d, d, o.data(), W_o, residual ? H + (int64_t)v * d : nullptr, dst);
+            for (int c = 0; c < d; ++c) dst[c] = store_round(dst[c], rounding);
+        }
+        for (int i = lo; i < hi; ++i)
+            std::memcpy(H + (int64_t)level_nodes[i] * d, fresh.data() + (int64_t)(i - lo) * d, sizeof(double) * d);
+    }
+}
+
+int orc_num_threads(void) {
+    int t = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        t = omp_get_num_threads();
+    }
+#endif
+    return t;
+}
+
+}  /* extern "C" */
