@@ -1,0 +1,197 @@
+/*
+ * dg4 -- fused sparse attention over And-Inverter Graphs for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libdg4.so.  One GPU per handle.  The caller owns every tensor and the
+ * stream; the library owns only what hangs off a dg4_graph.  Forward calls enqueue
+ * work on the given stream and return; they never allocate, never synchronise and
+ * never block without bound.  Argument errors are returned synchronously; nothing
+ * throws, aborts or traps.
+ *
+ * Paper: DeepGate4 (arXiv 2502.01681).  Passages are cited by section / equation.
+ *
+ * Conventions
+ *   - "host" / "device" in a comment says where a pointer must live.
+ *   - Tensors are row-major [rows, d] with a leading dimension `ld*` in ELEMENTS.
+ *     Base pointers must be 16-byte aligned and ld * sizeof(element) a multiple
+ *     of 16 bytes, otherwise DG4_ERR_INVALID_ARG.
+ *   - d = 128 only.  heads in {1, 2, 4, 8, 16}.  Attention: fp32 or bf16 storage,
+ *     fp32 arithmetic.  Projections: bf16 storage, fp32 accumulation.
+ *     Anything else returns DG4_ERR_UNSUPPORTED (there is no fallback path).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef DG4_H
+#define DG4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DG4_OK = 0,
+    DG4_ERR_INVALID_ARG = -1,  /* null pointer, bad size, bad alignment                      */
+    DG4_ERR_NOT_SORTED  = -2,  /* row_ptr not starting at 0 / not non-decreasing              */
+    DG4_ERR_BAD_DEGREE  = -3,  /* a node with more than two fan-ins                           */
+    DG4_ERR_BAD_LEVEL   = -4,  /* an edge (u, v) with level[u] >= level[v], or a source id
+                                  out of range, or a negative level                           */
+    DG4_ERR_UNSUPPORTED = -5,  /* d, heads, dtype or hops outside the supported set           */
+    DG4_ERR_ALLOC       = -6,  /* device or host allocation failed                            */
+    DG4_ERR_CUDA        = -7,  /* a CUDA runtime call failed; see dg4_last_error()            */
+    DG4_ERR_TIMEOUT     = -8   /* a bounded device-side wait ran out                          */
+} dg4_status;
+
+typedef enum { DG4_F32 = 0, DG4_BF16 = 1 } dg4_dtype;
+
+enum {
+    DG4_FLAG_RESIDUAL = 1      /* output projection adds the layer's input row                */
+};
+
+/* Per-call description of the attention layer. */
+typedef struct {
+    int32_t d;                 /* model width; 128                                            */
+    int32_t heads;             /* number of heads; d_head = d / heads                         */
+    int32_t dtype;             /* dg4_dtype of Q, K, V, O (and of X, H, weights)              */
+    int32_t flags;             /* DG4_FLAG_*                                                  */
+    float   scale;             /* multiplies every dot-product score, e.g. 1/sqrt(d_head)     */
+} dg4_desc;
+
+typedef struct dg4_graph dg4_graph;   /* opaque; device-resident index arrays of one circuit */
+
+typedef struct {
+    int64_t n_nodes;
+    int64_t n_edges;
+    int64_t n_nbr;             /* total neighbourhood entries, sum over v of |N(v)|           */
+    int32_t n_levels;          /* 1 + max level                                               */
+    int32_t max_class;         /* 2^(hops+1) - 1: upper bound of |N(v)|                       */
+    int32_t hops;
+    int32_t perm_chunk;        /* chunk length of the degree-class permutation (0 = global)   */
+    int32_t n_chunks;
+    int32_t device;
+} dg4_graph_info_t;
+
+/* Index arrays a graph handle holds (all int32), for dg4_graph_export. */
+typedef enum {
+    DG4_ARR_NBR_PTR = 0,        /* [n+1]                 start of N(v) in NBR_IDX                        */
+    DG4_ARR_NBR_IDX = 1,        /* [n_nbr]               members of N(v): v first, the rest ascending    */
+    DG4_ARR_LEVEL_PTR = 2,      /* [n_levels+1]          start of level l in LEVEL_NODES                 */
+    DG4_ARR_LEVEL_NODES = 3,    /* [n]                   node ids ordered by (level, id)                 */
+    DG4_ARR_PERM = 4,           /* [n]                   ids ordered by (chunk, |N(v)|, id)              */
+    DG4_ARR_CLASS_PTR = 5,      /* [n_chunks, max_class+1]  start of class c+1 of a chunk in PERM;
+                                                         last entry of a row = end of the chunk        */
+    DG4_ARR_LEVEL_PERM = 6,     /* [n]                   ids ordered by (level, |N(v)|, id)              */
+    DG4_ARR_LEVEL_CLASS_PTR = 7 /* [n_levels, max_class+1]  same as CLASS_PTR with levels as segments    */
+} dg4_array_id;
+
+const char* dg4_status_string(dg4_status s);
+/* Detail of the last error on the calling thread ("" if none).  Valid until the next failing call. */
+const char* dg4_last_error(void);
+
+/*
+ * Graph prep.  Sec. 3.2: node kinds are told apart by in-degree (0 primary input, 1 NOT, 2 AND); Eq. 1
+ * defines the logic level; cone_k(v) = { u : a path u -> v of length <= k } with v included, at most
+ * 2^(k+1)-1 members.  Sec. 3.5 restricts attention to that set (the "virtual edges").
+ *
+ * Validates the circuit on the host, uploads it, and builds on the device:
+ *   the neighbourhood lists N(v) = cone_hops(v) as a CSR (v first, then ascending id, duplicates
+ *   collapsed), the level buckets, and the degree-class orderings (stable by (segment, |N(v)|, id),
+ *   segments = consecutive id chunks of perm_chunk nodes, and = levels).
+ *
+ *   n_nodes     >= 1
+ *   row_ptr     host, [n_nodes+1], destination-sorted CSR of DIRECT fan-ins (no self entry)
+ *   col_idx     host, [row_ptr[n_nodes]], source ids; any order inside a row; a repeated source is allowed
+ *   level       host, [n_nodes]; any layering with level[u] < level[v] on every edge is accepted
+ *   hops        1 (fan-ins + self) or 2 (2-hop fan-in cone + self)
+ *   perm_chunk  0 (one chunk) or a positive multiple of 1024
+ *   device      CUDA ordinal; made current for the duration of the call and restored
+ *   out         receives the handle; untouched on error
+ *
+ * Allocates device memory and synchronises; not for use inside a timed or captured region.
+ * Errors: INVALID_ARG, NOT_SORTED, BAD_DEGREE, BAD_LEVEL, UNSUPPORTED, ALLOC, CUDA.
+ */
+dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, const int32_t* col_idx,
+                            const int32_t* level, int32_t hops, int32_t perm_chunk, int32_t device,
+                            dg4_graph** out);
+
+/* Re-runs the device part of graph prep (neighbourhoods, buckets, class orderings) from the circuit the
+ * handle already holds, on `stream`, reusing the handle's buffers.  Asynchronous; allocates nothing.
+ * The arrays are unchanged in content; this entry exists so the device pass can be timed on its own. */
+dg4_status dg4_graph_rebuild(dg4_graph* g, void* stream);
+
+dg4_status dg4_graph_destroy(dg4_graph* g);     /* NULL is accepted */
+dg4_status dg4_graph_info(const dg4_graph* g, dg4_graph_info_t* out);
+
+/* Copies one index array to the host (synchronises the device).  host_dst may be NULL to query the
+ * length only.  capacity and *n_written count int32 elements.  INVALID_ARG if capacity is too small. */
+dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, int32_t* host_dst, int64_t capacity,
+                            int64_t* n_written);
+
+/* Device pointer to one index array (owned by the handle, valid until destroy); NULL on bad arguments. */
+const int32_t* dg4_graph_device_array(const dg4_graph* g, dg4_array_id which);
+
+/*
+ * QKV projection: [Q | K | V] = X * W_qkv^T for every node (Sec. 3.5: the Transformer block is kept and
+ * only its attention is restricted, so the block's dense projections stay).
+ *   X      device, [n, d] bf16, leading dimension ldx
+ *   W_qkv  device, [3d, d] bf16 row-major (output-major): rows 0..d-1 give Q, d..2d-1 K, 2d..3d-1 V
+ *   Q,K,V  device, [n, d] bf16 each.  K and V may interleave in one [n, 2d] buffer (V = K + d, ldk = ldv = 2d).
+ * fp32 accumulation, one rounding to bf16 per stored element.  UNSUPPORTED unless desc->dtype is bf16.
+ */
+dg4_status dg4_qkv_project(const dg4_graph* g, const dg4_desc* desc,
+                           const void* X, int64_t ldx, const void* W_qkv,
+                           void* Q, int64_t ldq, void* K, int64_t ldk, void* V, int64_t ldv, void* stream);
+
+/*
+ * Fused sparse attention (Sec. 3.5; kernel mapping informed by Sec. 3.7's remarks on low in-degree):
+ * for every node v and head h,
+ *     s_u = scale * <Q[v,h,:], K[u,h,:]>  for u in N(v),   alpha = softmax_u(s),   O[v,h,:] = sum_u alpha_u V[u,h,:]
+ * Scores live in registers only; no per-edge tensor is written.  fp32 arithmetic; O rounded once on store.
+ *   Q, K, V  device, [n, d] of desc->dtype;   O  device, [n, d], must not alias K or V.
+ */
+dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* desc,
+                               const void* Q, int64_t ldq, const void* K, int64_t ldk,
+                               const void* V, int64_t ldv, void* O, int64_t ldo, void* stream);
+
+/*
+ * Output projection: H_out = O * W_o^T (+ H_res if desc->flags has DG4_FLAG_RESIDUAL and H_res != NULL).
+ *   O device [n, d] bf16;  W_o device [d, d] bf16 (output-major);  H_res device [n, d] bf16 or NULL;
+ *   H_out device [n, d] bf16; may alias H_res (each row is read before it is written by the same thread).
+ */
+dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc,
+                           const void* O, int64_t ldo, const void* W_o,
+                           const void* H_res, int64_t ldh, void* H_out, int64_t ldho, void* stream);
+
+/* Bytes of caller-provided device workspace the two layer calls need for this graph (256-byte aligned base). */
+size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* desc);
+
+/*
+ * One layer for all nodes at once: QKV projection -> sparse attention -> output projection (+ residual),
+ * every node reading the same input H_in.   H_in, H_out: device [n, d] bf16; they may be the same buffer
+ * only if ldh == ldho (rows are then updated in place after all reads of the layer's input are done).
+ */
+dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc* desc,
+                                  const void* H_in, int64_t ldh, const void* W_qkv, const void* W_o,
+                                  void* H_out, int64_t ldho, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/*
+ * One layer in the paper's level-by-level order (Sec. 1 and Sec. 3.4: gates are encoded in strict
+ * topological order and each gate is computed once).  Levels 0, 1, ... are processed in turn; a node
+ * takes its query and its own key/value from its row as it was when the call started, and the key/value
+ * of every other member of N(v) (all on lower levels) from that node's row as already updated by this
+ * call.  H is updated in place.
+ *   H              device, [n, d] bf16, leading dimension ldh
+ *   workspace      device, at least dg4_layer_workspace_bytes() bytes
+ *   device_status  device int32 or NULL; receives a dg4_status (0, or DG4_ERR_TIMEOUT if a bounded
+ *                  device-side wait ran out; the call still returns and the context stays usable)
+ */
+dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc* desc,
+                                   void* H, int64_t ldh, const void* W_qkv, const void* W_o,
+                                   void* workspace, size_t workspace_bytes,
+                                   int32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DG4_H */

@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libdg4.so (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdarg.h>
+
+#include "dg4.h"
+
+// ---- error plumbing -------------------------------------------------------------------------
+void dg4_set_error(const char* fmt, ...);
+
+#define DG4_CUDA_TRY(expr)                                                                   \
+    do {                                                                                     \
+        cudaError_t _e = (expr);                                                             \
+        if (_e != cudaSuccess) {                                                             \
+            dg4_set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(_e), __FILE__, __LINE__); \
+            return (_e == cudaErrorMemoryAllocation) ? DG4_ERR_ALLOC : DG4_ERR_CUDA;         \
+        }                                                                                    \
+    } while (0)
+
+#define DG4_FAIL(code, ...)          \
+    do {                             \
+        dg4_set_error(__VA_ARGS__);  \
+        return (code);               \
+    } while (0)
+
+// ---- the graph handle -----------------------------------------------------------------------
+struct dg4_graph {
+    int32_t device = 0;
+    int32_t n = 0;            // nodes
+    int64_t e = 0;            // direct fan-in edges
+    int64_t n_nbr = 0;        // neighbourhood entries
+    int32_t n_levels = 0;
+    int32_t hops = 0;
+    int32_t max_class = 0;
+    int32_t perm_chunk = 0;   // 0 = one chunk
+    int32_t n_chunks = 1;
+
+    // circuit as uploaded
+    int32_t* row_ptr = nullptr;   // [n+1]
+    int32_t* col_idx = nullptr;   // [e]
+    int32_t* level = nullptr;     // [n]
+    // built by graph prep
+    int32_t* nbr_ptr = nullptr;          // [n+1]
+    int32_t* nbr_idx = nullptr;          // [n_nbr]
+    int32_t* level_ptr = nullptr;        // [n_levels+1]
+    int32_t* level_nodes = nullptr;      // [n]
+    int32_t* perm = nullptr;             // [n]
+    int32_t* class_ptr = nullptr;        // [n_chunks*(max_class+1)]
+    int32_t* level_perm = nullptr;       // [n]
+    int32_t* level_class_ptr = nullptr;  // [n_levels*(max_class+1)]
+    // scratch of graph prep (kept so that a rebuild allocates nothing)
+    int32_t* seq_a = nullptr;            // [n]
+    int32_t* seq_b = nullptr;            // [n]
+    int32_t* hist = nullptr;             // [hist_len]
+    int32_t* block_sums = nullptr;       // [block_sums_len]
+    int64_t hist_len = 0;
+    int64_t block_sums_len = 0;
+    // host copy of the level boundaries (the levelised driver launches per level)
+    int32_t* h_level_ptr = nullptr;      // [n_levels+1]
+};
+
+// ---- kernels' host launchers (each enqueues on `st` and returns) -----------------------------
+dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only);
+
+struct dg4i_attn_args {
+    const void* Q; int64_t ldq;
+    const void* K; int64_t ldk;
+    const void* V; int64_t ldv;
+    void* O; int64_t ldo;
+    const int32_t* nbr_ptr;
+    const int32_t* nbr_idx;
+    const int32_t* node_list;   // nullable: node ids to process; else ids first..first+count-1
+    int32_t first;
+    int32_t count;
+    int32_t heads;
+    int32_t max_nbr;            // 3 or 7
+    int32_t dtype;
+    float scale;
+};
+dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st);
+
+// Y[r, 0:n_out] = A[r, 0:128] * W[0:n_out, 0:128]^T (+ R[r, :]) for rows r of a list (or 0..rows-1).
+// Output column block j (of 128) goes to out[j] with leading dimension ldo[j].
+struct dg4i_proj_args {
+    const __nv_bfloat16* A; int64_t lda;
+    const __nv_bfloat16* W;            // [n_out, 128] row-major
+    int32_t n_out;                     // 128, 256 or 384
+    __nv_bfloat16* out[3]; int64_t ldo[3];
+    const __nv_bfloat16* R; int64_t ldr;   // nullable residual, added to column block 0 only
+    const int32_t* row_list;           // nullable
+    int32_t first;                     // offset into row_list (or first row id)
+    int32_t rows;
+};
+dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st);

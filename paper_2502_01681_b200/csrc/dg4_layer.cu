@@ -1,0 +1,231 @@
+// Public forward entry points: argument checks, then launches on the caller's stream.
+// The all-parallel layer is QKV projection -> sparse attention -> output projection over all nodes.
+// The levelised layer (Sec. 1 / Sec. 3.4: strict topological order, each gate computed once) projects
+// Q|K|V of every node from the layer's input once -- a node's own query, key and value always come from
+// its row as it was at the start of the layer -- and then, level by level, runs the attention for that
+// level's nodes, writes their new rows, and refreshes their K|V rows so that higher levels gather the
+// updated ones.
+
+#include "dg4_internal.h"
+
+#include <string.h>
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+
+dg4_status check_desc(const dg4_desc* d, bool need_bf16) {
+    if (!d) DG4_FAIL(DG4_ERR_INVALID_ARG, "null descriptor");
+    if (d->d != 128) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d = %d: only d = 128 is supported", d->d);
+    if (d->dtype != DG4_F32 && d->dtype != DG4_BF16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "unknown dtype %d", d->dtype);
+    if (need_bf16 && d->dtype != DG4_BF16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "projections are bf16 only");
+    const int lanes = d->dtype == DG4_BF16 ? 16 : 32;
+    if (d->heads < 1 || d->heads > lanes || (lanes % d->heads) != 0)
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must be a power of two up to %d", d->heads, lanes);
+    if (!(d->scale == d->scale) || d->scale > 3.0e38f || d->scale < -3.0e38f)
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "scale is not finite");
+    return DG4_OK;
+}
+
+dg4_status check_tensor(const char* name, const void* p, int64_t ld, int elem_size, int min_ld) {
+    if (!p) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is null", name);
+    if (!aligned16(p)) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    if (ld < min_ld) DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimension of %s (%lld) is below %d", name, (long long)ld, min_ld);
+    if ((ld * elem_size) % 16 != 0)
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimension of %s (%lld elements) is not a multiple of 16 bytes", name, (long long)ld);
+    return DG4_OK;
+}
+
+#define CHECK(expr) do { dg4_status _s = (expr); if (_s != DG4_OK) return _s; } while (0)
+
+struct Workspace {
+    __nv_bfloat16* Q;    // [n, 128]
+    __nv_bfloat16* KV;   // [n, 256]: K | V interleaved per node (one 512-byte stretch per neighbour)
+    __nv_bfloat16* O;    // [n, 128]
+};
+
+size_t workspace_bytes(int64_t n) { return (size_t)n * 128 * 2 * 4 + 256; }
+
+Workspace carve(void* ws, int64_t n) {
+    Workspace w;
+    char* p = (char*)ws;
+    w.Q = (__nv_bfloat16*)p;
+    w.KV = (__nv_bfloat16*)(p + (size_t)n * 256);
+    w.O = (__nv_bfloat16*)(p + (size_t)n * 768);
+    return w;
+}
+
+dg4i_attn_args attn_args(const dg4_graph* g, const dg4_desc* d, const void* Q, int64_t ldq, const void* K,
+                         int64_t ldk, const void* V, int64_t ldv, void* O, int64_t ldo) {
+    dg4i_attn_args a;
+    a.Q = Q; a.ldq = ldq; a.K = K; a.ldk = ldk; a.V = V; a.ldv = ldv; a.O = O; a.ldo = ldo;
+    a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.heads = d->heads; a.max_nbr = g->max_class; a.dtype = d->dtype; a.scale = d->scale;
+    return a;
+}
+
+}  // namespace
+
+void dg4_set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+extern "C" const char* dg4_last_error(void) { return g_err; }
+
+extern "C" const char* dg4_status_string(dg4_status s) {
+    switch (s) {
+        case DG4_OK: return "ok";
+        case DG4_ERR_INVALID_ARG: return "invalid argument";
+        case DG4_ERR_NOT_SORTED: return "CSR is not sorted by destination";
+        case DG4_ERR_BAD_DEGREE: return "node with more than two fan-ins";
+        case DG4_ERR_BAD_LEVEL: return "levels do not increase along an edge";
+        case DG4_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DG4_ERR_ALLOC: return "allocation failed";
+        case DG4_ERR_CUDA: return "CUDA error";
+        case DG4_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+extern "C" dg4_status dg4_qkv_project(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
+                                       const void* W_qkv, void* Q, int64_t ldq, void* K, int64_t ldk, void* V,
+                                       int64_t ldv, void* stream) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(check_desc(desc, true));
+    CHECK(check_tensor("X", X, ldx, 2, 128));
+    CHECK(check_tensor("W_qkv", W_qkv, 128, 2, 128));
+    CHECK(check_tensor("Q", Q, ldq, 2, 128));
+    CHECK(check_tensor("K", K, ldk, 2, 128));
+    CHECK(check_tensor("V", V, ldv, 2, 128));
+    dg4i_proj_args a;
+    a.A = (const __nv_bfloat16*)X; a.lda = ldx; a.W = (const __nv_bfloat16*)W_qkv; a.n_out = 384;
+    a.out[0] = (__nv_bfloat16*)Q; a.ldo[0] = ldq;
+    a.out[1] = (__nv_bfloat16*)K; a.ldo[1] = ldk;
+    a.out[2] = (__nv_bfloat16*)V; a.ldo[2] = ldv;
+    a.R = nullptr; a.ldr = 0; a.row_list = nullptr; a.first = 0; a.rows = g->n;
+    return dg4i_proj_launch(a, (cudaStream_t)stream);
+}
+
+extern "C" dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* desc, const void* Q, int64_t ldq,
+                                           const void* K, int64_t ldk, const void* V, int64_t ldv, void* O,
+                                           int64_t ldo, void* stream) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(check_desc(desc, false));
+    const int es = desc->dtype == DG4_BF16 ? 2 : 4;
+    CHECK(check_tensor("Q", Q, ldq, es, 128));
+    CHECK(check_tensor("K", K, ldk, es, 128));
+    CHECK(check_tensor("V", V, ldv, es, 128));
+    CHECK(check_tensor("O", O, ldo, es, 128));
+    if (O == K || O == V) DG4_FAIL(DG4_ERR_INVALID_ARG, "O must not alias K or V");
+    return dg4i_attn_launch(attn_args(g, desc, Q, ldq, K, ldk, V, ldv, O, ldo), (cudaStream_t)stream);
+}
+
+extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, const void* O, int64_t ldo,
+                                       const void* W_o, const void* H_res, int64_t ldh, void* H_out, int64_t ldho,
+                                       void* stream) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(check_desc(desc, true));
+    CHECK(check_tensor("O", O, ldo, 2, 128));
+    CHECK(check_tensor("W_o", W_o, 128, 2, 128));
+    CHECK(check_tensor("H_out", H_out, ldho, 2, 128));
+    const bool res = (desc->flags & DG4_FLAG_RESIDUAL) && H_res;
+    if (res) CHECK(check_tensor("H_res", H_res, ldh, 2, 128));
+    if (H_out == O) DG4_FAIL(DG4_ERR_INVALID_ARG, "H_out must not alias O");
+    dg4i_proj_args a;
+    a.A = (const __nv_bfloat16*)O; a.lda = ldo; a.W = (const __nv_bfloat16*)W_o; a.n_out = 128;
+    a.out[0] = (__nv_bfloat16*)H_out; a.ldo[0] = ldho; a.out[1] = a.out[2] = nullptr; a.ldo[1] = a.ldo[2] = 0;
+    a.R = res ? (const __nv_bfloat16*)H_res : nullptr; a.ldr = ldh; a.row_list = nullptr; a.first = 0; a.rows = g->n;
+    return dg4i_proj_launch(a, (cudaStream_t)stream);
+}
+
+extern "C" size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* desc) {
+    (void)desc;
+    return g ? workspace_bytes(g->n) : 0;
+}
+
+namespace {
+dg4_status check_layer_args(const dg4_graph* g, const dg4_desc* desc, const void* H, int64_t ldh, const void* W_qkv,
+                            const void* W_o, void* ws, size_t ws_bytes) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(check_desc(desc, true));
+    CHECK(check_tensor("H", H, ldh, 2, 128));
+    CHECK(check_tensor("W_qkv", W_qkv, 128, 2, 128));
+    CHECK(check_tensor("W_o", W_o, 128, 2, 128));
+    if (!ws) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
+    if ((((uintptr_t)ws) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+    if (ws_bytes < workspace_bytes(g->n))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", ws_bytes, workspace_bytes(g->n));
+    return DG4_OK;
+}
+}  // namespace
+
+extern "C" dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, const void* H_in, int64_t ldh,
+                                              const void* W_qkv, const void* W_o, void* H_out, int64_t ldho,
+                                              void* workspace, size_t workspace_bytes_, void* stream) {
+    CHECK(check_layer_args(g, desc, H_in, ldh, W_qkv, W_o, workspace, workspace_bytes_));
+    CHECK(check_tensor("H_out", H_out, ldho, 2, 128));
+    if (H_out == H_in && ldh != ldho) DG4_FAIL(DG4_ERR_INVALID_ARG, "in-place use needs equal leading dimensions");
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w = carve(workspace, g->n);
+
+    dg4i_proj_args p;
+    p.A = (const __nv_bfloat16*)H_in; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
+    p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n;
+    CHECK(dg4i_proj_launch(p, st));
+
+    CHECK(dg4i_attn_launch(attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128), st));
+
+    dg4i_proj_args o;
+    o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
+    o.out[0] = (__nv_bfloat16*)H_out; o.ldo[0] = ldho; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
+    o.R = (desc->flags & DG4_FLAG_RESIDUAL) ? (const __nv_bfloat16*)H_in : nullptr; o.ldr = ldh;
+    o.row_list = nullptr; o.first = 0; o.rows = g->n;
+    return dg4i_proj_launch(o, st);
+}
+
+extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                               const void* W_qkv, const void* W_o, void* workspace,
+                                               size_t workspace_bytes_, int32_t* device_status, void* stream) {
+    CHECK(check_layer_args(g, desc, H, ldh, W_qkv, W_o, workspace, workspace_bytes_));
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w = carve(workspace, g->n);
+    if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
+
+    // Q | K | V of every node from the layer's input
+    dg4i_proj_args p;
+    p.A = (const __nv_bfloat16*)H; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
+    p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n;
+    CHECK(dg4i_proj_launch(p, st));
+
+    const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;
+    for (int l = 0; l < g->n_levels; ++l) {
+        const int first = g->h_level_ptr[l], count = g->h_level_ptr[l + 1] - first;
+        if (count <= 0) continue;
+        dg4i_attn_args a = attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128);
+        a.node_list = g->level_nodes; a.first = first; a.count = count;
+        CHECK(dg4i_attn_launch(a, st));
+
+        dg4i_proj_args o;
+        o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
+        o.out[0] = (__nv_bfloat16*)H; o.ldo[0] = ldh; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
+        o.R = (desc->flags & DG4_FLAG_RESIDUAL) ? (const __nv_bfloat16*)H : nullptr; o.ldr = ldh;
+        o.row_list = g->level_nodes; o.first = first; o.rows = count;
+        CHECK(dg4i_proj_launch(o, st));
+
+        if (l + 1 < g->n_levels) {   // refresh K | V of the finished level for the levels above
+            dg4i_proj_args k;
+            k.A = (const __nv_bfloat16*)H; k.lda = ldh; k.W = W_kv; k.n_out = 256;
+            k.out[0] = w.KV; k.ldo[0] = 256; k.out[1] = w.KV + 128; k.ldo[1] = 256; k.out[2] = nullptr; k.ldo[2] = 0;
+            k.R = nullptr; k.ldr = 0; k.row_list = g->level_nodes; k.first = first; k.rows = count;
+            CHECK(dg4i_proj_launch(k, st));
+        }
+    }
+    return DG4_OK;
+}

@@ -1,0 +1,322 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU checker on the same seeded
+inputs.  Index arrays must match bit for bit; fp32 attention within 1e-5 max-abs; bf16 tensors within
+2e-2 of the row norm (per row, L2) of the checker run with the same storage rounding."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2502_01681_b200 import dg4, synth
+from tests.gpu_util import bf16_weights, dev_bf16, f64_of_bits, host_f64_of_bf16
+from tests.helpers import binary_in_tree, csr_from_fanins, levels_of, random_dag, rel_row_err
+
+pytestmark = pytest.mark.gpu
+
+BF16_ROW_TOL = 2e-2      # relative to the row norm
+F32_ABS_TOL = 1e-5
+
+
+# ----------------------------------------------------------------------------- graph prep
+
+def _check_graph_arrays(rp, ci, level, hops, chunk):
+    g = dg4.dg4_graph_create(rp, ci, level, hops, chunk)
+    n = len(level)
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    lptr, lnodes = orc.level_buckets(level)
+    mc = 2 ** (hops + 1) - 1
+    eff_chunk = 0 if chunk >= n else chunk
+    perm, cptr = orc.class_order(np.arange(n, dtype=np.int32), orc.chunk_ptr(n, eff_chunk), ptr, mc)
+    lperm, lcptr = orc.class_order(lnodes, lptr, ptr, mc)
+
+    def same(which, want):
+        got = dg4.dg4_graph_export(g, which)
+        assert got.shape == want.ravel().shape and (got == want.ravel()).all(), which
+
+    for _ in range(2):                      # the second round checks that a rebuild reproduces everything
+        same(dg4.DG4_ARR_NBR_PTR, ptr)
+        same(dg4.DG4_ARR_NBR_IDX, idx)
+        same(dg4.DG4_ARR_LEVEL_PTR, lptr)
+        same(dg4.DG4_ARR_LEVEL_NODES, lnodes)
+        same(dg4.DG4_ARR_PERM, perm)
+        same(dg4.DG4_ARR_CLASS_PTR, cptr)
+        same(dg4.DG4_ARR_LEVEL_PERM, lperm)
+        same(dg4.DG4_ARR_LEVEL_CLASS_PTR, lcptr)
+        dg4.dg4_graph_rebuild(g)
+    info = dg4.dg4_graph_info(g)
+    assert info.n_nodes == n and info.n_nbr == len(idx) and info.n_levels == len(lptr) - 1 and info.max_class == mc
+    return g
+
+
+@pytest.mark.parametrize("hops", [1, 2])
+def test_graph_prep_small_shapes(hops):
+    cases = []
+    cases.append([[]])                                             # a single primary input
+    cases.append([[] for _ in range(5)])                           # no edges at all
+    cases.append([[]] + [[i - 1] for i in range(1, 40)])           # a chain of inverters
+    cases.append(binary_in_tree(5)[0])                             # every gate at maximum class
+    cases.append([[], [], [0, 0], [2, 2], [1, 3], [3, 4]])         # tied inputs, 1-path and 2-path to one node
+    rng = np.random.default_rng(0)
+    cases.append(random_dag(rng, 7, 3000, window=40))              # spans several 1024-element tiles, ragged tail
+    for fanins in cases:
+        rp, ci = csr_from_fanins(fanins)
+        _check_graph_arrays(rp, ci, levels_of(fanins), hops, 0)
+
+
+@pytest.mark.parametrize("cfg,shrink,chunk", [(1, 1, 0), (1, 1, 1024), (2, 4, 2048), (3, 20, 8192), (4, 10, 0),
+                                              (5, 100, 4096), (5, 100, 0)])
+def test_graph_prep_matches_checker_on_workloads(cfg, shrink, chunk):
+    w = synth.workload(cfg, shrink)
+    g = w.graph()
+    _check_graph_arrays(g.row_ptr, g.col_idx, g.level, w.hops, chunk)
+
+
+def test_graph_prep_accepts_any_strict_layering():
+    fanins = random_dag(np.random.default_rng(3), 5, 500, window=20)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins) * 3 + 1        # still strictly increasing along edges, with empty levels
+    _check_graph_arrays(rp, ci, level, 2, 0)
+
+
+# ----------------------------------------------------------------------------- attention
+
+def _attention_case(rp, ci, level, hops, heads, dtype, scale, std, seed=0):
+    n = len(level)
+    g = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    q, k, v = (synth.normal_f32(seed, 50 + i, (n, 128), std) for i in range(3))
+    if dtype == "f32":
+        dq, dk, dv = (torch.from_numpy(t).cuda() for t in (q, k, v))
+        want = orc.attention(q, k, v, ptr, idx, heads, scale)
+        o = torch.empty_like(dq)
+        dg4.dg4_sparse_attn_fwd(g, dg4.desc(heads, dg4.DG4_F32, scale), dq, dk, dv, o)
+        torch.cuda.synchronize()
+        got = o.cpu().numpy().astype(np.float64)
+        return got, want
+    bq, bk, bv = (synth.f32_to_bf16_bits(t) for t in (q, k, v))
+    want = orc.round_bf16(orc.attention(f64_of_bits(bq), f64_of_bits(bk), f64_of_bits(bv), ptr, idx, heads, scale))
+    dq, dk, dv = dev_bf16(bq), dev_bf16(bk), dev_bf16(bv)
+    o = torch.empty_like(dq)
+    dg4.dg4_sparse_attn_fwd(g, dg4.desc(heads, dg4.DG4_BF16, scale), dq, dk, dv, o)
+    torch.cuda.synchronize()
+    return host_f64_of_bf16(o), want
+
+
+def test_attention_config1_fp32():
+    w = synth.workload(1)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, 1, 0)
+    q, k, v = w.qkv_f32()
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, 1)
+    want = orc.attention(q, k, v, ptr, idx, w.heads, w.scale)
+    dq, dk, dv = (torch.from_numpy(t).cuda() for t in (q, k, v))
+    o = torch.empty_like(dq)
+    dg4.dg4_sparse_attn_fwd(gr, dg4.desc(w.heads, dg4.DG4_F32, w.scale), dq, dk, dv, o)
+    torch.cuda.synchronize()
+    err = np.abs(o.cpu().numpy().astype(np.float64) - want).max()
+    assert err <= F32_ABS_TOL, err
+    # primary inputs attend only themselves: their output is their V row, bit for bit
+    assert torch.equal(o[:g.n_pi], dv[:g.n_pi])
+
+
+@pytest.mark.parametrize("hops", [1, 2])
+@pytest.mark.parametrize("heads", [1, 2, 4, 8, 16, 32])
+def test_attention_fp32_heads_and_hops(hops, heads):
+    fanins = random_dag(np.random.default_rng(heads), 9, 1500, window=30)
+    rp, ci = csr_from_fanins(fanins)
+    got, want = _attention_case(rp, ci, levels_of(fanins), hops, heads, "f32", 1.0 / np.sqrt(128 // heads), 1.0)
+    assert np.abs(got - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+
+
+@pytest.mark.parametrize("hops", [1, 2])
+@pytest.mark.parametrize("heads", [1, 2, 4, 8, 16])
+def test_attention_bf16_heads_and_hops(hops, heads):
+    fanins = random_dag(np.random.default_rng(100 + heads), 9, 1500, window=30)
+    rp, ci = csr_from_fanins(fanins)
+    got, want = _attention_case(rp, ci, levels_of(fanins), hops, heads, "bf16", 1.0 / np.sqrt(128 // heads), 1.0)
+    assert rel_row_err(got, want).max() <= BF16_ROW_TOL
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_attention_peaked_softmax(dtype):
+    # scale 1 and unit-variance inputs: scores reach tens, the softmax is far from uniform
+    fanins = random_dag(np.random.default_rng(7), 9, 2000, window=30)
+    rp, ci = csr_from_fanins(fanins)
+    got, want = _attention_case(rp, ci, levels_of(fanins), 2, 8, dtype, 1.0, 2.0)
+    if dtype == "f32":
+        assert np.abs(got - want).max() <= 5e-5      # values up to ~8; same relative accuracy
+    else:
+        assert rel_row_err(got, want).max() <= BF16_ROW_TOL
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_attention_degenerate_graphs(dtype):
+    shapes = {
+        "single": [[]],
+        "edgeless": [[] for _ in range(33)],
+        "chain": [[]] + [[i - 1] for i in range(1, 70)],
+        "tree": binary_in_tree(6)[0],
+        "tied": [[], [], [0, 0], [2, 2], [1, 3], [3, 4]],
+    }
+    for name, fanins in shapes.items():
+        rp, ci = csr_from_fanins(fanins)
+        got, want = _attention_case(rp, ci, levels_of(fanins), 2, 8, dtype, 0.25, 1.0)
+        if dtype == "f32":
+            assert np.abs(got - want).max() <= F32_ABS_TOL, name
+        else:
+            assert rel_row_err(got, want).max() <= BF16_ROW_TOL, name
+
+
+def test_attention_strided_interleaved_kv():
+    # K and V interleaved in one [n, 256] buffer, as the layer calls lay them out
+    fanins = random_dag(np.random.default_rng(11), 9, 1000, window=30)
+    rp, ci = csr_from_fanins(fanins)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, levels_of(fanins), 2, 0)
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    bq, bk, bv = (synth.normal_bf16_bits(5, 60 + i, (n, 128), 1.0) for i in range(3))
+    kv = torch.empty(n, 256, dtype=torch.bfloat16, device="cuda")
+    kv[:, :128] = dev_bf16(bk)
+    kv[:, 128:] = dev_bf16(bv)
+    o = torch.empty(n, 128, dtype=torch.bfloat16, device="cuda")
+    dg4.dg4_sparse_attn_fwd(g, dg4.desc(8, dg4.DG4_BF16, 0.25), dev_bf16(bq), kv[:, :128], kv[:, 128:], o)
+    torch.cuda.synchronize()
+    want = orc.round_bf16(orc.attention(f64_of_bits(bq), f64_of_bits(bk), f64_of_bits(bv), ptr, idx, 8, 0.25))
+    assert rel_row_err(host_f64_of_bf16(o), want).max() <= BF16_ROW_TOL
+
+
+def test_attention_config3_full_size():
+    w = synth.workload(3)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, 2, 0)
+    bq, bk, bv = w.qkv_bf16_bits()
+    dq, dk, dv = dev_bf16(bq), dev_bf16(bk), dev_bf16(bv)
+    o = torch.empty_like(dq)
+    dg4.dg4_sparse_attn_fwd(gr, dg4.desc(8, dg4.DG4_BF16, w.scale), dq, dk, dv, o)
+    torch.cuda.synchronize()
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, 2)
+    assert (dg4.dg4_graph_export(gr, dg4.DG4_ARR_NBR_IDX) == idx).all()
+    want = orc.round_bf16(orc.attention(f64_of_bits(bq), f64_of_bits(bk), f64_of_bits(bv), ptr, idx, 8, w.scale))
+    assert rel_row_err(host_f64_of_bf16(o), want).max() <= BF16_ROW_TOL
+
+
+# ----------------------------------------------------------------------------- projections
+
+@pytest.mark.parametrize("n", [1, 127, 128, 129, 1000, 4133])
+def test_projections_match_checker(n):
+    fanins = [[] for _ in range(n)]
+    rp, ci = csr_from_fanins(fanins)
+    g = dg4.dg4_graph_create(rp, ci, np.zeros(n, np.int32), 1, 0)
+    xb = synth.normal_bf16_bits(9, 1, (n, 128), 1.0)
+    wq_bits, wq = bf16_weights(synth.normal_f32(9, 2, (384, 128), 0.05))
+    wo_bits, wo = bf16_weights(synth.normal_f32(9, 3, (128, 128), 0.05))
+    x = f64_of_bits(xb)
+    dsc = dg4.desc(8, dg4.DG4_BF16, 0.25, residual=True)
+    dx = dev_bf16(xb)
+    q, k, v, h = (torch.empty(n, 128, dtype=torch.bfloat16, device="cuda") for _ in range(4))
+    dg4.dg4_qkv_project(g, dsc, dx, dev_bf16(wq_bits), q, k, v)
+    dg4.dg4_out_project(g, dsc, q, dev_bf16(wo_bits), dx, h)
+    torch.cuda.synchronize()
+    want = orc.round_bf16(orc.project(x, wq))
+    got = np.concatenate([host_f64_of_bf16(t) for t in (q, k, v)], axis=1)
+    assert rel_row_err(got, want).max() <= BF16_ROW_TOL
+    want_h = orc.round_bf16(orc.project(host_f64_of_bf16(q), wo, x))
+    assert rel_row_err(host_f64_of_bf16(h), want_h).max() <= BF16_ROW_TOL
+
+
+# ----------------------------------------------------------------------------- whole layers
+
+def _weights(w, layers):
+    out = []
+    for l in range(layers):
+        out.append(bf16_weights(w.w_qkv_f32(l)) + bf16_weights(w.w_o_f32(l)))
+    return out
+
+
+def _run_layers_gpu(gr, w, xb, weights, mode):
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual)
+    ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    h = dev_bf16(xb).clone()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for (wq_bits, _, wo_bits, _) in weights:
+        if mode == "parallel":
+            dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), h, ws)
+        else:
+            dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), ws, status)
+            assert int(status.item()) == 0
+    torch.cuda.synchronize()
+    return host_f64_of_bf16(h)
+
+
+def _run_layers_checker(g, w, xb, weights, mode):
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    h = f64_of_bits(xb)
+    if mode == "levelised":
+        lptr, lnodes = orc.level_buckets(g.level)
+    for (_, wq, _, wo) in weights:
+        if mode == "parallel":
+            h = orc.layer_parallel(h, wq, wo, ptr, idx, w.heads, w.scale, residual=w.residual, rounding="bf16")
+        else:
+            h = orc.layer_levelised(h, wq, wo, ptr, idx, lptr, lnodes, w.heads, w.scale, residual=w.residual,
+                                    rounding="bf16")
+    return h
+
+
+@pytest.mark.parametrize("cfg,shrink,mode", [(2, 1, "parallel"), (2, 7, "parallel"), (5, 200, "parallel"),
+                                             (4, 20, "levelised"), (5, 400, "levelised"), (2, 10, "levelised")])
+def test_layers_match_checker(cfg, shrink, mode):
+    w = synth.workload(cfg, shrink)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+    xb = w.x_bf16_bits()
+    weights = _weights(w, w.layers)
+    got = _run_layers_gpu(gr, w, xb, weights, mode)
+    want = _run_layers_checker(g, w, xb, weights, mode)
+    err = rel_row_err(got, want)
+    assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
+
+
+def test_levelised_differs_from_parallel_and_is_repeatable():
+    w = synth.workload(4, 20)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+    xb = w.x_bf16_bits()
+    weights = _weights(w, 1)
+    a = _run_layers_gpu(gr, w, xb, weights, "levelised")
+    b = _run_layers_gpu(gr, w, xb, weights, "levelised")
+    p = _run_layers_gpu(gr, w, xb, weights, "parallel")
+    assert (a == b).all()                                   # a race between levels would show up as a diff
+    lvl0 = g.level == 0
+    assert (a[lvl0] == p[lvl0]).all()                       # level-0 rows never see an updated row
+    assert np.abs(a - p).max() > 0
+
+
+# ----------------------------------------------------------------------------- error paths (no GPU fault)
+
+def test_forward_calls_reject_bad_arguments():
+    fanins = random_dag(np.random.default_rng(1), 4, 60, window=8)
+    rp, ci = csr_from_fanins(fanins)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, levels_of(fanins), 1, 0)
+    t = torch.zeros(n, 128, dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros(n, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_sparse_attn_fwd(g, dg4.desc(3, dg4.DG4_BF16, 1.0), t, t, t, o)
+    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_sparse_attn_fwd(g, dg4.desc(8, dg4.DG4_BF16, 1.0, d=64), t, t, t, o)
+    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_sparse_attn_fwd(g, dg4.desc(8, dg4.DG4_BF16, 1.0), t, t, t, t)
+    assert e.value.status == dg4.DG4_ERR_INVALID_ARG
+    odd = torch.zeros(n * 128 + 8, dtype=torch.bfloat16, device="cuda")[1:n * 128 + 1].view(n, 128)
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_sparse_attn_fwd(g, dg4.desc(8, dg4.DG4_BF16, 1.0), odd, t, t, o)
+    assert e.value.status == dg4.DG4_ERR_INVALID_ARG
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_qkv_project(g, dg4.desc(8, dg4.DG4_F32, 1.0), t, t, t, t, t)
+    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+    small = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_layer_fwd_parallel(g, dg4.desc(8, dg4.DG4_BF16, 1.0), t, t, t, o, small)
+    assert e.value.status == dg4.DG4_ERR_INVALID_ARG
+    torch.cuda.synchronize()
