@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-attention layer over a synthetic And-Inverter Graph.
+
+One step = one pass of the whole hot path over the 10M-node workload (50 000 primary inputs + 10 000 000
+gates, log-uniform locality window, 2-hop cones, d = 128, 8 heads, bf16):
+    device graph prep (neighbourhood CSR, level buckets, class orderings)
+    + 3 layers all-nodes-parallel (QKV projection, fused sparse attention, output projection + residual)
+    + 3 layers levelised (the same layer in topological level order).
+The metric is AIG nodes per second per sparse-attention layer: nodes x layer passes / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--shrink S]
+
+With N > 1 (under torchrun) every rank runs its own circuit of the same shape (weak scaling, no collective
+on the data path); the reported time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "AIG nodes/s per sparse-attention layer"
+UNIT = "nodes/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def workload_config(w, n_levels=None, n_nbr=None):
+    c = {"workload": w.name, "n_pi": w.n_pi, "n_gates": w.n_gates, "hops": w.hops, "d": w.d, "heads": w.heads,
+         "layers": w.layers, "modes": list(w.modes), "window_log2": list(w.win_exp), "not_ratio": w.not_ratio,
+         "residual": w.residual, "l2": "inputs larger than L2 (no flush)"}
+    if n_levels is not None:
+        c["n_levels"] = int(n_levels)
+    if n_nbr is not None:
+        c["n_nbr"] = int(n_nbr)
+    return c
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU checker timed on a bounded sample (reported baseline; also the --impl reference arm)
+# --------------------------------------------------------------------------------------------------
+
+def cpu_sample_problem(w, sample_nodes):
+    """A circuit of about `sample_nodes` nodes from the workload's own generator (same primary-input share,
+    window distribution, NOT ratio, hops and tensor recipe; node counts divided), small enough for the CPU."""
+    from oracle import oracle as orc
+    from paper_2502_01681_b200 import synth
+    ws = synth.workload(5, max(1, round(w.n / sample_nodes)))
+    g = ws.graph()
+    sample_nodes = g.n
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    lptr, lnodes = orc.level_buckets(g.level)
+    x = synth.bf16_bits_to_f32(w.x_bf16_bits(sample_nodes)).astype(np.float64)
+    wq = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(w.w_qkv_f32(0))).astype(np.float64)
+    wo = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(w.w_o_f32(0))).astype(np.float64)
+    return g, ptr, idx, lptr, lnodes, x, wq, wo
+
+
+def sample_text(prob):
+    g = prob[0]
+    return (f"the workload's generator at {g.n} nodes ({len(prob[3]) - 1} levels): graph prep + 1 parallel layer "
+            f"+ 1 levelised layer, fp64")
+
+
+def cpu_step(w, prob):
+    """One parallel + one levelised layer of the checker on the sample; returns seconds."""
+    from oracle import oracle as orc
+    g, ptr, idx, lptr, lnodes, x, wq, wo = prob
+    t0 = time.perf_counter()
+    orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    orc.level_buckets(g.level)
+    orc.layer_parallel(x, wq, wo, ptr, idx, w.heads, w.scale, residual=w.residual, rounding="bf16")
+    orc.layer_levelised(x, wq, wo, ptr, idx, lptr, lnodes, w.heads, w.scale, residual=w.residual, rounding="bf16")
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, sample_nodes=100_000):
+    from oracle import oracle as orc
+    prob = cpu_sample_problem(w, sample_nodes)
+    dt = cpu_step(w, prob)
+    return {"value": prob[0].n * 2 / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": sample_text(prob) + f", {dt:.1f} s"}
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU checker as it stands, on the host cores, on a bounded sample per step."""
+    from oracle import oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_nodes = 50_000
+    prob = cpu_sample_problem(w, sample_nodes)
+    for _ in range(args.warmup):
+        cpu_step(w, prob)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        cpu_step(w, prob)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = prob[0].n * 2 / dt
+    sample = "per step: " + sample_text(prob)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.idx = device_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            sm, mx, reasons = [], [], set()
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            if sm:
+                out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                       "samples": len(sm)}
+        finally:
+            try:
+                os.unlink(self.path)
+            except OSError:
+                pass
+        return out
+
+
+# --------------------------------------------------------------------------------------------------
+# the GPU arm
+# --------------------------------------------------------------------------------------------------
+
+def run_ours(args, w):
+    import torch
+    from paper_2502_01681_b200 import dg4, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank its own circuit of the same shape (weak scaling)
+    w.seed = w.seed + 1000 * rank
+    g = w.graph()
+    n = g.n
+    x_host = torch.empty((n, w.d), dtype=torch.int16).pin_memory()
+    w.x_bf16_bits(out=x_host.numpy().view(np.uint16))
+    wq = [torch.from_numpy(synth.f32_to_bf16_bits(w.w_qkv_f32(l)).view(np.int16)).cuda().view(torch.bfloat16)
+          for l in range(w.layers)]
+    wo = [torch.from_numpy(synth.f32_to_bf16_bits(w.w_o_f32(l)).view(np.int16)).cuda().view(torch.bfloat16)
+          for l in range(w.layers)]
+    out_host = torch.empty((n, w.d), dtype=torch.int16).pin_memory()
+
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local)
+    info = gr.info
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual)
+    ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    x_dev = x_host.cuda().view(torch.bfloat16)
+    h_par = torch.empty_like(x_dev)
+    h_lev = torch.empty_like(x_dev)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # views into the workspace, laid out as the layer calls lay it out: Q [n,128] | KV [n,256] | O [n,128]
+    wsb = ws.view(torch.bfloat16)
+    q_v = wsb[: n * 128].view(n, 128)
+    kv_v = wsb[n * 128: n * 384].view(n, 256)
+    o_v = wsb[n * 384: n * 512].view(n, 128)
+    stream = torch.cuda.current_stream()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    stage_ev = []          # (name, start, stop) per step
+
+    def step(record):
+        marks = []
+
+        def mark(name, fn):
+            if record:
+                a, b = ev(), ev()
+                a.record(stream)
+                fn()
+                b.record(stream)
+                marks.append((name, a, b))
+            else:
+                fn()
+
+        mark("graph_prep", lambda: dg4.dg4_graph_rebuild(gr))
+        h_par.copy_(x_dev)
+        for l in range(w.layers):
+            mark("qkv", lambda: dg4.dg4_qkv_project(gr, dsc, h_par, wq[l], q_v, kv_v[:, :128], kv_v[:, 128:]))
+            mark("attn", lambda: dg4.dg4_sparse_attn_fwd(gr, dsc, q_v, kv_v[:, :128], kv_v[:, 128:], o_v))
+            mark("out", lambda: dg4.dg4_out_project(gr, dsc, o_v, wo[l], h_par, h_par))
+        h_lev.copy_(x_dev)
+        for l in range(w.layers):
+            mark("levelised", lambda: dg4.dg4_layer_fwd_levelised(gr, dsc, h_lev, wq[l], wo[l], ws, status))
+        if record:
+            stage_ev.append(marks)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = dg4.dg4_launch_count()
+    t_start, t_stop = ev(), ev()
+    barrier()
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step(True)
+    t_stop.record(stream)
+    barrier()
+    launches = dg4.dg4_launch_count() - launches0
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "device status reported an error"
+    total_ms = t_start.elapsed_time(t_stop)
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    layer_passes = w.layers * 2
+    value = world * n * layer_passes / (ms_per_step * 1e-3)
+
+    stages = {}
+    for marks in stage_ev:
+        for name, a, b in marks:
+            stages.setdefault(name, []).append(a.elapsed_time(b))
+    attn_ms = float(np.mean(stages["attn"]))
+    alg_bytes = 516.0 * n + 516.0 * info.n_nbr
+    peak, peak_kind = measured_hbm_peak()
+    achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
+    per_step = lambda name: float(np.sum(stages[name])) / args.steps
+    stage_report = {
+        "graph_prep_ms": per_step("graph_prep"),
+        "qkv_ms_per_layer": per_step("qkv") / w.layers,
+        "attn_ms_per_layer": attn_ms,
+        "out_ms_per_layer": per_step("out") / w.layers,
+        "levelised_ms_per_layer": per_step("levelised") / w.layers,
+        "parallel_layer_nodes_per_s": n / ((per_step("qkv") + per_step("attn") + per_step("out")) / w.layers * 1e-3),
+        "levelised_layer_nodes_per_s": n / (per_step("levelised") / w.layers * 1e-3),
+        "attn_kernel_nodes_per_s": n / (attn_ms * 1e-3),
+    }
+
+    # ---- end to end through the C ABI from host buffers -----------------------------------------
+    e2e_steps = max(1, min(2, args.steps))
+    h2d = x_host.numel() * 2 + (g.row_ptr.nbytes + g.col_idx.nbytes + g.level.nbytes)
+    d2h = out_host.numel() * 2
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        gr2 = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local)
+        x2 = x_host.cuda(non_blocking=True).view(torch.bfloat16)
+        hp = x2.clone()
+        for l in range(w.layers):
+            dg4.dg4_layer_fwd_parallel(gr2, dsc, hp, wq[l], wo[l], hp, ws)
+        for l in range(w.layers):
+            dg4.dg4_layer_fwd_levelised(gr2, dsc, x2, wq[l], wo[l], ws, status)
+        out_host.copy_(x2.view(torch.int16), non_blocking=True)
+        torch.cuda.synchronize()
+        dg4.dg4_graph_destroy(gr2)
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * n * layer_passes / e2e_s
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(w, info.n_levels, info.n_nbr),
+            "stages": stage_report,
+            "roofline": {"bound": "hbm", "kernel": "sparse_attn_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_nominal_8000": achieved / 8000.0,
+                         "algorithmic_bytes_per_launch": alg_bytes,
+                         "unique_row_floor_bytes": 4.0 * 256 * n + 4.0 * (info.n_nbr + n),
+                         "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.shrink == 1 else None},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "ms_per_step": e2e_s * 1e3, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) of one sparse_attn_kernel launch on the full workload, from the ncu capture
+# summarised under profiles/; None while no capture of the current kernel exists.
+TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shrink", type=int, default=1, help="divide the workload's node counts (profiling only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.shrink == 1 else args.warmup
+    from paper_2502_01681_b200 import synth
+    w = synth.workload(5, args.shrink)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

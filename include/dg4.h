@@ -88,6 +88,10 @@ const char* dg4_status_string(dg4_status s);
 /* Detail of the last error on the calling thread ("" if none).  Valid until the next failing call. */
 const char* dg4_last_error(void);
 
+/* Number of GPU kernels this library has launched in the calling process so far (monotone; for the
+ * accounting of benchmarks -- the paper has no counterpart). */
+int64_t dg4_launch_count(void);
+
 /*
  * Graph prep.  Sec. 3.2: node kinds are told apart by in-degree (0 primary input, 1 NOT, 2 AND); Eq. 1
  * defines the logic level; cone_k(v) = { u : a path u -> v of length <= k } with v included, at most

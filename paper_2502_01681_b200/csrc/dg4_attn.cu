@@ -163,6 +163,7 @@ dg4_status launch_for_heads(const dg4i_attn_args& a, cudaStream_t st) {
         case 32: sparse_attn_kernel<BF16, 32, MAXN><<<blocks, threads, 0, st>>>(a); break;
         default: DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
     }
+    dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }

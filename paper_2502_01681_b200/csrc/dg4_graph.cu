@@ -148,8 +148,11 @@ dg4_status exclusive_scan(const int32_t* in, int32_t* out, int64_t n, int32_t* b
     if (n <= 0) return DG4_OK;
     int nb = (int)((n + kScanTile - 1) / kScanTile);
     scan_reduce_kernel<<<nb, kScanThreads, 0, st>>>(in, n, block_sums);
+    dg4i_count_launch();
     scan_sums_kernel<<<1, 1024, 0, st>>>(block_sums, nb);
+    dg4i_count_launch();
     scan_apply_kernel<<<nb, kScanThreads, 0, st>>>(in, out, n, block_sums);
+    dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
@@ -227,10 +230,12 @@ dg4_status radix_pass(dg4_graph* g, const int32_t* src, int shift, int by_class,
     DG4_CUDA_TRY(cudaMemsetAsync(g->hist, 0, len * sizeof(int32_t), st));
     radix_pass_kernel<RADIX, false><<<nb, kTile, 0, st>>>(g->n, src, g->level, shift, g->nbr_ptr, by_class, bpc,
                                                           g->hist, nullptr);
+    dg4i_count_launch();
     dg4_status s = exclusive_scan(g->hist, g->hist, len, g->block_sums, st);
     if (s != DG4_OK) return s;
     radix_pass_kernel<RADIX, true><<<nb, kTile, 0, st>>>(g->n, src, g->level, shift, g->nbr_ptr, by_class, bpc,
                                                          g->hist, dst);
+    dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
@@ -269,13 +274,16 @@ dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only
 
     // neighbourhood sizes -> nbr_ptr
     cone_count_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr);
+    dg4i_count_launch();
     if ((s = exclusive_scan(g->nbr_ptr, g->nbr_ptr, (int64_t)n + 1, g->block_sums, st)) != DG4_OK) return s;
     if (sizes_only) return DG4_OK;
     cone_fill_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr, g->nbr_idx);
+    dg4i_count_launch();
 
     // level buckets
     DG4_CUDA_TRY(cudaMemsetAsync(g->level_ptr, 0, ((size_t)g->n_levels + 1) * sizeof(int32_t), st));
     level_hist_kernel<<<nbk, tb, 0, st>>>(n, g->level, g->level_ptr);
+    dg4i_count_launch();
     if ((s = exclusive_scan(g->level_ptr, g->level_ptr, (int64_t)g->n_levels + 1, g->block_sums, st)) != DG4_OK) return s;
     if ((s = sort_by_level(g, nullptr, g->level_nodes, st)) != DG4_OK) return s;
 
@@ -285,12 +293,14 @@ dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only
     int bpc = g->perm_chunk > 0 ? g->perm_chunk / kTile : nb;
     DG4_CUDA_TRY(cudaMemsetAsync(g->class_ptr, 0, ((size_t)g->n_chunks * mc1 + 1) * sizeof(int32_t), st));
     class_hist_kernel<<<nbk, tb, 0, st>>>(n, g->nbr_ptr, g->level, 0, g->perm_chunk, g->max_class, g->class_ptr);
+    dg4i_count_launch();
     if ((s = exclusive_scan(g->class_ptr, g->class_ptr, (int64_t)g->n_chunks * mc1 + 1, g->block_sums, st)) != DG4_OK) return s;
     if ((s = radix_pass<8>(g, nullptr, 0, 1, bpc, g->n_chunks, g->perm, st)) != DG4_OK) return s;
 
     // degree-class order inside level buckets: stable by class, then stable by level
     DG4_CUDA_TRY(cudaMemsetAsync(g->level_class_ptr, 0, ((size_t)g->n_levels * mc1 + 1) * sizeof(int32_t), st));
     class_hist_kernel<<<nbk, tb, 0, st>>>(n, g->nbr_ptr, g->level, 1, 0, g->max_class, g->level_class_ptr);
+    dg4i_count_launch();
     if ((s = exclusive_scan(g->level_class_ptr, g->level_class_ptr, (int64_t)g->n_levels * mc1 + 1, g->block_sums, st)) != DG4_OK) return s;
     if ((s = radix_pass<8>(g, nullptr, 0, 1, nb, 1, g->seq_a, st)) != DG4_OK) return s;
     if ((s = sort_by_level(g, g->seq_a, g->level_perm, st)) != DG4_OK) return s;

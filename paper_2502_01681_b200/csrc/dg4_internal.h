@@ -27,6 +27,9 @@ void dg4_set_error(const char* fmt, ...);
         return (code);               \
     } while (0)
 
+// ---- launch accounting (every kernel launch of the library bumps this counter) ------------------
+void dg4i_count_launch(int n = 1);
+
 // ---- the graph handle -----------------------------------------------------------------------
 struct dg4_graph {
     int32_t device = 0;

@@ -9,10 +9,12 @@
 #include "dg4_internal.h"
 
 #include <string.h>
+#include <atomic>
 
 namespace {
 
 thread_local char g_err[512] = "";
+std::atomic<long long> g_launches{0};
 
 bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
@@ -76,6 +78,10 @@ void dg4_set_error(const char* fmt, ...) {
 }
 
 extern "C" const char* dg4_last_error(void) { return g_err; }
+
+void dg4i_count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+extern "C" int64_t dg4_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 extern "C" const char* dg4_status_string(dg4_status s) {
     switch (s) {

@@ -54,6 +54,7 @@ dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st) {
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "projection width %d is not supported", a.n_out);
     unsigned blocks = (unsigned)((a.rows + kRows - 1) / kRows);
     proj_simple_kernel<<<blocks, 128, 0, st>>>(a);
+    dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }

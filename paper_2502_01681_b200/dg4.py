@@ -34,7 +34,7 @@ DG4_FLAG_RESIDUAL = 1
  DG4_ARR_LEVEL_PERM, DG4_ARR_LEVEL_CLASS_PTR) = range(8)
 
 EXPORTS = [
-    "dg4_status_string", "dg4_last_error", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",
+    "dg4_status_string", "dg4_last_error", "dg4_launch_count", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
 ]
@@ -82,6 +82,8 @@ def load():
     lib.dg4_status_string.argtypes = [ctypes.c_int]
     lib.dg4_last_error.restype = ctypes.c_char_p
     lib.dg4_last_error.argtypes = []
+    lib.dg4_launch_count.restype = ctypes.c_int64
+    lib.dg4_launch_count.argtypes = []
     lib.dg4_graph_create.restype = ctypes.c_int
     lib.dg4_graph_create.argtypes = [ctypes.c_int32, i32p, i32p, i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                      ctypes.POINTER(vp)]
@@ -158,6 +160,10 @@ class Graph:
     @property
     def n(self) -> int:
         return int(self.info.n_nodes)
+
+
+def dg4_launch_count() -> int:
+    return int(load().dg4_launch_count())
 
 
 def dg4_graph_create(row_ptr, col_idx, level, hops: int, perm_chunk: int = 0, device: int = 0) -> Graph:
