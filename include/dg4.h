@@ -180,6 +180,31 @@ dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc* desc,
                                   void* stream);
 
 /*
+ * The all-nodes-parallel layer for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a deployment aid.)
+ *
+ * Who needs it: programs in which nobody may call cudaMalloc (or a framework allocator) by the time the layer
+ * runs -- a service that divided up the GPU at start-up and locked the pool, a plug-in inside a host
+ * application that owns the device heap, a latency-critical loop that cannot take the device-wide
+ * synchronisation cudaMalloc / cudaFree imply.  Same computation and same arguments as
+ * dg4_layer_fwd_parallel, minus the workspace: the intermediates (Q, K|V, O) live in a fixed 32 MiB array
+ * that is part of the library image and is held on every GPU that loads the library until the process exits.
+ *
+ *   - Capacity: graphs of at most dg4_static_max_nodes() = 32 768 nodes (1 KiB of scratch per node);
+ *     larger graphs are rejected with DG4_ERR_INVALID_ARG and a message naming the limit.
+ *   - The graph's device must be current.  The first call on a device looks up the array's device address
+ *     (once per device); make that first call outside any stream capture.
+ *   - The call allocates nothing and frees nothing, on the host or on the device.
+ *   - All calls share the one array.  It is never cleared and needs no clearing (a call writes every scratch
+ *     row before reading it), but calls that overlap on the GPU -- different streams, or several host
+ *     threads -- race on it: run them one after another.
+ */
+dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg4_desc* desc,
+                                         const void* H_in, int64_t ldh, const void* W_qkv, const void* W_o,
+                                         void* H_out, int64_t ldho, void* stream);
+int64_t dg4_static_max_nodes(void);
+
+/*
  * One layer in the paper's level-by-level order (Sec. 1 and Sec. 3.4: gates are encoded in strict
  * topological order and each gate is computed once).  Levels 0, 1, ... are processed in turn; a node
  * takes its query and its own key/value from its row as it was when the call started, and the key/value

@@ -37,6 +37,7 @@ EXPORTS = [
     "dg4_status_string", "dg4_last_error", "dg4_launch_count", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
+    "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes",
 ]
 
 
@@ -109,6 +110,10 @@ def load():
     lib.dg4_layer_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
     lib.dg4_layer_fwd_levelised.restype = ctypes.c_int
     lib.dg4_layer_fwd_levelised.argtypes = [vp, dp, vp, i64, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.dg4_layer_fwd_parallel_static.restype = ctypes.c_int
+    lib.dg4_layer_fwd_parallel_static.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp]
+    lib.dg4_static_max_nodes.restype = ctypes.c_int64
+    lib.dg4_static_max_nodes.argtypes = []
     _lib = lib
     return lib
 
@@ -237,3 +242,15 @@ def dg4_layer_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv, W_o, workspace, d
     _check(load().dg4_layer_fwd_levelised(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), _ptr(W_qkv), _ptr(W_o),
                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                                           _ptr(device_status), _stream(stream)))
+
+
+def dg4_static_max_nodes() -> int:
+    return int(load().dg4_static_max_nodes())
+
+
+def dg4_layer_fwd_parallel_static(g: Graph, dsc: dg4_desc, H_in, W_qkv, W_o, H_out, stream=None):
+    """The parallel layer without a workspace argument: its scratch is a fixed array inside the library, for
+    callers that cannot allocate device memory.  Graphs above dg4_static_max_nodes() are rejected; calls must
+    not overlap on the GPU."""
+    _check(load().dg4_layer_fwd_parallel_static(g.handle, ctypes.byref(dsc), _ptr(H_in), _ld(H_in), _ptr(W_qkv),
+                                                _ptr(W_o), _ptr(H_out), _ld(H_out), _stream(stream)))
