@@ -131,6 +131,10 @@ dg4_status dg4_graph_info(const dg4_graph* g, dg4_graph_info_t* out);
 dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, int32_t* host_dst, int64_t capacity,
                             int64_t* n_written);
 
+/* Waits for the device to go idle and reads the handle's status word: DG4_OK, or DG4_ERR_TIMEOUT if a bounded
+ * device-side wait of an earlier forward call ran out (that call's output is then incomplete). */
+dg4_status dg4_graph_poll_status(const dg4_graph* g, int32_t* out);
+
 /* Device pointer to one index array (owned by the handle, valid until destroy); NULL on bad arguments. */
 const int32_t* dg4_graph_device_array(const dg4_graph* g, dg4_array_id which);
 

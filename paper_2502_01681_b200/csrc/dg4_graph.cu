@@ -330,7 +330,7 @@ void free_graph(dg4_graph* g) {
     if (!g) return;
     int32_t* bufs[] = {g->row_ptr, g->col_idx, g->level, g->nbr_ptr, g->nbr_idx, g->level_ptr, g->level_nodes,
                        g->perm, g->class_ptr, g->level_perm, g->level_class_ptr, g->seq_a, g->seq_b, g->hist,
-                       g->block_sums};
+                       g->block_sums, g->dev_status};
     for (int32_t* b : bufs)
         if (b) cudaFree(b);
     free(g->h_level_ptr);
@@ -430,6 +430,8 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     TRY_ALLOC(g->seq_b, n);
     TRY_ALLOC(g->hist, g->hist_len);
     TRY_ALLOC(g->block_sums, g->block_sums_len);
+    TRY_ALLOC(g->dev_status, 1);
+    if (cudaMemset(g->dev_status, 0, sizeof(int32_t)) != cudaSuccess) { dg4_set_error("cudaMemset failed"); return fail(DG4_ERR_CUDA); }
 
     auto cuda_fail = [&](cudaError_t e, const char* what) {
         dg4_set_error("%s failed: %s", what, cudaGetErrorString(e));
@@ -520,5 +522,13 @@ extern "C" dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, i
     DeviceGuard guard(g->device);
     DG4_CUDA_TRY(cudaDeviceSynchronize());
     DG4_CUDA_TRY(cudaMemcpy(host_dst, src, (size_t)len * 4, cudaMemcpyDeviceToHost));
+    return DG4_OK;
+}
+
+extern "C" dg4_status dg4_graph_poll_status(const dg4_graph* g, int32_t* out) {
+    if (!g || !out) DG4_FAIL(DG4_ERR_INVALID_ARG, "null pointer argument");
+    DeviceGuard guard(g->device);
+    DG4_CUDA_TRY(cudaDeviceSynchronize());
+    DG4_CUDA_TRY(cudaMemcpy(out, g->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
     return DG4_OK;
 }

@@ -64,6 +64,8 @@ struct dg4_graph {
     int64_t block_sums_len = 0;
     // host copy of the level boundaries (the levelised driver launches per level)
     int32_t* h_level_ptr = nullptr;      // [n_levels+1]
+    // device status word written by kernels whose bounded waits ran out (0 = ok)
+    int32_t* dev_status = nullptr;
 };
 
 // ---- kernels' host launchers (each enqueues on `st` and returns) -----------------------------
@@ -97,5 +99,6 @@ struct dg4i_proj_args {
     const int32_t* row_list;           // nullable
     int32_t first;                     // offset into row_list (or first row id)
     int32_t rows;
+    int32_t* status = nullptr;         // device status word: receives DG4_ERR_TIMEOUT if a bounded wait runs out
 };
 dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st);

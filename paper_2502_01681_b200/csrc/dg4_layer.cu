@@ -113,7 +113,7 @@ extern "C" dg4_status dg4_qkv_project(const dg4_graph* g, const dg4_desc* desc, 
     a.out[0] = (__nv_bfloat16*)Q; a.ldo[0] = ldq;
     a.out[1] = (__nv_bfloat16*)K; a.ldo[1] = ldk;
     a.out[2] = (__nv_bfloat16*)V; a.ldo[2] = ldv;
-    a.R = nullptr; a.ldr = 0; a.row_list = nullptr; a.first = 0; a.rows = g->n;
+    a.R = nullptr; a.ldr = 0; a.row_list = nullptr; a.first = 0; a.rows = g->n; a.status = g->dev_status;
     return dg4i_proj_launch(a, (cudaStream_t)stream);
 }
 
@@ -146,6 +146,7 @@ extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, 
     a.A = (const __nv_bfloat16*)O; a.lda = ldo; a.W = (const __nv_bfloat16*)W_o; a.n_out = 128;
     a.out[0] = (__nv_bfloat16*)H_out; a.ldo[0] = ldho; a.out[1] = a.out[2] = nullptr; a.ldo[1] = a.ldo[2] = 0;
     a.R = res ? (const __nv_bfloat16*)H_res : nullptr; a.ldr = ldh; a.row_list = nullptr; a.first = 0; a.rows = g->n;
+    a.status = g->dev_status;
     return dg4i_proj_launch(a, (cudaStream_t)stream);
 }
 
@@ -178,11 +179,12 @@ extern "C" dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc*
     if (H_out == H_in && ldh != ldho) DG4_FAIL(DG4_ERR_INVALID_ARG, "in-place use needs equal leading dimensions");
     cudaStream_t st = (cudaStream_t)stream;
     Workspace w = carve(workspace, g->n);
+    int32_t* status_word = g->dev_status;
 
     dg4i_proj_args p;
     p.A = (const __nv_bfloat16*)H_in; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
     p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;
-    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
 
     CHECK(dg4i_attn_launch(attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128), st));
@@ -191,7 +193,7 @@ extern "C" dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc*
     o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
     o.out[0] = (__nv_bfloat16*)H_out; o.ldo[0] = ldho; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
     o.R = (desc->flags & DG4_FLAG_RESIDUAL) ? (const __nv_bfloat16*)H_in : nullptr; o.ldr = ldh;
-    o.row_list = nullptr; o.first = 0; o.rows = g->n;
+    o.row_list = nullptr; o.first = 0; o.rows = g->n; o.status = status_word;
     return dg4i_proj_launch(o, st);
 }
 
@@ -202,12 +204,13 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     cudaStream_t st = (cudaStream_t)stream;
     Workspace w = carve(workspace, g->n);
     if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
+    int32_t* status_word = device_status ? device_status : g->dev_status;
 
     // Q | K | V of every node from the layer's input
     dg4i_proj_args p;
     p.A = (const __nv_bfloat16*)H; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
     p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;
-    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
 
     const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;
@@ -222,14 +225,14 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
         o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
         o.out[0] = (__nv_bfloat16*)H; o.ldo[0] = ldh; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
         o.R = (desc->flags & DG4_FLAG_RESIDUAL) ? (const __nv_bfloat16*)H : nullptr; o.ldr = ldh;
-        o.row_list = g->level_nodes; o.first = first; o.rows = count;
+        o.row_list = g->level_nodes; o.first = first; o.rows = count; o.status = status_word;
         CHECK(dg4i_proj_launch(o, st));
 
         if (l + 1 < g->n_levels) {   // refresh K | V of the finished level for the levels above
             dg4i_proj_args k;
             k.A = (const __nv_bfloat16*)H; k.lda = ldh; k.W = W_kv; k.n_out = 256;
             k.out[0] = w.KV; k.ldo[0] = 256; k.out[1] = w.KV + 128; k.ldo[1] = 256; k.out[2] = nullptr; k.ldo[2] = 0;
-            k.R = nullptr; k.ldr = 0; k.row_list = g->level_nodes; k.first = first; k.rows = count;
+            k.R = nullptr; k.ldr = 0; k.row_list = g->level_nodes; k.first = first; k.rows = count; k.status = status_word;
             CHECK(dg4i_proj_launch(k, st));
         }
     }

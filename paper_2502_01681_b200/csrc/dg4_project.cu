@@ -1,49 +1,311 @@
-// Dense projections of the layer: Y = A * W^T with K = 128, bf16 operands, fp32 accumulation, one rounding
-// to bf16 per stored element.  Used for [Q|K|V] = X * W_qkv^T, H' = O * W_o^T (+ residual) and, in levelised
-// mode, for refreshing the K|V rows of a finished level.
+// Dense projections of the layer on the 5th-generation tensor cores: Y = A * W^T with K = 128, bf16 operands,
+// fp32 accumulation in tensor memory, one rounding to bf16 per stored element.  Used for
+// [Q|K|V] = X * W_qkv^T, H' = O * W_o^T (+ residual) and, in levelised mode, for refreshing the K|V rows of a
+// finished level.
 //
-// First, plain CUDA-core version: 16 rows per block staged in shared memory, one output column per thread
-// and 128-column block.  Correct for any row list; the tensor-core kernel replaces it.
+// One persistent CTA per SM, six warps:
+//   warp 0  producer: brings the weight matrix into shared memory once (TMA), then streams 128-row tiles of A
+//           through a 2-stage ring -- by TMA when the rows are contiguous, by 16-byte gathers written in the
+//           same 128-byte-swizzled layout when the rows come from a list (level buckets);
+//   warp 1  owns the tensor memory allocation and issues tcgen05.mma (one lane): for every tile and every
+//           128-column block of the output, 8 MMAs of 128x128x16 into one of four 128-column accumulator slots;
+//   warps 2-5  epilogue: tcgen05.ld of their 32 rows, residual add, rounding, a swizzled staging buffer, and
+//           row-contiguous 16-byte stores (two rows per warp instruction).
+// The stages are coupled only by mbarriers, so loads, MMAs and stores of neighbouring tiles overlap.  The work is
+// bound by HBM traffic (96 flop per byte for QKV, below the machine's ridge), which is why nothing here tries to
+// raise tensor-pipe occupancy beyond what hides the memory time.
+//
+// Every wait is bounded; on expiry the kernel records DG4_ERR_TIMEOUT in the status word, lets all warps run
+// out of their loops, waits (bounded) for its own outstanding copies, frees tensor memory and returns.
 
 #include "dg4_internal.h"
+#include "dg4_sm100.cuh"
+
+#include <mutex>
 
 namespace {
 
-constexpr int kRows = 16;
+using namespace sm100;
 
-__global__ void __launch_bounds__(128) proj_simple_kernel(dg4i_proj_args a) {
-    __shared__ float xs[kRows][128];
-    __shared__ int rid[kRows];
-    const int r0 = blockIdx.x * kRows;
-    if (threadIdx.x < kRows) {
-        int r = r0 + threadIdx.x;
-        rid[threadIdx.x] = (r < a.rows) ? (a.row_list ? a.row_list[a.first + r] : a.first + r) : -1;
+constexpr int kThreads = 192;
+constexpr int kTileM = 128;
+constexpr int kHalfBytes = 128 * 128;             // one K-half of a 128-row operand tile: 128 rows x 128 bytes
+constexpr int kTileBytes = 2 * kHalfBytes;        // 32 KiB
+constexpr int kStages = 2;
+constexpr int kSlots = 4;                         // accumulator slots of 128 columns
+constexpr int kTmemCols = 512;
+constexpr int kStageRowBytes = 256;
+constexpr int kWarpStageBytes = 32 * kStageRowBytes;   // 8 KiB per epilogue warp
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffW = 0;                                  // up to 3 blocks x 32 KiB
+constexpr int kOffA = 3 * kTileBytes;                     // 2 stages x 32 KiB
+constexpr int kOffStage = kOffA + kStages * kTileBytes;   // 4 x 8 KiB
+constexpr int kOffBar = kOffStage + 4 * kWarpStageBytes;
+constexpr int kSmemBytes = kOffBar + 256 + 1024;          // barriers + slack for manual alignment
+
+struct Bars {
+    uint64_t w_full;
+    uint64_t a_full[kStages];
+    uint64_t a_empty[kStages];
+    uint64_t acc_full[kSlots];
+    uint64_t acc_empty[kSlots];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+struct ProjParams {
+    dg4i_proj_args a;
+    int32_t n_blocks;         // n_out / 128
+    int32_t n_tiles;
+    int32_t* status;          // device status word (nullable)
+};
+
+__device__ __forceinline__ void ld_nc_v4(const void* p, uint32_t* r) {
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p));
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t* r) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void st_global_v4(void* p, const uint32_t* r) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void raise_timeout(Bars* bars, int32_t* status) {
+    atomicExch(&bars->abort_flag, 1u);
+    if (status) atomicCAS(status, 0, (int)DG4_ERR_TIMEOUT);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, ProjParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    Bars* bars = reinterpret_cast<Bars*>(base_ptr + kOffBar);
+    const uint32_t sW = base + kOffW, sA = base + kOffA, sStage = base + kOffStage;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nb = p.n_blocks;
+    const bool listed = p.a.row_list != nullptr;
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bars->w_full), 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&bars->a_full[s]), 1); mbar_init(smem_u32(&bars->a_empty[s]), 1); }
+        for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), 4); }
+        bars->abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&map_w);
+        if (!listed) tma_prefetch_desc(&map_a);
     }
+    if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+    tc_fence_before();
     __syncthreads();
-    for (int i = threadIdx.x; i < kRows * 128; i += 128) {
-        int r = i >> 7, c = i & 127;
-        xs[r][c] = rid[r] >= 0 ? __bfloat162float(a.A[(size_t)rid[r] * a.lda + c]) : 0.f;
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+
+    const int my_tiles = (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            mbar_expect_tx(smem_u32(&bars->w_full), (uint32_t)(nb * kTileBytes));
+            for (int j = 0; j < nb; ++j)
+                for (int h = 0; h < 2; ++h)
+                    tma_load_2d(sW + (j * 2 + h) * kHalfBytes, &map_w, h * 64, j * 128, smem_u32(&bars->w_full));
+        }
+        int armed = 0;
+        for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
+            const int tile = blockIdx.x + i * gridDim.x;
+            const int s = i % kStages;
+            const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+            if (!mbar_wait(smem_u32(&bars->a_empty[s]), ph ^ 1u)) { raise_timeout(bars, p.status); break; }
+            const uint32_t dst = sA + s * kTileBytes;
+            if (!listed) {
+                if (lane == 0) {
+                    mbar_expect_tx(smem_u32(&bars->a_full[s]), (uint32_t)kTileBytes);
+                    tma_load_2d(dst, &map_a, 0, tile * kTileM, smem_u32(&bars->a_full[s]));
+                    tma_load_2d(dst + kHalfBytes, &map_a, 64, tile * kTileM, smem_u32(&bars->a_full[s]));
+                }
+                armed = i + 1;
+            } else {
+                // two rows per warp instruction: lanes 0-15 one row, lanes 16-31 the next; 16 bytes per lane
+                const int chunk = lane & 15, half = chunk >> 3, c8 = chunk & 7;
+#pragma unroll 4
+                for (int it = 0; it < 64; ++it) {
+                    const int row = it * 2 + (lane >> 4);
+                    const int r = tile * kTileM + row;
+                    uint32_t v[4] = {0u, 0u, 0u, 0u};
+                    if (r < p.a.rows) {
+                        const int64_t rid = p.a.row_list[p.a.first + r];
+                        ld_nc_v4(p.a.A + rid * p.a.lda + chunk * 8, v);
+                    }
+                    st_shared_v4(dst + half * kHalfBytes + sw128_offset(row, c8), v);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[s]));
+            }
+        }
+        // error path only: do not leave with tensor copies still landing in shared memory
+        if (*abort_flag && lane == 0 && !listed) {
+            mbar_wait(smem_u32(&bars->w_full), 0);
+            for (int i = (armed > kStages ? armed - kStages : 0); i < armed; ++i)
+                mbar_wait(smem_u32(&bars->a_full[i % kStages]), (uint32_t)(i / kStages) & 1u);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16_f32(128, 128);
+            bool ok = mbar_wait(smem_u32(&bars->w_full), 0);
+            if (!ok) raise_timeout(bars, p.status);
+            int item = 0;
+            for (int i = 0; i < my_tiles && ok && !*abort_flag; ++i) {
+                const int s = i % kStages;
+                if (!mbar_wait(smem_u32(&bars->a_full[s]), (uint32_t)(i / kStages) & 1u)) { raise_timeout(bars, p.status); break; }
+                tc_fence_after();
+                const uint32_t a_base = sA + s * kTileBytes;
+                for (int j = 0; j < nb; ++j, ++item) {
+                    const int slot = item % kSlots;
+                    if (!mbar_wait(smem_u32(&bars->acc_empty[slot]), ((uint32_t)(item / kSlots) & 1u) ^ 1u)) {
+                        raise_timeout(bars, p.status); ok = false; break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d = tmem + (uint32_t)(slot * 128);
+                    const uint32_t b_base = sW + j * kTileBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t off = (uint32_t)((ks >> 2) * kHalfBytes + (ks & 3) * 32);
+                        mma_bf16(d, smem_desc_sw128(a_base + off), smem_desc_sw128(b_base + off), idesc, ks > 0 ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&bars->acc_full[slot]));
+                }
+                mma_commit(smem_u32(&bars->a_empty[s]));   // the stage is free once these MMAs have read it
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;                       // TMEM lane quadrant this warp may read
+        const uint32_t stage = sStage + (uint32_t)((warp - 2) * kWarpStageBytes);
+        const int my_row = quad * 32 + lane;             // row of the tile held by this thread
+        int item = 0;
+        bool ok = true;
+        for (int i = 0; i < my_tiles && ok && !*abort_flag; ++i) {
+            const int tile = blockIdx.x + i * gridDim.x;
+            const int r_own = tile * kTileM + my_row;
+            int64_t rid_own = -1;
+            if (r_own < p.a.rows) rid_own = listed ? (int64_t)p.a.row_list[p.a.first + r_own] : (int64_t)p.a.first + r_own;
+            for (int j = 0; j < nb; ++j, ++item) {
+                const int slot = item % kSlots;
+                if (!mbar_wait(smem_u32(&bars->acc_full[slot]), (uint32_t)(item / kSlots) & 1u)) {
+                    raise_timeout(bars, p.status); ok = false; break;
+                }
+                tc_fence_after();
+                const uint32_t t_addr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128);
+                const bool add_res = (j == 0) && p.a.R != nullptr && rid_own >= 0;
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t acc[32];
+                    tmem_ld_32x32(t_addr + (uint32_t)(q * 32), acc);
+                    tmem_ld_wait();
+                    uint32_t res[16];
+                    if (add_res) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) ld_nc_v4(p.a.R + rid_own * p.a.ldr + q * 32 + c * 8, res + 4 * c);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t out[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float lo = __uint_as_float(acc[c * 8 + 2 * e]), hi = __uint_as_float(acc[c * 8 + 2 * e + 1]);
+                            if (add_res) {
+                                lo += __uint_as_float(res[4 * c + e] << 16);
+                                hi += __uint_as_float(res[4 * c + e] & 0xffff0000u);
+                            }
+                            out[e] = pack_bf16(lo, hi);
+                        }
+                        const int chunk = q * 4 + c;
+                        st_shared_v4(stage + (uint32_t)(lane * kStageRowBytes + ((chunk ^ (lane & 7)) << 4)), out);
+                    }
+                }
+                // all tensor-memory reads of this slot are done: hand it back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[slot]));
+                // row-contiguous stores: 16 lanes cover one 256-byte row, two rows per instruction
+                __nv_bfloat16* outp = p.a.out[j];
+                const int64_t ldo = p.a.ldo[j];
+                const int chunk = lane & 15;
+#pragma unroll 4
+                for (int it = 0; it < 16; ++it) {
+                    const int lr = it * 2 + (lane >> 4);
+                    const int64_t rid = __shfl_sync(0xffffffffu, (long long)rid_own, lr);
+                    uint32_t v[4];
+                    ld_shared_v4(stage + (uint32_t)(lr * kStageRowBytes + ((chunk ^ (lr & 7)) << 4)), v);
+                    if (rid >= 0) st_global_v4(outp + rid * ldo + chunk * 8, v);
+                }
+                __syncwarp();
+            }
+        }
     }
+
+    tc_fence_before();
     __syncthreads();
-    for (int c = threadIdx.x; c < a.n_out; c += 128) {
-        float acc[kRows];
-#pragma unroll
-        for (int r = 0; r < kRows; ++r) acc[r] = 0.f;
-        const __nv_bfloat16* w = a.W + (size_t)c * 128;
-        for (int k = 0; k < 128; ++k) {
-            float wk = __bfloat162float(w[k]);
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) acc[r] = fmaf(xs[r][k], wk, acc[r]);
-        }
-        const int blk = c >> 7, cc = c & 127;
-#pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            if (rid[r] < 0) continue;
-            float y = acc[r];
-            if (blk == 0 && a.R) y += __bfloat162float(a.R[(size_t)rid[r] * a.ldr + cc]);
-            a.out[blk][(size_t)rid[r] * a.ldo[blk] + cc] = __float2bfloat16_rn(y);
-        }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
     }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// host side: tensor maps and launch
+// ---------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_mu;
+EncodeTiledFn g_encode = nullptr;
+bool g_attr_set[64] = {};
+int g_sm_count[64] = {};
+
+dg4_status get_encoder(EncodeTiledFn* fn) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_encode) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+            cudaGetLastError();
+            DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        }
+        g_encode = (EncodeTiledFn)p;
+    }
+    *fn = g_encode;
+    return DG4_OK;
+}
+
+// [rows, 128] bf16 row-major with leading dimension ld; box = 64 columns x 128 rows, 128-byte swizzle.
+dg4_status make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) {
+    EncodeTiledFn enc;
+    dg4_status s = get_encoder(&enc);
+    if (s != DG4_OK) return s;
+    cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)(ld * 2)};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return DG4_OK;
 }
 
 }  // namespace
@@ -52,8 +314,35 @@ dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st) {
     if (a.rows <= 0) return DG4_OK;
     if (a.n_out != 128 && a.n_out != 256 && a.n_out != 384)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "projection width %d is not supported", a.n_out);
-    unsigned blocks = (unsigned)((a.rows + kRows - 1) / kRows);
-    proj_simple_kernel<<<blocks, 128, 0, st>>>(a);
+    int dev = 0;
+    DG4_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_attr_set[dev]) {
+            DG4_CUDA_TRY(cudaFuncSetAttribute(proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            DG4_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+            g_attr_set[dev] = true;
+        }
+    }
+    ProjParams p;
+    p.a = a;
+    p.n_blocks = a.n_out / 128;
+    p.n_tiles = (a.rows + kTileM - 1) / kTileM;
+    p.status = a.status;
+    CUtensorMap map_a, map_w;
+    dg4_status s = make_map(&map_w, a.W, a.n_out, 128);
+    if (s != DG4_OK) return s;
+    if (!a.row_list) {
+        // contiguous rows: the map starts at the first row, so tile coordinates start at 0
+        s = make_map(&map_a, a.A + (int64_t)a.first * a.lda, a.rows, a.lda);
+        p.a.A = a.A;
+    } else {
+        map_a = map_w;   // unused by the kernel in list mode
+    }
+    if (s != DG4_OK) return s;
+    int grid = p.n_tiles < g_sm_count[dev] ? p.n_tiles : g_sm_count[dev];
+    proj_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
     dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;

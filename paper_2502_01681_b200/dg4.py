@@ -35,7 +35,7 @@ DG4_FLAG_RESIDUAL = 1
 
 EXPORTS = [
     "dg4_status_string", "dg4_last_error", "dg4_launch_count", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",
-    "dg4_graph_info", "dg4_graph_export", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
+    "dg4_graph_info", "dg4_graph_export", "dg4_graph_poll_status", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes",
 ]
@@ -96,6 +96,8 @@ def load():
     lib.dg4_graph_info.argtypes = [vp, ctypes.POINTER(dg4_graph_info_t)]
     lib.dg4_graph_export.restype = ctypes.c_int
     lib.dg4_graph_export.argtypes = [vp, ctypes.c_int, i32p, i64, ctypes.POINTER(i64)]
+    lib.dg4_graph_poll_status.restype = ctypes.c_int
+    lib.dg4_graph_poll_status.argtypes = [vp, i32p]
     lib.dg4_graph_device_array.restype = vp
     lib.dg4_graph_device_array.argtypes = [vp, ctypes.c_int]
     lib.dg4_qkv_project.restype = ctypes.c_int
@@ -207,6 +209,12 @@ def dg4_graph_export(g: Graph, which: int) -> np.ndarray:
     _check(lib.dg4_graph_export(g.handle, which, out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), out.shape[0],
                                 ctypes.byref(n)))
     return out[:n.value]
+
+
+def dg4_graph_poll_status(g: Graph) -> int:
+    out = ctypes.c_int32(0)
+    _check(load().dg4_graph_poll_status(g.handle, ctypes.byref(out)))
+    return int(out.value)
 
 
 def dg4_graph_device_array(g: Graph, which: int) -> int:
