@@ -45,7 +45,9 @@ typedef enum {
 typedef enum { DG4_F32 = 0, DG4_BF16 = 1 } dg4_dtype;
 
 enum {
-    DG4_FLAG_RESIDUAL = 1      /* output projection adds the layer's input row                */
+    DG4_FLAG_RESIDUAL = 1,     /* output projection adds the layer's input row                */
+    DG4_FLAG_LEVEL_LAUNCHES = 2 /* levelised layer: one group of kernel launches per level instead of the
+                                  single persistent kernel (same results; kept for comparison)   */
 };
 
 /* Per-call description of the attention layer. */

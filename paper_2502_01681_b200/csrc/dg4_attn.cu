@@ -12,62 +12,11 @@
 // softmax weight is 1, the case the paper skips as well).
 
 #include "dg4_internal.h"
+#include "dg4_attn_core.cuh"
 
 namespace {
 
-struct alignas(16) Piece { uint32_t w[4]; };
-
-__device__ __forceinline__ Piece ld_piece(const void* p) {
-    Piece r;
-    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
-    return r;
-}
-// streamed once: streaming (evict-first) policy so that gathered rows keep their place in the caches
-__device__ __forceinline__ Piece ld_piece_stream(const void* p) {
-    Piece r;
-    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
-    return r;
-}
-__device__ __forceinline__ void st_piece_stream(void* p, const Piece& v) {
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]) : "memory");
-}
-
-template <bool BF16> struct Elem;
-template <> struct Elem<true> {
-    static constexpr int kPerPiece = 8;
-    __device__ static __forceinline__ void unpack(const Piece& p, float* f) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            f[2 * i] = __uint_as_float(p.w[i] << 16);
-            f[2 * i + 1] = __uint_as_float(p.w[i] & 0xffff0000u);
-        }
-    }
-    __device__ static __forceinline__ Piece pack(const float* f) {
-        Piece p;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-            p.w[i] = *reinterpret_cast<uint32_t*>(&h);
-        }
-        return p;
-    }
-};
-template <> struct Elem<false> {
-    static constexpr int kPerPiece = 4;
-    __device__ static __forceinline__ void unpack(const Piece& p, float* f) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) f[i] = __uint_as_float(p.w[i]);
-    }
-    __device__ static __forceinline__ Piece pack(const float* f) {
-        Piece p;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) p.w[i] = __float_as_uint(f[i]);
-        return p;
-    }
-};
+using namespace attn;
 
 // BF16: storage type.  LPH: lanes per head.  MAXN: upper bound of the neighbourhood size (3 or 7).
 template <bool BF16, int LPH, int MAXN>
@@ -94,56 +43,16 @@ __global__ void __launch_bounds__(256) sparse_attn_kernel(dg4i_attn_args a) {
     for (int j = 0; j < MAXN; ++j) u[j] = __shfl_sync(0xffffffffu, my_idx, grp_base + j);
 #pragma unroll
     for (int j = 0; j < MAXN; ++j)
-        if (j < cnt) vq[j] = ld_piece((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
-    const bool need_scores = cnt > 1;
-    if (need_scores) {
+        if (j < cnt) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
+    if (cnt > 1) {
         qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
 #pragma unroll
         for (int j = 0; j < MAXN; ++j)
-            if (j < cnt) kq[j] = ld_piece((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
+            if (j < cnt) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
     }
-
     float acc[EPP];
-    if (!need_scores) {
-        Elem<BF16>::unpack(vq[0], acc);            // softmax over one element: weight exactly 1
-    } else {
-        float q[EPP];
-        Elem<BF16>::unpack(qp, q);
-        const float c = a.scale * 1.4426950408889634f;   // scores kept in log2 units
-        float s[MAXN];
-        float m = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < MAXN; ++j) {
-            float kf[EPP];
-            float dot = 0.f;
-            if (j < cnt) {
-                Elem<BF16>::unpack(kq[j], kf);
-#pragma unroll
-                for (int i = 0; i < EPP; ++i) dot = fmaf(q[i], kf[i], dot);
-            }
-#pragma unroll
-            for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            s[j] = (j < cnt) ? dot * c : -INFINITY;
-            m = fmaxf(m, s[j]);
-        }
-        float z = 0.f;
-#pragma unroll
-        for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
-#pragma unroll
-        for (int j = 0; j < MAXN; ++j) {
-            if (j < cnt) {
-                float p = exp2f(s[j] - m);
-                z += p;
-                float vf[EPP];
-                Elem<BF16>::unpack(vq[j], vf);
-#pragma unroll
-                for (int i = 0; i < EPP; ++i) acc[i] = fmaf(p, vf[i], acc[i]);
-            }
-        }
-        const float inv = 1.0f / z;
-#pragma unroll
-        for (int i = 0; i < EPP; ++i) acc[i] *= inv;
-    }
+    const unsigned mask = (G == 32) ? 0xffffffffu : (0xffffu << grp_base);
+    attend<BF16, LPH, MAXN>(qp, kq, vq, cnt, a.scale, mask, acc);
     if (live) st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
 }
 

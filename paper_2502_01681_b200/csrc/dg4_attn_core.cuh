@@ -1,0 +1,119 @@
+// Per-node arithmetic of the sparse attention shared by the stand-alone kernel and the levelised kernel:
+// a node's row is split into 16-byte pieces, one per lane; a head spans LPH adjacent lanes.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace attn {
+
+struct alignas(16) Piece { uint32_t w[4]; };
+
+__device__ __forceinline__ Piece ld_piece_nc(const void* p) {        // read-only for the whole kernel
+    Piece r;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ Piece ld_piece_cg(const void* p) {        // coherent at L2: data written by other CTAs
+    Piece r;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ Piece ld_piece_stream(const void* p) {    // streamed once: evict-first
+    Piece r;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_piece_stream(void* p, const Piece& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]) : "memory");
+}
+
+template <bool BF16> struct Elem;
+template <> struct Elem<true> {
+    static constexpr int kPerPiece = 8;
+    __device__ static __forceinline__ void unpack(const Piece& p, float* f) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(p.w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(p.w[i] & 0xffff0000u);
+        }
+    }
+    __device__ static __forceinline__ Piece pack(const float* f) {
+        Piece p;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            p.w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return p;
+    }
+};
+template <> struct Elem<false> {
+    static constexpr int kPerPiece = 4;
+    __device__ static __forceinline__ void unpack(const Piece& p, float* f) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = __uint_as_float(p.w[i]);
+    }
+    __device__ static __forceinline__ Piece pack(const float* f) {
+        Piece p;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p.w[i] = __float_as_uint(f[i]);
+        return p;
+    }
+};
+
+// Scores, softmax and weighted sum for one lane's piece of one node.  qp, kq[j], vq[j]: this lane's pieces
+// of the query row and of neighbour j's key / value rows (j < cnt; cnt >= 1).  `mask` names the lanes of this
+// node's group: they share cnt, so they take the same path and meet in the score-reduction shuffles; other
+// groups of the warp may be on a different path.
+template <bool BF16, int LPH, int MAXN>
+__device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const Piece* vq, int cnt, float scale,
+                                       unsigned mask, float* acc /*[kPerPiece]*/) {
+    constexpr int EPP = Elem<BF16>::kPerPiece;
+    if (cnt <= 1) {                                   // softmax over one element: weight exactly 1
+        Elem<BF16>::unpack(vq[0], acc);
+        return;
+    }
+    float q[EPP];
+    Elem<BF16>::unpack(qp, q);
+    const float c = scale * 1.4426950408889634f;      // scores kept in log2 units
+    float s[MAXN];
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < MAXN; ++j) {
+        float kf[EPP];
+        float dot = 0.f;
+        if (j < cnt) {
+            Elem<BF16>::unpack(kq[j], kf);
+#pragma unroll
+            for (int i = 0; i < EPP; ++i) dot = fmaf(q[i], kf[i], dot);
+        }
+#pragma unroll
+        for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
+        s[j] = (j < cnt) ? dot * c : -INFINITY;
+        m = fmaxf(m, s[j]);
+    }
+    float z = 0.f;
+#pragma unroll
+    for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXN; ++j) {
+        if (j < cnt) {
+            float p = exp2f(s[j] - m);
+            z += p;
+            float vf[EPP];
+            Elem<BF16>::unpack(vq[j], vf);
+#pragma unroll
+            for (int i = 0; i < EPP; ++i) acc[i] = fmaf(p, vf[i], acc[i]);
+        }
+    }
+    const float inv = 1.0f / z;
+#pragma unroll
+    for (int i = 0; i < EPP; ++i) acc[i] *= inv;
+}
+
+}  // namespace attn

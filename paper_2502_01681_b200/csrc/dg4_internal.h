@@ -102,3 +102,10 @@ struct dg4i_proj_args {
     int32_t* status = nullptr;         // device status word: receives DG4_ERR_TIMEOUT if a bounded wait runs out
 };
 dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st);
+
+// Persistent levelised kernel: Q and KV hold the projections of the layer's input for all nodes; H is updated in
+// place level by level.  `sync` is zeroed by the call and must hold dg4i_levelised_sync_bytes() bytes.
+size_t dg4i_levelised_sync_bytes(const dg4_graph* g);
+dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, const __nv_bfloat16* Q, __nv_bfloat16* KV,
+                                 __nv_bfloat16* H, int64_t ldh, const __nv_bfloat16* W_qkv, const __nv_bfloat16* W_o,
+                                 int32_t* sync, int32_t* status, cudaStream_t st);

@@ -48,7 +48,10 @@ struct Workspace {
     __nv_bfloat16* O;    // [n, 128]
 };
 
-size_t workspace_bytes(int64_t n) { return (size_t)n * 128 * 2 * 4 + 256; }
+size_t tensors_bytes(int64_t n) { return ((size_t)n * 128 * 2 * 4 + 255) & ~(size_t)255; }
+size_t workspace_bytes(const dg4_graph* g) {
+    return tensors_bytes(g->n) + ((dg4i_levelised_sync_bytes(g) + 255) & ~(size_t)255);
+}
 
 Workspace carve(void* ws, int64_t n) {
     Workspace w;
@@ -152,7 +155,7 @@ extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, 
 
 extern "C" size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* desc) {
     (void)desc;
-    return g ? workspace_bytes(g->n) : 0;
+    return g ? workspace_bytes(g) : 0;
 }
 
 namespace {
@@ -165,8 +168,8 @@ dg4_status check_layer_args(const dg4_graph* g, const dg4_desc* desc, const void
     CHECK(check_tensor("W_o", W_o, 128, 2, 128));
     if (!ws) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
     if ((((uintptr_t)ws) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
-    if (ws_bytes < workspace_bytes(g->n))
-        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", ws_bytes, workspace_bytes(g->n));
+    if (ws_bytes < workspace_bytes(g))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", ws_bytes, workspace_bytes(g));
     return DG4_OK;
 }
 }  // namespace
@@ -213,6 +216,14 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
 
+    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
+        // one persistent kernel walks the levels
+        int32_t* sync = (int32_t*)((char*)workspace + tensors_bytes(g->n));
+        return dg4i_levelised_launch(g, desc, w.Q, w.KV, (__nv_bfloat16*)H, ldh, (const __nv_bfloat16*)W_qkv,
+                                     (const __nv_bfloat16*)W_o, sync, status_word, st);
+    }
+
+    // alternative driver: one group of launches per level (attention, output projection, K|V refresh)
     const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;
     for (int l = 0; l < g->n_levels; ++l) {
         const int first = g->h_level_ptr[l], count = g->h_level_ptr[l + 1] - first;

@@ -29,6 +29,7 @@ DG4_ERR_TIMEOUT = -8
 
 DG4_F32, DG4_BF16 = 0, 1
 DG4_FLAG_RESIDUAL = 1
+DG4_FLAG_LEVEL_LAUNCHES = 2
 
 (DG4_ARR_NBR_PTR, DG4_ARR_NBR_IDX, DG4_ARR_LEVEL_PTR, DG4_ARR_LEVEL_NODES, DG4_ARR_PERM, DG4_ARR_CLASS_PTR,
  DG4_ARR_LEVEL_PERM, DG4_ARR_LEVEL_CLASS_PTR) = range(8)
@@ -146,8 +147,10 @@ def _ld(t):
     return int(t.stride(0))
 
 
-def desc(heads: int, dtype: int, scale: float, residual: bool = False, d: int = 128) -> dg4_desc:
-    return dg4_desc(d, heads, dtype, DG4_FLAG_RESIDUAL if residual else 0, float(scale))
+def desc(heads: int, dtype: int, scale: float, residual: bool = False, d: int = 128,
+         level_launches: bool = False) -> dg4_desc:
+    flags = (DG4_FLAG_RESIDUAL if residual else 0) | (DG4_FLAG_LEVEL_LAUNCHES if level_launches else 0)
+    return dg4_desc(d, heads, dtype, flags, float(scale))
 
 
 @dataclass

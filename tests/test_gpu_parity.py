@@ -233,7 +233,7 @@ def _weights(w, layers):
 
 
 def _run_layers_gpu(gr, w, xb, weights, mode):
-    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual)
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, level_launches=(mode == "level-launches"))
     ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
     h = dev_bf16(xb).clone()
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -250,7 +250,7 @@ def _run_layers_gpu(gr, w, xb, weights, mode):
 def _run_layers_checker(g, w, xb, weights, mode):
     ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
     h = f64_of_bits(xb)
-    if mode == "levelised":
+    if mode != "parallel":
         lptr, lnodes = orc.level_buckets(g.level)
     for (_, wq, _, wo) in weights:
         if mode == "parallel":
@@ -262,7 +262,9 @@ def _run_layers_checker(g, w, xb, weights, mode):
 
 
 @pytest.mark.parametrize("cfg,shrink,mode", [(2, 1, "parallel"), (2, 7, "parallel"), (5, 200, "parallel"),
-                                             (4, 20, "levelised"), (5, 400, "levelised"), (2, 10, "levelised")])
+                                             (4, 20, "levelised"), (5, 400, "levelised"), (2, 10, "levelised"),
+                                             (4, 5, "levelised"), (5, 50, "levelised"),
+                                             (4, 20, "level-launches"), (5, 400, "level-launches")])
 def test_layers_match_checker(cfg, shrink, mode):
     w = synth.workload(cfg, shrink)
     g = w.graph()
@@ -283,8 +285,10 @@ def test_levelised_differs_from_parallel_and_is_repeatable():
     weights = _weights(w, 1)
     a = _run_layers_gpu(gr, w, xb, weights, "levelised")
     b = _run_layers_gpu(gr, w, xb, weights, "levelised")
+    c = _run_layers_gpu(gr, w, xb, weights, "level-launches")
     p = _run_layers_gpu(gr, w, xb, weights, "parallel")
     assert (a == b).all()                                   # a race between levels would show up as a diff
+    assert rel_row_err(a, c).max() <= 1e-2                  # persistent kernel vs one launch group per level
     lvl0 = g.level == 0
     assert (a[lvl0] == p[lvl0]).all()                       # level-0 rows never see an updated row
     assert np.abs(a - p).max() > 0
