@@ -15,9 +15,10 @@
 //   4. refreshes the tile's K | V rows the same way: D2 = W_k * H'^T and W_v * H'^T, rounded and stored.
 // W_o, W_k and W_v stay resident in shared memory for the whole kernel (one TMA load each).
 //
-// Levels are separated by a counter barrier in global memory instead of kernel launches: each level has an
-// arrival counter; only CTAs that own a tile of the level arrive; the last one publishes "levels < l+1 done".
-// A CTA waits for that word only before a level in which it has work.  Launched cooperatively (all CTAs
+// Levels are separated by counters in global memory instead of kernel launches: each level has an arrival
+// counter that only the CTAs owning a tile of that level bump (release); before a level in which it has work a
+// CTA waits (acquire) until the previous non-empty level's counter is full.  Completion is transitive, because
+// every CTA that arrived on that level had itself waited for the level before it.  Launched cooperatively (all CTAs
 // co-resident).  Every wait is bounded; on expiry the kernel records DG4_ERR_TIMEOUT, raises an abort word that
 // every other wait polls, and all CTAs leave their loops, free tensor memory and return.
 
@@ -66,7 +67,6 @@ struct LevParams {
     int32_t residual;
     float scale;
     int32_t* arrive;                 // [n_levels], zero on entry
-    int32_t* done_level;             // zero on entry: number of leading levels that are complete
     int32_t* abort_word;             // zero on entry
     int32_t* status;
 };
@@ -93,8 +93,8 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release(int32_t* p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void red_release_add(int32_t* p, int v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t* r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
@@ -153,42 +153,78 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
     const int q4 = warp & 3, cg = warp >> 2;             // epilogue: TMEM lane quadrant and group of 8 node columns
     const int feat = q4 * 32 + lane;                     // output feature this thread holds in the epilogues
     uint32_t ph1 = 0, ph2 = 0;
-    int last_nonempty = -1;
+    int last_nonempty = -1, last_participants = 0;
     bool alive = true;
+    const int bid = blockIdx.x, nctas = gridDim.x;
+
+    // The index chain of a tile (node id -> list bounds -> neighbour ids) is three dependent loads that do not
+    // depend on any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
+    // level-to-level critical path: while level l is processed, the node id of this CTA's first tile of level
+    // l+3, the list bounds for level l+2 and the neighbour ids for level l+1 are in flight.
+    auto level_first = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv] : 0; };
+    auto level_size = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv + 1] - p.level_ptr[lv] : 0; };
+    auto stage_node = [&](int lv) -> int {            // node of (first tile of this CTA, this slot) at level lv
+        const int n_lv = level_size(lv);
+        const int r = bid * kTile + slot;
+        return (r < n_lv) ? p.level_nodes[level_first(lv) + r] : -1;
+    };
+    // pipeline state at the top of iteration l:
+    int v0 = -1, cnt0 = 1, idx0 = -1;                  // level l  : node id, list length, this lane's neighbour id
+    int vC = -1, cntC = 1, begC = 0;                   // level l+1: node id and list bounds
+    int vB = -1;                                       // level l+2: node id
+    {   // prologue: levels 0, 1, 2
+        v0 = stage_node(0);
+        vC = stage_node(1);
+        vB = stage_node(2);
+        int beg0 = 0;
+        if (v0 >= 0) { beg0 = p.nbr_ptr[v0]; cnt0 = p.nbr_ptr[v0 + 1] - beg0; }
+        if (vC >= 0) { begC = p.nbr_ptr[vC]; cntC = p.nbr_ptr[vC + 1] - begC; }
+        idx0 = (v0 >= 0 && sub < cnt0) ? p.nbr_idx[beg0 + sub] : v0;
+    }
 
     for (int l = 0; l < p.n_levels && alive; ++l) {
         const int first = p.level_ptr[l];
         const int n_l = p.level_ptr[l + 1] - first;
-        if (n_l <= 0) continue;
+        // issue the next load of every pipelined chain; the results are first used one level later
+        const int vA = stage_node(l + 3);                                               // level l+3: node id
+        int begB = 0, cntB = 1;                                                          // level l+2: list bounds
+        if (vB >= 0) { begB = p.nbr_ptr[vB]; cntB = p.nbr_ptr[vB + 1] - begB; }
+        const int idxC = (vC >= 0 && sub < cntC) ? p.nbr_idx[begC + sub] : vC;          // level l+1: neighbour id
         const int tiles = (n_l + kTile - 1) / kTile;
-        if ((int)blockIdx.x < tiles) {
+        if (n_l > 0 && bid < tiles) {
             bool waited = false;
-            for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-                // ---- indices of this tile (independent of other CTAs' results: loaded before the wait)
-                const int r = tile * kTile + slot;
-                const bool valid = r < n_l;
-                const int v = valid ? p.level_nodes[first + r] : -1;
-                int beg = 0, cnt = 1;
-                if (valid) { beg = p.nbr_ptr[v]; cnt = p.nbr_ptr[v + 1] - beg; }
-                const int my_idx = (valid && sub < cnt) ? p.nbr_idx[beg + sub] : v;
+            for (int tile = bid; tile < tiles; tile += nctas) {
+                int v, cnt, my_idx;
+                bool valid;
+                if (tile == bid) {
+                    v = v0; cnt = cnt0; my_idx = idx0; valid = v0 >= 0;
+                } else {                         // further tiles of a wide level: plain dependent loads
+                    const int r = tile * kTile + slot;
+                    valid = r < n_l;
+                    v = valid ? p.level_nodes[first + r] : -1;
+                    int beg = 0;
+                    cnt = 1;
+                    if (valid) { beg = p.nbr_ptr[v]; cnt = p.nbr_ptr[v + 1] - beg; }
+                    my_idx = (valid && sub < cnt) ? p.nbr_idx[beg + sub] : v;
+                }
 
                 if (!waited) {
-                    // ---- all lower levels must be complete (and nobody has given up)
+                    // ---- every tile of the previous non-empty level must have arrived (and nobody has given up)
                     if (tid == 0) {
                         int go = 1;
                         if (last_nonempty >= 0) {
                             uint32_t polls = 0;
-                            while (ld_acquire(p.done_level) < last_nonempty + 1) {
-                                if (++polls > (1u << 22) || ld_acquire(p.abort_word) != 0) { go = 0; break; }
-                                if (polls > 32) __nanosleep(64);
+                            while (ld_acquire(p.arrive + last_nonempty) < last_participants) {
+                                ++polls;
+                                if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(p.abort_word) != 0)) { go = 0; break; }
+                                if (polls > 64) __nanosleep(32);
                             }
                             if (!go && ld_acquire(p.abort_word) == 0) {
                                 atomicExch(p.abort_word, 1);
                                 if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
                             }
-                        } else if (ld_acquire(p.abort_word) != 0) {
-                            go = 0;
                         }
+                        if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = 0;
                         misc->go = go;
                     }
                     __syncthreads();
@@ -317,18 +353,17 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                 __syncthreads();    // the tile's shared buffers may be overwritten from here on
             }
             if (!alive) break;
-            // ---- this CTA's part of level l is in global memory: arrive; the last arrival publishes the level
-            if (tid == 0) {
-                __threadfence();
-                const int participants = tiles < (int)gridDim.x ? tiles : (int)gridDim.x;
-                const int old = atomicAdd(&p.arrive[l], 1);
-                if (old + 1 == participants) {
-                    __threadfence();
-                    st_release(p.done_level, l + 1);
-                }
-            }
+            // ---- this CTA's part of level l is in global memory: arrive on the level's counter (release)
+            if (tid == 0) red_release_add(p.arrive + l, 1);
         }
-        last_nonempty = l;
+        if (n_l > 0) {
+            last_nonempty = l;
+            last_participants = tiles < nctas ? tiles : nctas;
+        }
+        // rotate the pipeline by one level
+        v0 = vC; cnt0 = cntC; idx0 = idxC;
+        vC = vB; cntC = cntB; begC = begB;
+        vB = vA;
     }
 
     tc_fence_before();
@@ -429,7 +464,7 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, const
     p.Q = Q; p.KV = KV; p.H = H; p.ldh = ldh;
     p.nbr_ptr = g->nbr_ptr; p.nbr_idx = g->nbr_idx; p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
     p.n_levels = g->n_levels; p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
-    p.done_level = sync; p.abort_word = sync + 1; p.arrive = sync + 16; p.status = status;
+    p.abort_word = sync; p.arrive = sync + 16; p.status = status;
     const int grid = g_sm_count[dev];
     if (g->max_class <= 3) return launch_heads<3>(desc->heads, map_wo, map_wqkv, p, grid, st);
     return launch_heads<7>(desc->heads, map_wo, map_wqkv, p, grid, st);
