@@ -32,6 +32,17 @@ __device__ __forceinline__ void st_piece_stream(void* p, const Piece& v) {
                  :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]) : "memory");
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {      // 2^x, relative error about 2^-22
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_rcp(float x) {       // 1/x, relative error about 2^-23
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <bool BF16> struct Elem;
 template <> struct Elem<true> {
     static constexpr int kPerPiece = 8;
@@ -103,7 +114,7 @@ __device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const P
 #pragma unroll
     for (int j = 0; j < MAXN; ++j) {
         if (j < cnt) {
-            float p = exp2f(s[j] - m);
+            float p = fast_exp2(s[j] - m);
             z += p;
             float vf[EPP];
             Elem<BF16>::unpack(vq[j], vf);
@@ -111,7 +122,7 @@ __device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const P
             for (int i = 0; i < EPP; ++i) acc[i] = fmaf(p, vf[i], acc[i]);
         }
     }
-    const float inv = 1.0f / z;
+    const float inv = fast_rcp(z);
 #pragma unroll
     for (int i = 0; i < EPP; ++i) acc[i] *= inv;
 }

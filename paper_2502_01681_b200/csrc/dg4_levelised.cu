@@ -3,13 +3,13 @@
 //
 // Q | K | V of every node have been projected from the layer's input beforehand (a node's own query, key and
 // value always come from its row as it was when the layer started).  This kernel then walks the levels.
-// For a tile of 32 nodes of the current level a CTA
+// For a tile of 16 nodes of the current level a CTA
 //   1. gathers the K | V rows of every neighbour (16 lanes per node, 16 bytes per lane), computes scores,
-//      softmax and the weighted value sum in registers, and writes the 32 x 128 attention tile into shared
+//      softmax and the weighted value sum in registers, and writes the 16 x 128 attention tile into shared
 //      memory in the tensor core's K-major, 128-byte-swizzled operand layout;
 //   2. runs the output projection TRANSPOSED on the tensor cores: D1[feature, node] = W_o * O^T
-//      (tcgen05.mma, M = 128 features, N = 32 nodes, K = 128), so a tile of only 32 nodes costs a quarter of a
-//      128-row tile and all 16 warps take part in the epilogue (128 TMEM lanes x 32 columns);
+//      (tcgen05.mma, M = 128 features, N = 16 nodes, K = 128), so a small tile costs a fraction of a
+//      128-row tile and all warps take part in the epilogue (128 TMEM lanes x 16 columns);
 //   3. adds the residual, rounds to bf16, writes the new rows to H and -- in operand layout again -- to shared
 //      memory, and
 //   4. refreshes the tile's K | V rows the same way: D2 = W_k * H'^T and W_v * H'^T, rounded and stored.
@@ -33,17 +33,17 @@ namespace {
 using namespace sm100;
 using namespace attn;
 
-constexpr int kThreads = 512;
-constexpr int kTile = 32;                    // nodes per tile
+constexpr int kTile = 16;                    // nodes per tile
+constexpr int kThreads = kTile * 16;         // 16 lanes per node
 constexpr int kWBlock = 2 * 128 * 128;       // one 128 x 128 bf16 weight block: two K-halves of 16 KiB
-constexpr int kBHalf = kTile * 128;          // K-half of a 32-row operand tile: 4 KiB
-constexpr int kTmemCols = 128;
+constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
+constexpr int kTmemCols = 64;
 
 constexpr int kOffW = 0;                          // W_o | W_k | W_v : 96 KiB
-constexpr int kOffO = 3 * kWBlock;                // attention tile (operand layout)      8 KiB
-constexpr int kOffHp = kOffO + 2 * kBHalf;        // new rows (operand layout)            8 KiB
-constexpr int kOffHres = kOffHp + 2 * kBHalf;     // residual rows, plain [32][256 B]     8 KiB
-constexpr int kOffKV = kOffHres + kTile * 256;    // K|V staging, plain [32][512 B]      16 KiB
+constexpr int kOffO = 3 * kWBlock;                // attention tile (operand layout)
+constexpr int kOffHp = kOffO + 2 * kBHalf;        // new rows (operand layout)
+constexpr int kOffHres = kOffHp + 2 * kBHalf;     // residual rows, plain [kTile][256 B]
+constexpr int kOffKV = kOffHres + kTile * 256;    // K|V staging, plain [kTile][512 B]
 constexpr int kOffMisc = kOffKV + kTile * 512;
 constexpr int kSmemBytes = kOffMisc + 512 + 1024;
 
@@ -105,7 +105,7 @@ __device__ __forceinline__ uint16_t bf16_bits(float x) {
     __nv_bfloat16 h = __float2bfloat16_rn(x);
     return *reinterpret_cast<uint16_t*>(&h);
 }
-// byte offset of element k (0..127) of row `row` in a 32-row operand tile (two K-halves, 128-byte swizzle)
+// byte offset of element k (0..127) of row `row` in a kTile-row operand tile (two K-halves, 128-byte swizzle)
 __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
     return (uint32_t)((k >> 6) * kBHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
 }
@@ -150,6 +150,7 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
     }
 
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
+    static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
     const int q4 = warp & 3, cg = warp >> 2;             // epilogue: TMEM lane quadrant and group of 8 node columns
     const int feat = q4 * 32 + lane;                     // output feature this thread holds in the epilogues
     uint32_t ph1 = 0, ph2 = 0;
@@ -306,7 +307,7 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                         for (int ks = 0; ks < 8; ++ks) {
                             const uint32_t a_off = (uint32_t)((1 + blk) * kWBlock + (ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
                             const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                            mma_bf16(tmem + (uint32_t)(32 + 32 * blk), smem_desc_sw128(sW + a_off),
+                            mma_bf16(tmem + (uint32_t)(kTile + kTile * blk), smem_desc_sw128(sW + a_off),
                                      smem_desc_sw128(sHp + b_off), idesc, ks > 0 ? 1u : 0u);
                         }
                     }
@@ -327,8 +328,8 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                 tc_fence_after();
                 {
                     uint32_t dk[8], dv[8];
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(32 + cg * 8), dk);
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(64 + cg * 8), dv);
+                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile + cg * 8), dk);
+                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(2 * kTile + cg * 8), dv);
                     tmem_ld_wait();
 #pragma unroll
                     for (int nn = 0; nn < 8; ++nn) {
