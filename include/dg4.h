@@ -83,7 +83,10 @@ typedef enum {
     DG4_ARR_CLASS_PTR = 5,      /* [n_chunks, max_class+1]  start of class c+1 of a chunk in PERM;
                                                          last entry of a row = end of the chunk        */
     DG4_ARR_LEVEL_PERM = 6,     /* [n]                   ids ordered by (level, |N(v)|, id)              */
-    DG4_ARR_LEVEL_CLASS_PTR = 7 /* [n_levels, max_class+1]  same as CLASS_PTR with levels as segments    */
+    DG4_ARR_LEVEL_CLASS_PTR = 7,/* [n_levels, max_class+1]  same as CLASS_PTR with levels as segments    */
+    DG4_ARR_NBR_PAD = 8         /* [n, max_class+1]      fixed-width neighbour table read by the kernels:
+                                                         |N(v)|, then the members other than v ascending,
+                                                         then v repeated as filler                       */
 } dg4_array_id;
 
 const char* dg4_status_string(dg4_status s);

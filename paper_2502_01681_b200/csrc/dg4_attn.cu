@@ -19,62 +19,99 @@ namespace {
 using namespace attn;
 
 // BF16: storage type.  LPH: lanes per head.  MAXN: upper bound of the neighbourhood size (3 or 7).
+// Persistent: a group of G lanes walks the nodes slot, slot + (groups in the grid), ... so that the nodes in
+// flight across the GPU at any moment are a contiguous id range (their gathered rows overlap in L2).  The
+// fixed-width neighbour entry of the NEXT node is fetched while the current node's rows are in flight, which
+// takes the index lookup off the per-node dependency chain (one memory round trip per node instead of three).
 template <bool BF16, int LPH, int MAXN>
 __global__ void __launch_bounds__(256) sparse_attn_kernel(dg4i_attn_args a) {
     constexpr int G = BF16 ? 16 : 32;              // lanes per node
     constexpr int EPP = Elem<BF16>::kPerPiece;     // elements per 16-byte piece
     constexpr int ES = BF16 ? 2 : 4;
+    constexpr int W = MAXN + 1;                    // width of a neighbour-table entry
     const int lane = threadIdx.x & 31;
     const int sub = lane & (G - 1);                // lane within the node's group
     const int grp_base = lane - sub;               // first lane of the group inside the warp
-    int slot = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G);
-    const bool live = slot < a.count;
-    if (!live) slot = a.count - 1;                 // keep whole warps converged for the shuffles
-    const int v = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
-
-    const int beg = a.nbr_ptr[v];
-    const int cnt = a.nbr_ptr[v + 1] - beg;
-    int my_idx = (sub < cnt) ? a.nbr_idx[beg + sub] : v;
-
+    const unsigned mask = (G == 32) ? 0xffffffffu : (0xffffu << grp_base);
+    const int stride = (int)(gridDim.x * (blockDim.x / G));
+    int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) / G);
     const size_t col = (size_t)sub * EPP * ES;     // byte offset of this lane's piece inside a row
-    Piece kq[MAXN], vq[MAXN], qp;
-    int u[MAXN];
+
+    int v_next = -1, pad_next = 0;
+    if (slot < a.count) {
+        v_next = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
+        if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+    }
+    for (; slot < a.count; slot += stride) {
+        const int v = v_next;
+        const int pad = pad_next;
+        {   // next node of this group: its table entry arrives while this node's rows are gathered
+            const int s2 = slot + stride;
+            if (s2 < a.count) {
+                v_next = a.node_list ? a.node_list[a.first + s2] : a.first + s2;
+                if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+            }
+        }
+        const int cnt = __shfl_sync(mask, pad, grp_base);
+        Piece kq[MAXN], vq[MAXN], qp;
+        int u[MAXN];
+        u[0] = v;
 #pragma unroll
-    for (int j = 0; j < MAXN; ++j) u[j] = __shfl_sync(0xffffffffu, my_idx, grp_base + j);
-#pragma unroll
-    for (int j = 0; j < MAXN; ++j)
-        if (j < cnt) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
-    if (cnt > 1) {
-        qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
+        for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(mask, pad, grp_base + j);
 #pragma unroll
         for (int j = 0; j < MAXN; ++j)
-            if (j < cnt) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
+            if (j < cnt) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
+        if (cnt > 1) {
+            qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
+#pragma unroll
+            for (int j = 0; j < MAXN; ++j)
+                if (j < cnt) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
+        }
+        float acc[EPP];
+        attend<BF16, LPH, MAXN>(qp, kq, vq, cnt, a.scale, mask, acc);
+        st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
     }
-    float acc[EPP];
-    const unsigned mask = (G == 32) ? 0xffffffffu : (0xffffu << grp_base);
-    attend<BF16, LPH, MAXN>(qp, kq, vq, cnt, a.scale, mask, acc);
-    if (live) st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
+}
+
+struct LaunchShape { int sm_count = 0; int blocks_per_sm = 0; };
+
+template <bool BF16, int LPH, int MAXN>
+dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
+    constexpr int G = BF16 ? 16 : 32;
+    const int threads = 256;
+    static LaunchShape shape[64];
+    int dev = 0;
+    DG4_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
+    if (shape[dev].sm_count == 0) {
+        int sms = 0, per_sm = 0;
+        DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sparse_attn_kernel<BF16, LPH, MAXN>, threads, 0));
+        shape[dev].blocks_per_sm = per_sm > 0 ? per_sm : 1;
+        shape[dev].sm_count = sms;
+    }
+    const int nodes_per_block = threads / G;
+    const int64_t needed = ((int64_t)a.count + nodes_per_block - 1) / nodes_per_block;
+    const int64_t resident = (int64_t)shape[dev].sm_count * shape[dev].blocks_per_sm;
+    const unsigned blocks = (unsigned)(needed < resident ? needed : resident);
+    sparse_attn_kernel<BF16, LPH, MAXN><<<blocks, threads, 0, st>>>(a);
+    dg4i_count_launch();
+    DG4_CUDA_TRY(cudaGetLastError());
+    return DG4_OK;
 }
 
 template <bool BF16, int MAXN>
 dg4_status launch_for_heads(const dg4i_attn_args& a, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
-    const int threads = 256;
-    const int nodes_per_block = threads / G;
-    const unsigned blocks = (unsigned)((a.count + nodes_per_block - 1) / nodes_per_block);
-    const int lph = G / a.heads;
-    switch (lph) {
-        case 1: sparse_attn_kernel<BF16, 1, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        case 2: sparse_attn_kernel<BF16, 2, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        case 4: sparse_attn_kernel<BF16, 4, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        case 8: sparse_attn_kernel<BF16, 8, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        case 16: sparse_attn_kernel<BF16, 16, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        case 32: sparse_attn_kernel<BF16, 32, MAXN><<<blocks, threads, 0, st>>>(a); break;
-        default: DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
+    switch (G / a.heads) {
+        case 1: return launch_one<BF16, 1, MAXN>(a, st);
+        case 2: return launch_one<BF16, 2, MAXN>(a, st);
+        case 4: return launch_one<BF16, 4, MAXN>(a, st);
+        case 8: return launch_one<BF16, 8, MAXN>(a, st);
+        case 16: return launch_one<BF16, 16, MAXN>(a, st);
+        case 32: if (G == 32) return launch_one<BF16, (G == 32 ? 32 : 16), MAXN>(a, st);
     }
-    dg4i_count_launch();
-    DG4_CUDA_TRY(cudaGetLastError());
-    return DG4_OK;
+    DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
 }
 
 }  // namespace

@@ -62,6 +62,17 @@ template <> struct Elem<true> {
         }
         return p;
     }
+    // sum over the piece of q[i] * k[i], products and sums in fp32 (a bf16 x bf16 product is exact in fp32).
+    // The mixed-precision FMA takes the bf16 halves of the packed words directly: no unpacking instructions.
+    __device__ static __forceinline__ float dot(const Piece& q, const Piece& k) {
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            asm("{\n\t.reg .b16 ql, qh, kl, kh;\n\tmov.b32 {ql, qh}, %1;\n\tmov.b32 {kl, kh}, %2;\n\t"
+                "fma.rn.f32.bf16 %0, ql, kl, %0;\n\tfma.rn.f32.bf16 %0, qh, kh, %0;\n\t}"
+                : "+f"(acc) : "r"(q.w[i]), "r"(k.w[i]));
+        return acc;
+    }
 };
 template <> struct Elem<false> {
     static constexpr int kPerPiece = 4;
@@ -74,6 +85,12 @@ template <> struct Elem<false> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) p.w[i] = __float_as_uint(f[i]);
         return p;
+    }
+    __device__ static __forceinline__ float dot(const Piece& q, const Piece& k) {
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc = fmaf(__uint_as_float(q.w[i]), __uint_as_float(k.w[i]), acc);
+        return acc;
     }
 };
 
@@ -89,20 +106,13 @@ __device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const P
         Elem<BF16>::unpack(vq[0], acc);
         return;
     }
-    float q[EPP];
-    Elem<BF16>::unpack(qp, q);
     const float c = scale * 1.4426950408889634f;      // scores kept in log2 units
     float s[MAXN];
     float m = -INFINITY;
 #pragma unroll
     for (int j = 0; j < MAXN; ++j) {
-        float kf[EPP];
         float dot = 0.f;
-        if (j < cnt) {
-            Elem<BF16>::unpack(kq[j], kf);
-#pragma unroll
-            for (int i = 0; i < EPP; ++i) dot = fmaf(q[i], kf[i], dot);
-        }
+        if (j < cnt) dot = Elem<BF16>::dot(qp, kq[j]);
 #pragma unroll
         for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
         s[j] = (j < cnt) ? dot * c : -INFINITY;

@@ -57,7 +57,8 @@ __global__ void cone_count_kernel(int n, const int32_t* __restrict__ row_ptr, co
 }
 
 __global__ void cone_fill_kernel(int n, const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                                 int hops, const int32_t* __restrict__ nbr_ptr, int32_t* __restrict__ nbr_idx) {
+                                 int hops, const int32_t* __restrict__ nbr_ptr, int32_t* __restrict__ nbr_idx,
+                                 int pad_width, int32_t* __restrict__ nbr_pad) {
     int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= n) return;
     int m[6];
@@ -65,6 +66,10 @@ __global__ void cone_fill_kernel(int n, const int32_t* __restrict__ row_ptr, con
     int o = nbr_ptr[v];
     nbr_idx[o] = v;
     for (int i = 0; i < c; ++i) nbr_idx[o + 1 + i] = m[i];
+    // fixed-width copy for the attention kernels: [ |N(v)|, the members other than v ascending, v as filler ]
+    int32_t* row = nbr_pad + (size_t)v * pad_width;
+    row[0] = c + 1;
+    for (int i = 1; i < pad_width; ++i) row[i] = (i - 1 < c) ? m[i - 1] : v;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -277,7 +282,7 @@ dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only
     dg4i_count_launch();
     if ((s = exclusive_scan(g->nbr_ptr, g->nbr_ptr, (int64_t)n + 1, g->block_sums, st)) != DG4_OK) return s;
     if (sizes_only) return DG4_OK;
-    cone_fill_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr, g->nbr_idx);
+    cone_fill_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr, g->nbr_idx, g->pad_width, g->nbr_pad);
     dg4i_count_launch();
 
     // level buckets
@@ -328,7 +333,7 @@ struct DeviceGuard {
 
 void free_graph(dg4_graph* g) {
     if (!g) return;
-    int32_t* bufs[] = {g->row_ptr, g->col_idx, g->level, g->nbr_ptr, g->nbr_idx, g->level_ptr, g->level_nodes,
+    int32_t* bufs[] = {g->nbr_pad, g->row_ptr, g->col_idx, g->level, g->nbr_ptr, g->nbr_idx, g->level_ptr, g->level_nodes,
                        g->perm, g->class_ptr, g->level_perm, g->level_class_ptr, g->seq_a, g->seq_b, g->hist,
                        g->block_sums, g->dev_status};
     for (int32_t* b : bufs)
@@ -396,6 +401,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     g->e = n_edges;
     g->hops = hops;
     g->max_class = (1 << (hops + 1)) - 1;
+    g->pad_width = g->max_class + 1;           // 4 or 8 int32: 16 or 32 bytes per node
     g->n_levels = max_level + 1;
     g->perm_chunk = (perm_chunk >= n_nodes) ? 0 : perm_chunk;
     g->n_chunks = g->perm_chunk > 0 ? (n_nodes + g->perm_chunk - 1) / g->perm_chunk : 1;
@@ -449,6 +455,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     if ((ce = cudaMemcpy(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
     g->n_nbr = total;
     TRY_ALLOC(g->nbr_idx, g->n_nbr);
+    TRY_ALLOC(g->nbr_pad, n * g->pad_width);
 #undef TRY_ALLOC
     if ((s = dg4i_graph_device_pass(g, 0, false)) != DG4_OK) return fail(s);
 
@@ -492,6 +499,7 @@ const int32_t* array_of(const dg4_graph* g, dg4_array_id which, int64_t* len) {
     switch (which) {
         case DG4_ARR_NBR_PTR: *len = (int64_t)g->n + 1; return g->nbr_ptr;
         case DG4_ARR_NBR_IDX: *len = g->n_nbr; return g->nbr_idx;
+        case DG4_ARR_NBR_PAD: *len = (int64_t)g->n * g->pad_width; return g->nbr_pad;
         case DG4_ARR_LEVEL_PTR: *len = (int64_t)g->n_levels + 1; return g->level_ptr;
         case DG4_ARR_LEVEL_NODES: *len = g->n; return g->level_nodes;
         case DG4_ARR_PERM: *len = g->n; return g->perm;

@@ -49,6 +49,8 @@ struct dg4_graph {
     // built by graph prep
     int32_t* nbr_ptr = nullptr;          // [n+1]
     int32_t* nbr_idx = nullptr;          // [n_nbr]
+    int32_t* nbr_pad = nullptr;          // [n, pad_width]: |N(v)|, then the members other than v (filler: v)
+    int32_t pad_width = 0;               // max_class + 1
     int32_t* level_ptr = nullptr;        // [n_levels+1]
     int32_t* level_nodes = nullptr;      // [n]
     int32_t* perm = nullptr;             // [n]
@@ -76,8 +78,7 @@ struct dg4i_attn_args {
     const void* K; int64_t ldk;
     const void* V; int64_t ldv;
     void* O; int64_t ldo;
-    const int32_t* nbr_ptr;
-    const int32_t* nbr_idx;
+    const int32_t* nbr_pad;     // [n, max_nbr + 1] fixed-width neighbour table
     const int32_t* node_list;   // nullable: node ids to process; else ids first..first+count-1
     int32_t first;
     int32_t count;

@@ -66,7 +66,7 @@ dg4i_attn_args attn_args(const dg4_graph* g, const dg4_desc* d, const void* Q, i
                          int64_t ldk, const void* V, int64_t ldv, void* O, int64_t ldo) {
     dg4i_attn_args a;
     a.Q = Q; a.ldq = ldq; a.K = K; a.ldk = ldk; a.V = V; a.ldv = ldv; a.O = O; a.ldo = ldo;
-    a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.nbr_pad = g->nbr_pad; a.node_list = nullptr; a.first = 0; a.count = g->n;
     a.heads = d->heads; a.max_nbr = g->max_class; a.dtype = d->dtype; a.scale = d->scale;
     return a;
 }

@@ -32,7 +32,7 @@ DG4_FLAG_RESIDUAL = 1
 DG4_FLAG_LEVEL_LAUNCHES = 2
 
 (DG4_ARR_NBR_PTR, DG4_ARR_NBR_IDX, DG4_ARR_LEVEL_PTR, DG4_ARR_LEVEL_NODES, DG4_ARR_PERM, DG4_ARR_CLASS_PTR,
- DG4_ARR_LEVEL_PERM, DG4_ARR_LEVEL_CLASS_PTR) = range(8)
+ DG4_ARR_LEVEL_PERM, DG4_ARR_LEVEL_CLASS_PTR, DG4_ARR_NBR_PAD) = range(9)
 
 EXPORTS = [
     "dg4_status_string", "dg4_last_error", "dg4_launch_count", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",

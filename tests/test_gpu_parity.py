@@ -27,6 +27,10 @@ def _check_graph_arrays(rp, ci, level, hops, chunk):
     eff_chunk = 0 if chunk >= n else chunk
     perm, cptr = orc.class_order(np.arange(n, dtype=np.int32), orc.chunk_ptr(n, eff_chunk), ptr, mc)
     lperm, lcptr = orc.class_order(lnodes, lptr, ptr, mc)
+    pad = np.repeat(np.arange(n, dtype=np.int32)[:, None], mc + 1, axis=1)       # the same lists, fixed width
+    pad[:, 0] = np.diff(ptr)
+    for v in range(n):
+        pad[v, 1:pad[v, 0]] = idx[ptr[v] + 1:ptr[v + 1]]
 
     def same(which, want):
         got = dg4.dg4_graph_export(g, which)
@@ -35,6 +39,7 @@ def _check_graph_arrays(rp, ci, level, hops, chunk):
     for _ in range(2):                      # the second round checks that a rebuild reproduces everything
         same(dg4.DG4_ARR_NBR_PTR, ptr)
         same(dg4.DG4_ARR_NBR_IDX, idx)
+        same(dg4.DG4_ARR_NBR_PAD, pad)
         same(dg4.DG4_ARR_LEVEL_PTR, lptr)
         same(dg4.DG4_ARR_LEVEL_NODES, lnodes)
         same(dg4.DG4_ARR_PERM, perm)
