@@ -14,6 +14,11 @@
 #include "dg4_internal.h"
 #include "dg4_attn_core.cuh"
 
+// resident blocks per SM the compiler must allow for (caps registers per thread)
+#ifndef DG4_ATTN_MIN_BLOCKS
+#define DG4_ATTN_MIN_BLOCKS 2
+#endif
+
 namespace {
 
 using namespace attn;
@@ -24,7 +29,7 @@ using namespace attn;
 // fixed-width neighbour entry of the NEXT node is fetched while the current node's rows are in flight, which
 // takes the index lookup off the per-node dependency chain (one memory round trip per node instead of three).
 template <bool BF16, int LPH, int MAXN>
-__global__ void __launch_bounds__(256) sparse_attn_kernel(dg4i_attn_args a) {
+__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(dg4i_attn_args a) {
     constexpr int G = BF16 ? 16 : 32;              // lanes per node
     constexpr int EPP = Elem<BF16>::kPerPiece;     // elements per 16-byte piece
     constexpr int ES = BF16 ? 2 : 4;
