@@ -221,7 +221,8 @@ def run_ours(args, w):
     gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local)
     info = gr.info
     dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual)
-    ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, w.layers)),
+                     dtype=torch.uint8, device="cuda")
     x_dev = x_host.cuda().view(torch.bfloat16)
     h_par = torch.empty_like(x_dev)
     h_lev = torch.empty_like(x_dev)
@@ -256,8 +257,8 @@ def run_ours(args, w):
             mark("attn", lambda: dg4.dg4_sparse_attn_fwd(gr, dsc, q_v, kv_v[:, :128], kv_v[:, 128:], o_v))
             mark("out", lambda: dg4.dg4_out_project(gr, dsc, o_v, wo[l], h_par, h_par))
         h_lev.copy_(x_dev)
-        for l in range(w.layers if not args.no_levelised else 0):
-            mark("levelised", lambda: dg4.dg4_layer_fwd_levelised(gr, dsc, h_lev, wq[l], wo[l], ws, status))
+        if not args.no_levelised:        # all layers in one call: they run as a wavefront over the levels
+            mark("levelised", lambda: dg4.dg4_layers_fwd_levelised(gr, dsc, h_lev, wq, wo, ws, status))
         if record:
             stage_ev.append(marks)
 
@@ -323,8 +324,8 @@ def run_ours(args, w):
         hp = x2.clone()
         for l in range(w.layers):
             dg4.dg4_layer_fwd_parallel(gr2, dsc, hp, wq[l], wo[l], hp, ws)
-        for l in range(w.layers if not args.no_levelised else 0):
-            dg4.dg4_layer_fwd_levelised(gr2, dsc, x2, wq[l], wo[l], ws, status)
+        if not args.no_levelised:
+            dg4.dg4_layers_fwd_levelised(gr2, dsc, x2, wq, wo, ws, status)
         out_host.copy_(x2.view(torch.int16), non_blocking=True)
         torch.cuda.synchronize()
         dg4.dg4_graph_destroy(gr2)

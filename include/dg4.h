@@ -229,6 +229,21 @@ dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc* desc,
                                    void* workspace, size_t workspace_bytes,
                                    int32_t* device_status, void* stream);
 
+/*
+ * Several levelised layers in one call, run as a wavefront (Sec. 3.4's level order, applied to a stack of
+ * layers): the result is exactly that of n_layers successive dg4_layer_fwd_levelised calls with W_qkv[k], W_o[k],
+ * but layer k+1 starts on a level as soon as layer k has finished that level, so the chain of dependent steps is
+ * n_levels + n_layers - 1 long instead of n_layers * n_levels.
+ *   n_layers     1 .. 8
+ *   W_qkv, W_o   host arrays of n_layers device pointers ([3d, d] and [d, d] bf16 each)
+ *   workspace    device, at least dg4_layers_workspace_bytes() bytes, 256-byte aligned
+ * Other arguments as for dg4_layer_fwd_levelised.
+ */
+size_t dg4_layers_workspace_bytes(const dg4_graph* g, const dg4_desc* desc, int32_t n_layers);
+dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                    int32_t n_layers, const void* const* W_qkv, const void* const* W_o,
+                                    void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -49,8 +49,14 @@ struct Workspace {
 };
 
 size_t tensors_bytes(int64_t n) { return ((size_t)n * 128 * 2 * 4 + 255) & ~(size_t)255; }
-size_t workspace_bytes(const dg4_graph* g) {
-    return tensors_bytes(g->n) + ((dg4i_levelised_sync_bytes(g) + 255) & ~(size_t)255);
+size_t sync_bytes(const dg4_graph* g, int n_layers) { return (dg4i_levelised_sync_bytes(g, n_layers) + 255) & ~(size_t)255; }
+size_t workspace_bytes(const dg4_graph* g) { return tensors_bytes(g->n) + sync_bytes(g, 1); }
+// several levelised layers in one call: per layer a Q table [n,128] and a K|V table [n,256], then the counters
+size_t layer_tables_bytes(int64_t n) { return ((size_t)n * 768 + 255) & ~(size_t)255; }
+size_t layers_workspace_bytes(const dg4_graph* g, int n_layers) {
+    size_t multi = layer_tables_bytes(g->n) * (size_t)n_layers + sync_bytes(g, n_layers);
+    size_t single = workspace_bytes(g);          // the per-level-launch driver reuses one layer's workspace
+    return multi > single ? multi : single;
 }
 
 Workspace carve(void* ws, int64_t n) {
@@ -219,8 +225,11 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
         // one persistent kernel walks the levels
         int32_t* sync = (int32_t*)((char*)workspace + tensors_bytes(g->n));
-        return dg4i_levelised_launch(g, desc, w.Q, w.KV, (__nv_bfloat16*)H, ldh, (const __nv_bfloat16*)W_qkv,
-                                     (const __nv_bfloat16*)W_o, sync, status_word, st);
+        __nv_bfloat16* q1[1] = {w.Q};
+        __nv_bfloat16* kv1[1] = {w.KV};
+        const __nv_bfloat16* wq1[1] = {(const __nv_bfloat16*)W_qkv};
+        const __nv_bfloat16* wo1[1] = {(const __nv_bfloat16*)W_o};
+        return dg4i_levelised_launch(g, desc, 1, q1, kv1, (__nv_bfloat16*)H, ldh, wq1, wo1, sync, status_word, st);
     }
 
     // alternative driver: one group of launches per level (attention, output projection, K|V refresh)
@@ -248,4 +257,62 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
         }
     }
     return DG4_OK;
+}
+
+extern "C" size_t dg4_layers_workspace_bytes(const dg4_graph* g, const dg4_desc* desc, int32_t n_layers) {
+    (void)desc;
+    if (!g || n_layers < 1 || n_layers > DG4I_MAX_LAYERS) return 0;
+    return layers_workspace_bytes(g, n_layers);
+}
+
+extern "C" dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                                int32_t n_layers, const void* const* W_qkv, const void* const* W_o,
+                                                void* workspace, size_t workspace_bytes_, int32_t* device_status,
+                                                void* stream) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    if (n_layers < 1 || n_layers > DG4I_MAX_LAYERS)
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "n_layers = %d: between 1 and %d layers per call", n_layers, DG4I_MAX_LAYERS);
+    if (!W_qkv || !W_o) DG4_FAIL(DG4_ERR_INVALID_ARG, "null weight list");
+    CHECK(check_desc(desc, true));
+    CHECK(check_tensor("H", H, ldh, 2, 128));
+    for (int k = 0; k < n_layers; ++k) {
+        CHECK(check_tensor("W_qkv[k]", W_qkv[k], 128, 2, 128));
+        CHECK(check_tensor("W_o[k]", W_o[k], 128, 2, 128));
+    }
+    if (!workspace) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
+    if ((((uintptr_t)workspace) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+    if (workspace_bytes_ < layers_workspace_bytes(g, n_layers))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", workspace_bytes_,
+                 layers_workspace_bytes(g, n_layers));
+    cudaStream_t st = (cudaStream_t)stream;
+
+    if (desc->flags & DG4_FLAG_LEVEL_LAUNCHES) {       // comparison driver: layer after layer, a launch group per level
+        for (int k = 0; k < n_layers; ++k)
+            CHECK(dg4_layer_fwd_levelised(g, desc, H, ldh, W_qkv[k], W_o[k], workspace, workspace_bytes_, device_status, stream));
+        return DG4_OK;
+    }
+
+    if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
+    int32_t* status_word = device_status ? device_status : g->dev_status;
+    __nv_bfloat16* q[DG4I_MAX_LAYERS];
+    __nv_bfloat16* kv[DG4I_MAX_LAYERS];
+    const __nv_bfloat16* wq[DG4I_MAX_LAYERS];
+    const __nv_bfloat16* wo[DG4I_MAX_LAYERS];
+    const size_t per_layer = layer_tables_bytes(g->n);
+    for (int k = 0; k < n_layers; ++k) {
+        char* basep = (char*)workspace + per_layer * (size_t)k;
+        q[k] = (__nv_bfloat16*)basep;
+        kv[k] = (__nv_bfloat16*)(basep + (size_t)g->n * 256);
+        wq[k] = (const __nv_bfloat16*)W_qkv[k];
+        wo[k] = (const __nv_bfloat16*)W_o[k];
+    }
+    int32_t* sync = (int32_t*)((char*)workspace + per_layer * (size_t)n_layers);
+
+    // the first layer's Q | K | V of every node from the input rows; later layers' tables are filled on the fly
+    dg4i_proj_args p;
+    p.A = (const __nv_bfloat16*)H; p.lda = ldh; p.W = wq[0]; p.n_out = 384;
+    p.out[0] = q[0]; p.ldo[0] = 128; p.out[1] = kv[0]; p.ldo[1] = 256; p.out[2] = kv[0] + 128; p.ldo[2] = 256;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
+    CHECK(dg4i_proj_launch(p, st));
+    return dg4i_levelised_launch(g, desc, n_layers, q, kv, (__nv_bfloat16*)H, ldh, wq, wo, sync, status_word, st);
 }

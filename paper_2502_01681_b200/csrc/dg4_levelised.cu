@@ -1,26 +1,32 @@
-// Levelised layer as ONE persistent kernel (Sec. 1 / Sec. 3.4: gates are encoded level by level in
+// Levelised layers as ONE persistent kernel (Sec. 1 / Sec. 3.4: gates are encoded level by level in
 // topological order, each gate once, reading the rows already updated for lower levels).
 //
-// Q | K | V of every node have been projected from the layer's input beforehand (a node's own query, key and
-// value always come from its row as it was when the layer started).  This kernel then walks the levels.
-// For a tile of 16 nodes of the current level a CTA
-//   1. gathers the K | V rows of every neighbour (16 lanes per node, 16 bytes per lane), computes scores,
-//      softmax and the weighted value sum in registers, and writes the 16 x 128 attention tile into shared
-//      memory in the tensor core's K-major, 128-byte-swizzled operand layout;
-//   2. runs the output projection TRANSPOSED on the tensor cores: D1[feature, node] = W_o * O^T
-//      (tcgen05.mma, M = 128 features, N = 16 nodes, K = 128), so a small tile costs a fraction of a
-//      128-row tile and all warps take part in the epilogue (128 TMEM lanes x 16 columns);
-//   3. adds the residual, rounds to bf16, writes the new rows to H and -- in operand layout again -- to shared
-//      memory, and
-//   4. refreshes the tile's K | V rows the same way: D2 = W_k * H'^T and W_v * H'^T, rounded and stored.
-// W_o, W_k and W_v stay resident in shared memory for the whole kernel (one TMA load each).
+// Work of one tile (16 nodes of one level, for one layer k):
+//   1. gather the K | V rows of every neighbour from layer k's K|V table (16 lanes per node, 16 bytes per
+//      lane), compute scores, softmax and the weighted value sum in registers, and write the 16 x 128
+//      attention tile into shared memory in the tensor core's K-major, 128-byte-swizzled operand layout;
+//   2. output projection TRANSPOSED on the tensor cores: D[feature, node] = W_o * O^T (tcgen05.mma, M = 128
+//      features, N = 16 nodes, K = 128), so a small tile costs a fraction of a 128-row tile and all warps take
+//      part in the epilogue (128 TMEM lanes x 16 columns);
+//   3. add the residual, round to bf16, write the new rows to H and -- in operand layout again -- to shared
+//      memory;
+//   4. from the new rows, again transposed: refresh the tile's K | V rows of layer k (so that higher levels
+//      gather updated rows) and, if there is a layer k+1, project that layer's Q | K | V rows of these nodes
+//      (a node's own query, key and value always come from its row as the previous layer left it).
 //
-// Levels are separated by counters in global memory instead of kernel launches: each level has an arrival
-// counter that only the CTAs owning a tile of that level bump (release); before a level in which it has work a
-// CTA waits (acquire) until the previous non-empty level's counter is full.  Completion is transitive, because
-// every CTA that arrived on that level had itself waited for the level before it.  Launched cooperatively (all CTAs
-// co-resident).  Every wait is bounded; on expiry the kernel records DG4_ERR_TIMEOUT, raises an abort word that
-// every other wait polls, and all CTAs leave their loops, free tensor memory and return.
+// Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
+// (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
+// to layers round-robin; each keeps its layer's W_o, W_k, W_v and the next layer's W_q, W_k, W_v resident in
+// shared memory (one TMA load each).  With n layers the dependent chain is n_levels + n - 1 tile steps long
+// instead of n * n_levels, while computing exactly what n successive level-by-level sweeps compute.
+//
+// Levels are separated by counters in global memory instead of kernel launches: every (layer, level) has an
+// arrival counter that only the CTAs owning a tile of it bump (release); before a level in which it has work a
+// CTA waits (acquire) until the counter of its layer's previous non-empty level and the counter of the previous
+// layer's same level are full.  Completion is transitive, because every CTA that arrived had itself waited the
+// same way.  Launched cooperatively (all CTAs co-resident).  Every wait is bounded; on expiry the kernel records
+// DG4_ERR_TIMEOUT, raises an abort word that every other wait polls, and all CTAs leave their loops, free
+// tensor memory and return.
 
 #include "dg4_internal.h"
 #include "dg4_attn_core.cuh"
@@ -37,15 +43,17 @@ constexpr int kTile = 16;                    // nodes per tile
 constexpr int kThreads = kTile * 16;         // 16 lanes per node
 constexpr int kWBlock = 2 * 128 * 128;       // one 128 x 128 bf16 weight block: two K-halves of 16 KiB
 constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
-constexpr int kTmemCols = 64;
+constexpr int kTmemCols = 128;               // six accumulators of kTile columns
+constexpr int kStageRow = 1280;              // staging per node: K|V of this layer 512, Q of the next 256, its K|V 512
 
-constexpr int kOffW = 0;                          // W_o | W_k | W_v : 96 KiB
-constexpr int kOffO = 3 * kWBlock;                // attention tile (operand layout)
+constexpr int kOffW = 0;                          // W_o | W_k | W_v | next W_q | W_k | W_v : 192 KiB
+constexpr int kOffO = 6 * kWBlock;                // attention tile (operand layout)
 constexpr int kOffHp = kOffO + 2 * kBHalf;        // new rows (operand layout)
 constexpr int kOffHres = kOffHp + 2 * kBHalf;     // residual rows, plain [kTile][256 B]
-constexpr int kOffKV = kOffHres + kTile * 256;    // K|V staging, plain [kTile][512 B]
-constexpr int kOffMisc = kOffKV + kTile * 512;
-constexpr int kSmemBytes = kOffMisc + 512 + 1024;
+constexpr int kOffStage = kOffHres + kTile * 256; // output staging, plain [kTile][kStageRow]
+constexpr int kOffMisc = kOffStage + kTile * kStageRow;
+constexpr int kSmemBytes = kOffMisc + 256 + 1024;
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 struct Misc {
     uint64_t w_full, mma1, mma2;
@@ -54,20 +62,25 @@ struct Misc {
     int32_t node[kTile];
 };
 
+struct LayerMaps {
+    CUtensorMap wo[DG4I_MAX_LAYERS];
+    CUtensorMap wqkv[DG4I_MAX_LAYERS];
+};
+
 struct LevParams {
-    const __nv_bfloat16* Q;          // [n, 128]
-    __nv_bfloat16* KV;               // [n, 256]
-    __nv_bfloat16* H;                // [n, ldh]
+    __nv_bfloat16* Q[DG4I_MAX_LAYERS];     // [n, 128] per layer
+    __nv_bfloat16* KV[DG4I_MAX_LAYERS];    // [n, 256] per layer
+    __nv_bfloat16* H;                      // [n, ldh], updated in place by every layer in turn
     int64_t ldh;
-    const int32_t* nbr_ptr;
-    const int32_t* nbr_idx;
+    const int32_t* nbr_pad;                // [n, pad_width]
     const int32_t* level_ptr;
     const int32_t* level_nodes;
     int32_t n_levels;
+    int32_t n_layers;
     int32_t residual;
     float scale;
-    int32_t* arrive;                 // [n_levels], zero on entry
-    int32_t* abort_word;             // zero on entry
+    int32_t* arrive;                       // [n_layers, n_levels], zero on entry
+    int32_t* abort_word;                   // zero on entry
     int32_t* status;
 };
 
@@ -110,18 +123,44 @@ __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
     return (uint32_t)((k >> 6) * kBHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
 }
 
+__device__ __forceinline__ void give_up(const LevParams& p) {
+    atomicExch(p.abort_word, 1);
+    if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
+}
+
+// Polls until *counter >= target; false on abort or after ~1 s.
+__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word) {
+    uint32_t polls = 0;
+    while (ld_acquire(counter) < target) {
+        ++polls;
+        if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(abort_word) != 0)) return false;
+        if (polls > 64) __nanosleep(32);
+    }
+    return true;
+}
+
 template <int LPH, int MAXN>
 __global__ void __launch_bounds__(kThreads, 1)
-levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_constant__ CUtensorMap map_wqkv, LevParams p) {
+levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
     extern __shared__ uint8_t smem_raw[];
+    constexpr int W = MAXN + 1;                          // width of a neighbour-table entry
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
-    const uint32_t sW = base + kOffW, sO = base + kOffO, sHp = base + kOffHp, sHres = base + kOffHres, sKV = base + kOffKV;
+    const uint32_t sW = base + kOffW, sO = base + kOffO, sHp = base + kOffHp, sHres = base + kOffHres, sSt = base + kOffStage;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid >> 4, sub = tid & 15;          // node slot of the tile and lane within the node
     const int grp_base = lane - sub;
+    const unsigned gmask = 0xffffu << grp_base;
     const uint32_t bar_w = smem_u32(&misc->w_full), bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
+
+    // this CTA's layer, its rank among the CTAs of that layer, and how many CTAs each layer has
+    const int layer = (int)blockIdx.x % p.n_layers;
+    const int bid = (int)blockIdx.x / p.n_layers;
+    auto ctas_of = [&](int k) { return ((int)gridDim.x - k + p.n_layers - 1) / p.n_layers; };
+    const int nctas = ctas_of(layer);
+    const bool has_next = layer + 1 < p.n_layers;
+    const int n_acc = has_next ? 5 : 2;                  // accumulators of the second MMA group
 
     if (tid == 0) {
         mbar_init(bar_w, 1);
@@ -129,13 +168,16 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
         mbar_init(bar2, 1);
         misc->go = 1;
         mbar_fence_init();
-        tma_prefetch_desc(&map_wo);
-        tma_prefetch_desc(&map_wqkv);
-        mbar_expect_tx(bar_w, 3u * kWBlock);
+        tma_prefetch_desc(&maps.wo[layer]);
+        tma_prefetch_desc(&maps.wqkv[layer]);
+        mbar_expect_tx(bar_w, (uint32_t)((has_next ? 6 : 3) * kWBlock));
         for (int h = 0; h < 2; ++h) {
-            tma_load_2d(sW + h * (kWBlock / 2), &map_wo, h * 64, 0, bar_w);
-            tma_load_2d(sW + kWBlock + h * (kWBlock / 2), &map_wqkv, h * 64, 128, bar_w);
-            tma_load_2d(sW + 2 * kWBlock + h * (kWBlock / 2), &map_wqkv, h * 64, 256, bar_w);
+            tma_load_2d(sW + h * (kWBlock / 2), &maps.wo[layer], h * 64, 0, bar_w);
+            tma_load_2d(sW + kWBlock + h * (kWBlock / 2), &maps.wqkv[layer], h * 64, 128, bar_w);
+            tma_load_2d(sW + 2 * kWBlock + h * (kWBlock / 2), &maps.wqkv[layer], h * 64, 256, bar_w);
+            if (has_next)
+                for (int b = 0; b < 3; ++b)
+                    tma_load_2d(sW + (3 + b) * kWBlock + h * (kWBlock / 2), &maps.wqkv[layer + 1], h * 64, b * 128, bar_w);
         }
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
@@ -143,11 +185,7 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc->tmem_base;
-    bool weights_ok = mbar_wait(bar_w, 0);
-    if (!weights_ok && tid == 0) {
-        atomicExch(p.abort_word, 1);
-        if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
-    }
+    if (!mbar_wait(bar_w, 0) && tid == 0) give_up(p);
 
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
     static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
@@ -156,12 +194,17 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
     uint32_t ph1 = 0, ph2 = 0;
     int last_nonempty = -1, last_participants = 0;
     bool alive = true;
-    const int bid = blockIdx.x, nctas = gridDim.x;
 
-    // The index chain of a tile (node id -> list bounds -> neighbour ids) is three dependent loads that do not
-    // depend on any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
+    const char* kv_tab = (const char*)p.KV[layer];
+    const char* q_tab = (const char*)p.Q[layer];
+    int32_t* my_arrive = p.arrive + (size_t)layer * p.n_levels;
+    const int32_t* prev_arrive = layer > 0 ? p.arrive + (size_t)(layer - 1) * p.n_levels : nullptr;
+    const int prev_ctas = layer > 0 ? ctas_of(layer - 1) : 0;
+
+    // The index chain of a tile (node id -> neighbour-table entry) is two dependent loads that do not depend on
+    // any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
     // level-to-level critical path: while level l is processed, the node id of this CTA's first tile of level
-    // l+3, the list bounds for level l+2 and the neighbour ids for level l+1 are in flight.
+    // l+2 and the table entry for level l+1 are in flight.
     auto level_first = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv] : 0; };
     auto level_size = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv + 1] - p.level_ptr[lv] : 0; };
     auto stage_node = [&](int lv) -> int {            // node of (first tile of this CTA, this slot) at level lv
@@ -169,64 +212,40 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
         const int r = bid * kTile + slot;
         return (r < n_lv) ? p.level_nodes[level_first(lv) + r] : -1;
     };
-    // pipeline state at the top of iteration l:
-    int v0 = -1, cnt0 = 1, idx0 = -1;                  // level l  : node id, list length, this lane's neighbour id
-    int vC = -1, cntC = 1, begC = 0;                   // level l+1: node id and list bounds
-    int vB = -1;                                       // level l+2: node id
-    {   // prologue: levels 0, 1, 2
-        v0 = stage_node(0);
-        vC = stage_node(1);
-        vB = stage_node(2);
-        int beg0 = 0;
-        if (v0 >= 0) { beg0 = p.nbr_ptr[v0]; cnt0 = p.nbr_ptr[v0 + 1] - beg0; }
-        if (vC >= 0) { begC = p.nbr_ptr[vC]; cntC = p.nbr_ptr[vC + 1] - begC; }
-        idx0 = (v0 >= 0 && sub < cnt0) ? p.nbr_idx[beg0 + sub] : v0;
-    }
+    auto pad_of = [&](int v) -> int { return (v >= 0 && sub < W) ? p.nbr_pad[(size_t)v * W + sub] : 0; };
+    int v0 = stage_node(0);                            // level l  : node id and this lane's table word
+    int pad0 = pad_of(v0);
+    int vC = stage_node(1);                            // level l+1: node id
 
     for (int l = 0; l < p.n_levels && alive; ++l) {
         const int first = p.level_ptr[l];
         const int n_l = p.level_ptr[l + 1] - first;
         // issue the next load of every pipelined chain; the results are first used one level later
-        const int vA = stage_node(l + 3);                                               // level l+3: node id
-        int begB = 0, cntB = 1;                                                          // level l+2: list bounds
-        if (vB >= 0) { begB = p.nbr_ptr[vB]; cntB = p.nbr_ptr[vB + 1] - begB; }
-        const int idxC = (vC >= 0 && sub < cntC) ? p.nbr_idx[begC + sub] : vC;          // level l+1: neighbour id
+        const int vB = stage_node(l + 2);
+        const int padC = pad_of(vC);
         const int tiles = (n_l + kTile - 1) / kTile;
         if (n_l > 0 && bid < tiles) {
             bool waited = false;
             for (int tile = bid; tile < tiles; tile += nctas) {
-                int v, cnt, my_idx;
-                bool valid;
+                int v, pad;
                 if (tile == bid) {
-                    v = v0; cnt = cnt0; my_idx = idx0; valid = v0 >= 0;
+                    v = v0; pad = pad0;
                 } else {                         // further tiles of a wide level: plain dependent loads
                     const int r = tile * kTile + slot;
-                    valid = r < n_l;
-                    v = valid ? p.level_nodes[first + r] : -1;
-                    int beg = 0;
-                    cnt = 1;
-                    if (valid) { beg = p.nbr_ptr[v]; cnt = p.nbr_ptr[v + 1] - beg; }
-                    my_idx = (valid && sub < cnt) ? p.nbr_idx[beg + sub] : v;
+                    v = (r < n_l) ? p.level_nodes[first + r] : -1;
+                    pad = pad_of(v);
                 }
+                const bool valid = v >= 0;
 
                 if (!waited) {
-                    // ---- every tile of the previous non-empty level must have arrived (and nobody has given up)
+                    // ---- this layer's previous level and the previous layer's same level must be complete
                     if (tid == 0) {
-                        int go = 1;
-                        if (last_nonempty >= 0) {
-                            uint32_t polls = 0;
-                            while (ld_acquire(p.arrive + last_nonempty) < last_participants) {
-                                ++polls;
-                                if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(p.abort_word) != 0)) { go = 0; break; }
-                                if (polls > 64) __nanosleep(32);
-                            }
-                            if (!go && ld_acquire(p.abort_word) == 0) {
-                                atomicExch(p.abort_word, 1);
-                                if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
-                            }
-                        }
-                        if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = 0;
-                        misc->go = go;
+                        bool go = true;
+                        if (last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word);
+                        if (go && prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word);
+                        if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                        if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
+                        misc->go = go ? 1 : 0;
                     }
                     __syncthreads();
                     waited = true;
@@ -236,26 +255,27 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                 // ---- gather and attend
                 Piece kq[MAXN], vq[MAXN], qp, hres;
                 int u[MAXN];
+                const int cnt = valid ? __shfl_sync(gmask, pad, grp_base) : 1;
+                u[0] = v;
 #pragma unroll
-                for (int j = 0; j < MAXN; ++j) u[j] = __shfl_sync(0xffffffffu, my_idx, grp_base + j);
+                for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(gmask, pad, grp_base + j);
                 float acc[8];
                 if (valid) {
-                    const char* kv = (const char*)p.KV;
 #pragma unroll
                     for (int j = 0; j < MAXN; ++j)
-                        if (j < cnt) vq[j] = ld_piece_cg(kv + (size_t)u[j] * 512 + 256 + sub * 16);
+                        if (j < cnt) vq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + 256 + sub * 16);
                     if (cnt > 1) {
-                        qp = ld_piece_nc((const char*)p.Q + (size_t)v * 256 + sub * 16);
+                        qp = ld_piece_cg(q_tab + (size_t)v * 256 + sub * 16);
 #pragma unroll
                         for (int j = 0; j < MAXN; ++j)
-                            if (j < cnt) kq[j] = ld_piece_cg(kv + (size_t)u[j] * 512 + sub * 16);
+                            if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
                     }
                     if (p.residual) hres = ld_piece_cg((const char*)p.H + (size_t)v * p.ldh * 2 + sub * 16);
                 } else {
                     vq[0].w[0] = vq[0].w[1] = vq[0].w[2] = vq[0].w[3] = 0u;
                 }
                 if (!valid || !p.residual) hres.w[0] = hres.w[1] = hres.w[2] = hres.w[3] = 0u;
-                attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, 0xffffu << grp_base, acc);
+                attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, gmask, acc);
                 {
                     Piece o = Elem<true>::pack(acc);
                     st_shared_v4(sO + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), o.w);
@@ -265,7 +285,7 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                 fence_proxy_async_smem();
                 __syncthreads();
 
-                // ---- output projection, transposed: D1[feature, node] = W_o * O^T
+                // ---- output projection, transposed: D[feature, node] = W_o * O^T
                 if (tid == 0) {
                     tc_fence_after();
 #pragma unroll
@@ -276,10 +296,7 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                     }
                     mma_commit(bar1);
                 }
-                if (!mbar_wait(bar1, ph1) && tid == 0) {
-                    atomicExch(p.abort_word, 1);
-                    if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
-                }
+                if (!mbar_wait(bar1, ph1) && tid == 0) give_up(p);
                 ph1 ^= 1u;
                 tc_fence_after();
                 {
@@ -298,73 +315,73 @@ levelised_kernel(const __grid_constant__ CUtensorMap map_wo, const __grid_consta
                 fence_proxy_async_smem();
                 __syncthreads();
 
-                // ---- K | V refresh, transposed: D2 = W_k * H'^T and W_v * H'^T
+                // ---- from the new rows, transposed: this layer's K | V refresh and the next layer's Q | K | V
                 if (tid == 0) {
                     tc_fence_after();
-#pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
+                    for (int blk = 0; blk < n_acc; ++blk) {
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
                             const uint32_t a_off = (uint32_t)((1 + blk) * kWBlock + (ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
                             const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                            mma_bf16(tmem + (uint32_t)(kTile + kTile * blk), smem_desc_sw128(sW + a_off),
+                            mma_bf16(tmem + (uint32_t)(kTile * (1 + blk)), smem_desc_sw128(sW + a_off),
                                      smem_desc_sw128(sHp + b_off), idesc, ks > 0 ? 1u : 0u);
                         }
                     }
                     mma_commit(bar2);
                 }
                 // meanwhile: the new rows go to H (16 lanes cover one 256-byte row)
+                const int node_v = misc->node[slot];
                 {
-                    const int node_v = misc->node[slot];
                     uint32_t w4[4];
                     ld_shared_v4(sHp + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), w4);
                     if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
                 }
-                if (!mbar_wait(bar2, ph2) && tid == 0) {
-                    atomicExch(p.abort_word, 1);
-                    if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
-                }
+                if (!mbar_wait(bar2, ph2) && tid == 0) give_up(p);
                 ph2 ^= 1u;
                 tc_fence_after();
-                {
-                    uint32_t dk[8], dv[8];
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile + cg * 8), dk);
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(2 * kTile + cg * 8), dv);
+                // accumulator blk (0: K, 1: V, 2: next Q, 3: next K, 4: next V) -> byte offset inside a staging row
+                for (int blk = 0; blk < n_acc; ++blk) {
+                    uint32_t d[8];
+                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile * (1 + blk) + cg * 8), d);
                     tmem_ld_wait();
+                    const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
 #pragma unroll
-                    for (int nn = 0; nn < 8; ++nn) {
-                        const int node = cg * 8 + nn;
-                        st_shared_b16(sKV + (uint32_t)(node * 512 + feat * 2), bf16_bits(__uint_as_float(dk[nn])));
-                        st_shared_b16(sKV + (uint32_t)(node * 512 + 256 + feat * 2), bf16_bits(__uint_as_float(dv[nn])));
-                    }
+                    for (int nn = 0; nn < 8; ++nn)
+                        st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[nn])));
                 }
                 tc_fence_before();
                 __syncthreads();
-                {
-                    const int node_v = misc->node[slot];
-                    if (node_v >= 0) {
+                if (node_v >= 0) {
+                    const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {        // this layer's K | V row
+                        ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
+                        st_global_v4((char*)p.KV[layer] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
+                    }
+                    if (has_next) {                      // the next layer's Q row and (not yet updated) K | V row
+                        ld_shared_v4(row + (uint32_t)(512 + sub * 16), w4);
+                        st_global_v4((char*)p.Q[layer + 1] + (size_t)node_v * 256 + sub * 16, w4);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            uint32_t w4[4];
-                            ld_shared_v4(sKV + (uint32_t)(slot * 512 + (sub + 16 * h) * 16), w4);
-                            st_global_v4((char*)p.KV + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
+                            ld_shared_v4(row + (uint32_t)(768 + (sub + 16 * h) * 16), w4);
+                            st_global_v4((char*)p.KV[layer + 1] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
                         }
                     }
                 }
                 __syncthreads();    // the tile's shared buffers may be overwritten from here on
             }
             if (!alive) break;
-            // ---- this CTA's part of level l is in global memory: arrive on the level's counter (release)
-            if (tid == 0) red_release_add(p.arrive + l, 1);
+            // ---- this CTA's part of (layer, level l) is in global memory: arrive on its counter (release)
+            if (tid == 0) red_release_add(my_arrive + l, 1);
         }
         if (n_l > 0) {
             last_nonempty = l;
             last_participants = tiles < nctas ? tiles : nctas;
         }
         // rotate the pipeline by one level
-        v0 = vC; cnt0 = cntC; idx0 = idxC;
-        vC = vB; cntC = cntB; begC = begB;
-        vB = vA;
+        v0 = vC; pad0 = padC;
+        vC = vB;
     }
 
     tc_fence_before();
@@ -412,38 +429,42 @@ dg4_status make_weight_map(CUtensorMap* m, const void* base, int64_t rows) {
 }
 
 template <int LPH, int MAXN>
-dg4_status launch(const CUtensorMap& map_wo, const CUtensorMap& map_wqkv, const LevParams& p, int grid, cudaStream_t st) {
+dg4_status launch(const LayerMaps& maps, const LevParams& p, int grid, cudaStream_t st) {
     auto kern = levelised_kernel<LPH, MAXN>;
     DG4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     int per_sm = 0;
     DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
     if (per_sm < 1) DG4_FAIL(DG4_ERR_CUDA, "the levelised kernel does not fit on this device");
-    void* args[] = {(void*)&map_wo, (void*)&map_wqkv, (void*)&p};
+    void* args[] = {(void*)&maps, (void*)&p};
     DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, kSmemBytes, st));
     dg4i_count_launch();
     return DG4_OK;
 }
 
 template <int MAXN>
-dg4_status launch_heads(int heads, const CUtensorMap& a, const CUtensorMap& b, const LevParams& p, int grid, cudaStream_t st) {
+dg4_status launch_heads(int heads, const LayerMaps& maps, const LevParams& p, int grid, cudaStream_t st) {
     switch (16 / heads) {
-        case 1: return launch<1, MAXN>(a, b, p, grid, st);
-        case 2: return launch<2, MAXN>(a, b, p, grid, st);
-        case 4: return launch<4, MAXN>(a, b, p, grid, st);
-        case 8: return launch<8, MAXN>(a, b, p, grid, st);
-        case 16: return launch<16, MAXN>(a, b, p, grid, st);
+        case 1: return launch<1, MAXN>(maps, p, grid, st);
+        case 2: return launch<2, MAXN>(maps, p, grid, st);
+        case 4: return launch<4, MAXN>(maps, p, grid, st);
+        case 8: return launch<8, MAXN>(maps, p, grid, st);
+        case 16: return launch<16, MAXN>(maps, p, grid, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported", heads);
 }
 
 }  // namespace
 
-size_t dg4i_levelised_sync_bytes(const dg4_graph* g) { return ((size_t)g->n_levels + 64) * sizeof(int32_t); }
+size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers) {
+    return ((size_t)g->n_levels * (size_t)n_layers + 64) * sizeof(int32_t);
+}
 
-// Q, KV: projected from the layer's input for all nodes.  sync: dg4i_levelised_sync_bytes() bytes, 16-byte aligned.
-dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, const __nv_bfloat16* Q, __nv_bfloat16* KV,
-                                 __nv_bfloat16* H, int64_t ldh, const __nv_bfloat16* W_qkv, const __nv_bfloat16* W_o,
-                                 int32_t* sync, int32_t* status, cudaStream_t st) {
+dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers, __nv_bfloat16* const* Q,
+                                 __nv_bfloat16* const* KV, __nv_bfloat16* H, int64_t ldh,
+                                 const __nv_bfloat16* const* W_qkv, const __nv_bfloat16* const* W_o, int32_t* sync,
+                                 int32_t* status, cudaStream_t st) {
+    if (n_layers < 1 || n_layers > DG4I_MAX_LAYERS)
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "n_layers = %d: between 1 and %d layers per call", n_layers, DG4I_MAX_LAYERS);
     int dev = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
@@ -456,17 +477,24 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, const
         }
     }
     if (!g_coop[dev]) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device %d cannot launch cooperative kernels", dev);
-    CUtensorMap map_wo, map_wqkv;
-    dg4_status s;
-    if ((s = make_weight_map(&map_wo, W_o, 128)) != DG4_OK) return s;
-    if ((s = make_weight_map(&map_wqkv, W_qkv, 384)) != DG4_OK) return s;
-    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g), st));
+    if (g_sm_count[dev] < n_layers) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer SMs than layers");
+    LayerMaps maps;
     LevParams p;
-    p.Q = Q; p.KV = KV; p.H = H; p.ldh = ldh;
-    p.nbr_ptr = g->nbr_ptr; p.nbr_idx = g->nbr_idx; p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
-    p.n_levels = g->n_levels; p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
+    dg4_status s;
+    for (int k = 0; k < DG4I_MAX_LAYERS; ++k) {
+        const int kk = k < n_layers ? k : 0;           // unused slots repeat layer 0 (never read)
+        if ((s = make_weight_map(&maps.wo[k], W_o[kk], 128)) != DG4_OK) return s;
+        if ((s = make_weight_map(&maps.wqkv[k], W_qkv[kk], 384)) != DG4_OK) return s;
+        p.Q[k] = Q[kk];
+        p.KV[k] = KV[kk];
+    }
+    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, n_layers), st));
+    p.H = H; p.ldh = ldh;
+    p.nbr_pad = g->nbr_pad; p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
+    p.n_levels = g->n_levels; p.n_layers = n_layers;
+    p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status;
     const int grid = g_sm_count[dev];
-    if (g->max_class <= 3) return launch_heads<3>(desc->heads, map_wo, map_wqkv, p, grid, st);
-    return launch_heads<7>(desc->heads, map_wo, map_wqkv, p, grid, st);
+    if (g->max_class <= 3) return launch_heads<3>(desc->heads, maps, p, grid, st);
+    return launch_heads<7>(desc->heads, maps, p, grid, st);
 }

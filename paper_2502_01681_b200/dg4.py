@@ -38,7 +38,7 @@ EXPORTS = [
     "dg4_status_string", "dg4_last_error", "dg4_launch_count", "dg4_graph_create", "dg4_graph_rebuild", "dg4_graph_destroy",
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_poll_status", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
-    "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes",
+    "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
 ]
 
 
@@ -113,6 +113,11 @@ def load():
     lib.dg4_layer_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
     lib.dg4_layer_fwd_levelised.restype = ctypes.c_int
     lib.dg4_layer_fwd_levelised.argtypes = [vp, dp, vp, i64, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.dg4_layers_workspace_bytes.restype = ctypes.c_size_t
+    lib.dg4_layers_workspace_bytes.argtypes = [vp, dp, ctypes.c_int32]
+    lib.dg4_layers_fwd_levelised.restype = ctypes.c_int
+    lib.dg4_layers_fwd_levelised.argtypes = [vp, dp, vp, i64, ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp,
+                                             ctypes.c_size_t, vp, vp]
     lib.dg4_layer_fwd_parallel_static.restype = ctypes.c_int
     lib.dg4_layer_fwd_parallel_static.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp]
     lib.dg4_static_max_nodes.restype = ctypes.c_int64
@@ -265,3 +270,20 @@ def dg4_layer_fwd_parallel_static(g: Graph, dsc: dg4_desc, H_in, W_qkv, W_o, H_o
     not overlap on the GPU."""
     _check(load().dg4_layer_fwd_parallel_static(g.handle, ctypes.byref(dsc), _ptr(H_in), _ld(H_in), _ptr(W_qkv),
                                                 _ptr(W_o), _ptr(H_out), _ld(H_out), _stream(stream)))
+
+
+def dg4_layers_workspace_bytes(g: Graph, dsc: dg4_desc, n_layers: int) -> int:
+    return int(load().dg4_layers_workspace_bytes(g.handle, ctypes.byref(dsc), n_layers))
+
+
+def dg4_layers_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, workspace, device_status=None,
+                             stream=None):
+    """Several levelised layers in one call (same result as one dg4_layer_fwd_levelised call per layer)."""
+    n = len(W_qkv_list)
+    assert n == len(W_o_list)
+    arr = ctypes.c_void_p * n
+    wq = arr(*[t.data_ptr() for t in W_qkv_list])
+    wo = arr(*[t.data_ptr() for t in W_o_list])
+    _check(load().dg4_layers_fwd_levelised(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), n, wq, wo, _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), _ptr(device_status),
+                                           _stream(stream)))

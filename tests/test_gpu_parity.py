@@ -239,9 +239,16 @@ def _weights(w, layers):
 
 def _run_layers_gpu(gr, w, xb, weights, mode):
     dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, level_launches=(mode == "level-launches"))
-    ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, len(weights))),
+                     dtype=torch.uint8, device="cuda")
     h = dev_bf16(xb).clone()
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if mode == "wavefront":              # all layers in one call
+        dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dev_bf16(w_[0]) for w_ in weights], [dev_bf16(w_[2]) for w_ in weights],
+                                     ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        return host_f64_of_bf16(h)
     for (wq_bits, _, wo_bits, _) in weights:
         if mode == "parallel":
             dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), h, ws)
@@ -269,7 +276,9 @@ def _run_layers_checker(g, w, xb, weights, mode):
 @pytest.mark.parametrize("cfg,shrink,mode", [(2, 1, "parallel"), (2, 7, "parallel"), (5, 200, "parallel"),
                                              (4, 20, "levelised"), (5, 400, "levelised"), (2, 10, "levelised"),
                                              (4, 5, "levelised"), (5, 50, "levelised"),
-                                             (4, 20, "level-launches"), (5, 400, "level-launches")])
+                                             (4, 20, "level-launches"), (5, 400, "level-launches"),
+                                             (4, 20, "wavefront"), (5, 400, "wavefront"), (5, 50, "wavefront"),
+                                             (2, 10, "wavefront"), (4, 5, "wavefront")])
 def test_layers_match_checker(cfg, shrink, mode):
     w = synth.workload(cfg, shrink)
     g = w.graph()
@@ -294,6 +303,10 @@ def test_levelised_differs_from_parallel_and_is_repeatable():
     p = _run_layers_gpu(gr, w, xb, weights, "parallel")
     assert (a == b).all()                                   # a race between levels would show up as a diff
     assert rel_row_err(a, c).max() <= 1e-2                  # persistent kernel vs one launch group per level
+    w3 = _weights(w, 3)
+    d = _run_layers_gpu(gr, w, xb, w3, "levelised")         # three calls, layer after layer
+    e = _run_layers_gpu(gr, w, xb, w3, "wavefront")         # one call, layers as a wavefront
+    assert (d == e).all()
     lvl0 = g.level == 0
     assert (a[lvl0] == p[lvl0]).all()                       # level-0 rows never see an updated row
     assert np.abs(a - p).max() > 0
