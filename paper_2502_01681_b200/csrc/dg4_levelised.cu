@@ -106,6 +106,12 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ int ld_relaxed(const int32_t* p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_acquire() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -128,15 +134,20 @@ __device__ __forceinline__ void give_up(const LevParams& p) {
     if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
 }
 
-// Polls until *counter >= target; false on abort or after ~1 s.
-__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word) {
+// Polls until *c1 >= t1 and (if c2 is given) *c2 >= t2; false on abort or after ~1 s.  The two counters are read
+// with relaxed loads so that both are in flight in the same round trip; one fence then orders everything the
+// arriving CTAs released before this CTA's later reads.
+__device__ __forceinline__ bool wait_counters(const int32_t* c1, int t1, const int32_t* c2, int t2,
+                                              const int32_t* abort_word) {
     uint32_t polls = 0;
-    while (ld_acquire(counter) < target) {
+    for (;;) {
+        const int a = c1 ? ld_relaxed(c1) : t1;
+        const int b = c2 ? ld_relaxed(c2) : t2;
+        if (a >= t1 && b >= t2) { fence_acquire(); return true; }
         ++polls;
         if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(abort_word) != 0)) return false;
         if (polls > 64) __nanosleep(32);
     }
-    return true;
 }
 
 template <int LPH, int MAXN>
@@ -240,9 +251,9 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                 if (!waited) {
                     // ---- this layer's previous level and the previous layer's same level must be complete
                     if (tid == 0) {
-                        bool go = true;
-                        if (last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word);
-                        if (go && prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word);
+                        bool go = wait_counters(last_nonempty >= 0 ? my_arrive + last_nonempty : nullptr, last_participants,
+                                                prev_arrive ? prev_arrive + l : nullptr, tiles < prev_ctas ? tiles : prev_ctas,
+                                                p.abort_word);
                         if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                         if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
                         misc->go = go ? 1 : 0;
