@@ -58,7 +58,7 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 struct Misc {
     uint64_t w_full, mma1, mma2;
     uint32_t tmem_base;
-    int32_t go;
+    int32_t go, go2;
     int32_t node[kTile];
 };
 
@@ -106,12 +106,6 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ int ld_relaxed(const int32_t* p) {
-    int v;
-    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void fence_acquire() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -134,20 +128,15 @@ __device__ __forceinline__ void give_up(const LevParams& p) {
     if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
 }
 
-// Polls until *c1 >= t1 and (if c2 is given) *c2 >= t2; false on abort or after ~1 s.  The two counters are read
-// with relaxed loads so that both are in flight in the same round trip; one fence then orders everything the
-// arriving CTAs released before this CTA's later reads.
-__device__ __forceinline__ bool wait_counters(const int32_t* c1, int t1, const int32_t* c2, int t2,
-                                              const int32_t* abort_word) {
+// Polls (acquire) until *counter >= target; false on abort or after ~1 s.
+__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word) {
     uint32_t polls = 0;
-    for (;;) {
-        const int a = c1 ? ld_relaxed(c1) : t1;
-        const int b = c2 ? ld_relaxed(c2) : t2;
-        if (a >= t1 && b >= t2) { fence_acquire(); return true; }
+    while (ld_acquire(counter) < target) {
         ++polls;
         if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(abort_word) != 0)) return false;
         if (polls > 64) __nanosleep(32);
     }
+    return true;
 }
 
 template <int LPH, int MAXN>
@@ -178,6 +167,7 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
         mbar_init(bar1, 1);
         mbar_init(bar2, 1);
         misc->go = 1;
+        misc->go2 = 1;
         mbar_fence_init();
         tma_prefetch_desc(&maps.wo[layer]);
         tma_prefetch_desc(&maps.wqkv[layer]);
@@ -199,6 +189,8 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
     if (!mbar_wait(bar_w, 0) && tid == 0) give_up(p);
 
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
+    // matrix descriptors of the resident operands; stepping along K or to another block only adds to the address field
+    const uint64_t dW = smem_desc_sw128(sW), dO = smem_desc_sw128(sO), dHp = smem_desc_sw128(sHp);
     static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
     const int q4 = warp & 3, cg = warp >> 2;             // epilogue: TMEM lane quadrant and group of 8 node columns
     const int feat = q4 * 32 + lane;                     // output feature this thread holds in the epilogues
@@ -250,17 +242,22 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
 
                 if (!waited) {
                     // ---- this layer's previous level and the previous layer's same level must be complete
+                    // (two pollers in different warps, so that both counters are watched at the same time)
                     if (tid == 0) {
-                        bool go = wait_counters(last_nonempty >= 0 ? my_arrive + last_nonempty : nullptr, last_participants,
-                                                prev_arrive ? prev_arrive + l : nullptr, tiles < prev_ctas ? tiles : prev_ctas,
-                                                p.abort_word);
+                        bool go = true;
+                        if (last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word);
                         if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                         if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
                         misc->go = go ? 1 : 0;
+                    } else if (tid == 32) {
+                        bool go = true;
+                        if (prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word);
+                        if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                        misc->go2 = go ? 1 : 0;
                     }
                     __syncthreads();
                     waited = true;
-                    if (!misc->go) { alive = false; break; }
+                    if (!misc->go || !misc->go2) { alive = false; break; }
                 }
 
                 // ---- gather and attend
@@ -303,7 +300,7 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t a_off = (uint32_t)((ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
                         const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                        mma_bf16(tmem, smem_desc_sw128(sW + a_off), smem_desc_sw128(sO + b_off), idesc, ks > 0 ? 1u : 0u);
+                        mma_bf16(tmem, dW + (a_off >> 4), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
                     }
                     mma_commit(bar1);
                 }
@@ -329,13 +326,16 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                 // ---- from the new rows, transposed: this layer's K | V refresh and the next layer's Q | K | V
                 if (tid == 0) {
                     tc_fence_after();
-                    for (int blk = 0; blk < n_acc; ++blk) {
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {
-                            const uint32_t a_off = (uint32_t)((1 + blk) * kWBlock + (ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
-                            const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                            mma_bf16(tmem + (uint32_t)(kTile * (1 + blk)), smem_desc_sw128(sW + a_off),
-                                     smem_desc_sw128(sHp + b_off), idesc, ks > 0 ? 1u : 0u);
+                    for (int blk = 0; blk < 5; ++blk) {
+                        if (blk < n_acc) {
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks) {
+                                const uint32_t a_off = (uint32_t)((1 + blk) * kWBlock + (ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
+                                const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
+                                mma_bf16(tmem + (uint32_t)(kTile * (1 + blk)), dW + (a_off >> 4), dHp + (b_off >> 4), idesc,
+                                         ks > 0 ? 1u : 0u);
+                            }
                         }
                     }
                     mma_commit(bar2);
@@ -351,14 +351,22 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                 ph2 ^= 1u;
                 tc_fence_after();
                 // accumulator blk (0: K, 1: V, 2: next Q, 3: next K, 4: next V) -> byte offset inside a staging row
-                for (int blk = 0; blk < n_acc; ++blk) {
-                    uint32_t d[8];
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile * (1 + blk) + cg * 8), d);
-                    tmem_ld_wait();
-                    const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
+                {
+                    uint32_t d[5][8];
 #pragma unroll
-                    for (int nn = 0; nn < 8; ++nn)
-                        st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[nn])));
+                    for (int blk = 0; blk < 5; ++blk)
+                        if (blk < n_acc)
+                            tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile * (1 + blk) + cg * 8), d[blk]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int blk = 0; blk < 5; ++blk) {
+                        if (blk < n_acc) {
+                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
+#pragma unroll
+                            for (int nn = 0; nn < 8; ++nn)
+                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
+                        }
+                    }
                 }
                 tc_fence_before();
                 __syncthreads();
