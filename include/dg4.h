@@ -244,6 +244,14 @@ dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, vo
                                     int32_t n_layers, const void* const* W_qkv, const void* const* W_o,
                                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
 
+/*
+ * Diagnostic (the paper has no counterpart): launches one small CTA that waits, with the same bounded wait the
+ * pipelines of this library use, on a barrier nothing ever arrives on.  The wait gives up after its poll limit
+ * (about a second) and the kernel writes DG4_ERR_TIMEOUT to *device_status (device int32) and returns normally:
+ * nothing traps, the context stays usable.  Asynchronous on `stream`.
+ */
+dg4_status dg4_selftest_bounded_wait(int32_t* device_status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -39,6 +39,7 @@ EXPORTS = [
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_poll_status", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
+    "dg4_selftest_bounded_wait",
 ]
 
 
@@ -118,6 +119,8 @@ def load():
     lib.dg4_layers_fwd_levelised.restype = ctypes.c_int
     lib.dg4_layers_fwd_levelised.argtypes = [vp, dp, vp, i64, ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp,
                                              ctypes.c_size_t, vp, vp]
+    lib.dg4_selftest_bounded_wait.restype = ctypes.c_int
+    lib.dg4_selftest_bounded_wait.argtypes = [vp, vp]
     lib.dg4_layer_fwd_parallel_static.restype = ctypes.c_int
     lib.dg4_layer_fwd_parallel_static.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp]
     lib.dg4_static_max_nodes.restype = ctypes.c_int64
@@ -287,3 +290,7 @@ def dg4_layers_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, w
     _check(load().dg4_layers_fwd_levelised(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), n, wq, wo, _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), _ptr(device_status),
                                            _stream(stream)))
+
+
+def dg4_selftest_bounded_wait(device_status, stream=None):
+    _check(load().dg4_selftest_bounded_wait(_ptr(device_status), _stream(stream)))

@@ -342,3 +342,12 @@ def test_forward_calls_reject_bad_arguments():
         dg4.dg4_layer_fwd_parallel(g, dg4.desc(8, dg4.DG4_BF16, 1.0), t, t, t, o, small)
     assert e.value.status == dg4.DG4_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    # a wait nothing can satisfy ends by itself; the kernel reports it and the context stays usable
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dg4.dg4_selftest_bounded_wait(status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == dg4.DG4_ERR_TIMEOUT
+    assert float((torch.ones(8, device="cuda") * 2).sum().item()) == 16.0
