@@ -335,11 +335,14 @@ def run_ours(args, w):
     e2e_steps = max(1, min(2, args.steps))
     h2d = x_host.numel() * 2 + (g.row_ptr.nbytes + g.col_idx.nbytes + g.level.nbytes)
     d2h = out_host.numel() * 2
+    side = torch.cuda.Stream()
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
+        with torch.cuda.stream(side):                 # the feature upload runs while the host validates the circuit
+            x2 = x_host.cuda(non_blocking=True).view(torch.bfloat16)
         gr2 = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local)
-        x2 = x_host.cuda(non_blocking=True).view(torch.bfloat16)
+        stream.wait_stream(side)
         hp = x2.clone()
         for l in range(w.layers):
             dg4.dg4_layer_fwd_parallel(gr2, dsc, hp, wq[l], wo[l], hp, ws)

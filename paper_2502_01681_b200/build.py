@@ -31,7 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc"),
+           "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-pthread", "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc"),
            "-o", LIB] + SOURCES
     if verbose:
         cmd.insert(1, "-Xptxas=-v")

@@ -10,6 +10,8 @@
 #include "dg4_internal.h"
 
 #include <new>
+#include <thread>
+#include <vector>
 #include <stdlib.h>
 #include <string.h>
 
@@ -366,24 +368,52 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     if (perm_chunk < 0 || (perm_chunk % kTile) != 0)
         DG4_FAIL(DG4_ERR_INVALID_ARG, "perm_chunk must be 0 or a positive multiple of %d (got %d)", kTile, perm_chunk);
 
-    // ---- a1: validation on the host -----------------------------------------------------------
+    // ---- a1: validation on the host (node ranges checked by a few threads; the error of the lowest node wins)
     if (row_ptr[0] != 0) DG4_FAIL(DG4_ERR_NOT_SORTED, "row_ptr[0] must be 0");
-    int32_t max_level = 0;
-    for (int32_t v = 0; v < n_nodes; ++v) {
-        int32_t b = row_ptr[v], e = row_ptr[v + 1];
-        if (e < b) DG4_FAIL(DG4_ERR_NOT_SORTED, "row_ptr decreases at node %d", v);
-        if (e - b > 2) DG4_FAIL(DG4_ERR_BAD_DEGREE, "node %d has %d fan-ins (an AIG node has at most 2)", v, e - b);
-        if (level[v] < 0) DG4_FAIL(DG4_ERR_BAD_LEVEL, "node %d has negative level %d", v, level[v]);
-        if (e > b && !col_idx) DG4_FAIL(DG4_ERR_INVALID_ARG, "col_idx is null but the graph has edges");
-        for (int32_t i = b; i < e; ++i) {
-            int32_t u = col_idx[i];
-            if (u < 0 || u >= n_nodes) DG4_FAIL(DG4_ERR_BAD_LEVEL, "edge %d: source id %d out of range", i, u);
-            if (level[u] >= level[v])
-                DG4_FAIL(DG4_ERR_BAD_LEVEL, "edge %d -> %d: level %d is not below level %d", u, v, level[u], level[v]);
-        }
-        if (level[v] > max_level) max_level = level[v];
-    }
     const int64_t n_edges = row_ptr[n_nodes];
+    if (n_edges < 0) DG4_FAIL(DG4_ERR_NOT_SORTED, "row_ptr[n_nodes] is negative");
+    if (n_edges > 0 && !col_idx) DG4_FAIL(DG4_ERR_INVALID_ARG, "col_idx is null but the graph has edges");
+    struct Finding { dg4_status code = DG4_OK; int32_t node = 0; char msg[160] = ""; int32_t max_level = 0; };
+    auto check_range = [&](int32_t v0, int32_t v1, Finding* f) {
+        auto fail = [&](dg4_status c, int32_t v, const char* fmt, int a0, int a1, int a2, int a3) {
+            f->code = c; f->node = v;
+            snprintf(f->msg, sizeof(f->msg), fmt, a0, a1, a2, a3);
+        };
+        for (int32_t v = v0; v < v1; ++v) {
+            const int32_t b = row_ptr[v], e = row_ptr[v + 1];
+            if (e < b || b < 0 || e > n_edges) return fail(DG4_ERR_NOT_SORTED, v, "row_ptr is not non-decreasing within [0, %d] at node %d", (int)n_edges, v, 0, 0);
+            if (e - b > 2) return fail(DG4_ERR_BAD_DEGREE, v, "node %d has %d fan-ins (an AIG node has at most 2)", v, e - b, 0, 0);
+            if (level[v] < 0) return fail(DG4_ERR_BAD_LEVEL, v, "node %d has negative level %d", v, level[v], 0, 0);
+            for (int32_t i = b; i < e; ++i) {
+                const int32_t u = col_idx[i];
+                if (u < 0 || u >= n_nodes) return fail(DG4_ERR_BAD_LEVEL, v, "edge %d: source id %d out of range", i, u, 0, 0);
+                if (level[u] >= level[v])
+                    return fail(DG4_ERR_BAD_LEVEL, v, "edge %d -> %d: level %d is not below level %d", u, v, level[u], level[v]);
+            }
+            if (level[v] > f->max_level) f->max_level = level[v];
+        }
+    };
+    int n_thr = (int)std::thread::hardware_concurrency();
+    if (n_thr > 16) n_thr = 16;
+    if (n_thr < 1 || n_nodes < (1 << 18)) n_thr = 1;
+    std::vector<Finding> found((size_t)n_thr);
+    if (n_thr == 1) {
+        check_range(0, n_nodes, &found[0]);
+    } else {
+        std::vector<std::thread> pool;
+        const int64_t per = ((int64_t)n_nodes + n_thr - 1) / n_thr;
+        for (int t = 0; t < n_thr; ++t) {
+            const int64_t v0 = per * t, v1 = (v0 + per < n_nodes) ? v0 + per : n_nodes;
+            if (v0 >= v1) continue;
+            pool.emplace_back(check_range, (int32_t)v0, (int32_t)v1, &found[(size_t)t]);
+        }
+        for (auto& th : pool) th.join();
+    }
+    int32_t max_level = 0;
+    for (const Finding& f : found) {              // ranges are in node order: the first finding is the lowest node
+        if (f.code != DG4_OK) DG4_FAIL(f.code, "%s", f.msg);
+        if (f.max_level > max_level) max_level = f.max_level;
+    }
     if (max_level >= n_nodes) DG4_FAIL(DG4_ERR_BAD_LEVEL, "max level %d is not below the node count", max_level);
 
     int ndev = 0;

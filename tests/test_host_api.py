@@ -62,3 +62,16 @@ def test_null_handles_are_rejected_not_dereferenced():
     import ctypes
     assert lib.dg4_sparse_attn_fwd(None, ctypes.byref(d), None, 128, None, 128, None, 128, None, 128, None) \
         == dg4.DG4_ERR_INVALID_ARG
+
+
+def test_large_circuits_are_validated_in_parallel_and_the_lowest_bad_node_is_reported():
+    n = 300_000                                    # above the size at which validation uses several threads
+    row_ptr = np.arange(n + 1, dtype=np.int32) - 1
+    row_ptr[0] = 0                                 # node 0 is a primary input, node v > 0 has fan-in v - 1
+    col_idx = np.arange(n - 1, dtype=np.int32)
+    level = np.arange(n, dtype=np.int32)
+    level[200_000] = 5                             # level does not increase along edge 199999 -> 200000
+    level[250_000] = -3                            # a later fault that must not be the one reported
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_graph_create(row_ptr, col_idx, level, 2, 0)
+    assert e.value.status == dg4.DG4_ERR_BAD_LEVEL and "200000" in e.value.detail
