@@ -169,17 +169,34 @@ dg4_status exclusive_scan(const int32_t* in, int32_t* out, int64_t n, int32_t* b
 // ------------------------------------------------------------------------------------------------
 __global__ void level_hist_kernel(int n, const int32_t* __restrict__ level, int32_t* __restrict__ hist) {
     int v = blockIdx.x * blockDim.x + threadIdx.x;
-    if (v < n) atomicAdd(&hist[level[v]], 1);
+    int key = (v < n) ? level[v] : -1;
+    // lanes of a warp that hold the same level add once, through their lowest lane
+    unsigned peers = __match_any_sync(0xffffffffu, key);
+    if (key >= 0 && (peers & ((1u << (threadIdx.x & 31)) - 1u)) == 0) atomicAdd(&hist[key], __popc(peers));
 }
 
-// segment of v: v / chunk (by_level == 0) or level[v]
-__global__ void class_hist_kernel(int n, const int32_t* __restrict__ nbr_ptr, const int32_t* __restrict__ level,
-                                  int by_level, int chunk, int max_class, int32_t* __restrict__ hist) {
+// segment of v: v / chunk (by_level == 0) or level[v].  A block of 256 consecutive ids lies inside one chunk
+// (chunks are multiples of 1024), so in chunk mode the block first counts in shared memory and then issues at
+// most max_class global atomics; in level mode the counters are spread over the levels and contention is low.
+__global__ void __launch_bounds__(256) class_hist_kernel(int n, const int32_t* __restrict__ nbr_ptr,
+                                                         const int32_t* __restrict__ level, int by_level, int chunk,
+                                                         int max_class, int32_t* __restrict__ hist) {
+    __shared__ int local[8];
     int v = blockIdx.x * blockDim.x + threadIdx.x;
-    if (v >= n) return;
-    int cls = nbr_ptr[v + 1] - nbr_ptr[v];
-    int seg = by_level ? level[v] : (chunk > 0 ? v / chunk : 0);
-    atomicAdd(&hist[(int64_t)seg * (max_class + 1) + (cls - 1)], 1);
+    if (by_level) {
+        if (v >= n) return;
+        int cls = nbr_ptr[v + 1] - nbr_ptr[v];
+        atomicAdd(&hist[(int64_t)level[v] * (max_class + 1) + (cls - 1)], 1);
+        return;
+    }
+    if (threadIdx.x < 8) local[threadIdx.x] = 0;
+    __syncthreads();
+    if (v < n) atomicAdd(&local[nbr_ptr[v + 1] - nbr_ptr[v] - 1], 1);
+    __syncthreads();
+    if (threadIdx.x < max_class && local[threadIdx.x] > 0) {
+        int seg = chunk > 0 ? (int)(((int64_t)blockIdx.x * blockDim.x) / chunk) : 0;
+        atomicAdd(&hist[(int64_t)seg * (max_class + 1) + threadIdx.x], local[threadIdx.x]);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
