@@ -351,3 +351,41 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     torch.cuda.synchronize()
     assert int(status.item()) == dg4.DG4_ERR_TIMEOUT
     assert float((torch.ones(8, device="cuda") * 2).sum().item()) == 16.0
+
+
+@pytest.mark.parametrize("hops,heads,residual,mode", [(1, 1, True, "wavefront"), (2, 4, False, "wavefront"),
+                                                      (2, 16, True, "wavefront"), (1, 2, False, "parallel"),
+                                                      (2, 16, True, "parallel"), (1, 4, True, "level-launches")])
+def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
+    rng = np.random.default_rng(1000 * hops + heads)
+    fanins = random_dag(rng, 40, 6000, window=300)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    n = len(fanins)
+    gr = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+    xb = synth.normal_bf16_bits(7, 1, (n, 128), 1.0)
+    weights = [bf16_weights(synth.normal_f32(7, 10 + l, (384, 128), 0.05)) +
+               bf16_weights(synth.normal_f32(7, 20 + l, (128, 128), 0.05)) for l in range(2)]
+    scale = 1.0 / np.sqrt(128 // heads)
+    dsc = dg4.desc(heads, dg4.DG4_BF16, scale, residual=residual, level_launches=(mode == "level-launches"))
+    ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, 2)),
+                     dtype=torch.uint8, device="cuda")
+    h = dev_bf16(xb).clone()
+    if mode == "parallel":
+        for w_ in weights:
+            dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(w_[0]), dev_bf16(w_[2]), h, ws)
+    else:
+        dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dev_bf16(w_[0]) for w_ in weights], [dev_bf16(w_[2]) for w_ in weights], ws)
+    torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(gr) == 0
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    lptr, lnodes = orc.level_buckets(level)
+    want = f64_of_bits(xb)
+    for (_, wq, _, wo) in weights:
+        if mode == "parallel":
+            want = orc.layer_parallel(want, wq, wo, ptr, idx, heads, scale, residual=residual, rounding="bf16")
+        else:
+            want = orc.layer_levelised(want, wq, wo, ptr, idx, lptr, lnodes, heads, scale, residual=residual,
+                                       rounding="bf16")
+    err = rel_row_err(host_f64_of_bf16(h), want)
+    assert err.max() <= BF16_ROW_TOL, err.max()
