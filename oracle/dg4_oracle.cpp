@@ -18,6 +18,8 @@
  *   orc_attention         Sec. 3.5: multi-head attention restricted to that set; dot-product score and
  *                         softmax per destination (the paper leaves the score function to a figure;
  *                         the dot-product reading is this library's stated choice)
+ *   orc_attention_additive  the same restricted attention with the additive LeakyReLU score of GAT layers
+ *                         (node-level scalars), the form the kernels of Sec. 3.7 aggregate with
  *   orc_project           the dense projections of the Transformer block kept around the attention
  *   orc_layer_parallel    QKV projection -> attention -> output projection (+ residual), all nodes at once
  *   orc_layer_levelised   the same layer applied level by level in topological order, each level
@@ -194,6 +196,38 @@ void orc_attention(int n, int d, int heads, double scale, const double* Q, const
             }
             attend_one(dh, scale, Q + (int64_t)v * d + h * dh, cnt, kr.data(), vr.data(),
                        O + (int64_t)v * d + h * dh, alpha ? a.data() : nullptr);
+            if (alpha) for (int j = 0; j < cnt; ++j) alpha[(int64_t)(lo + j) * heads + h] = a[j];
+        }
+    }
+}
+
+/* Additive (GAT-style) score variant of the restricted attention, the form the fused GAT kernels discussed in
+ * Sec. 2 and Sec. 3.7 aggregate with: per head, e_u = LeakyReLU(S_src[u,h] + S_dst[v,h]) with node-level scalars,
+ * alpha = softmax over the neighbourhood, O[v,h,:] = sum_u alpha_u V[u,h,:].  (The definition is the published
+ * graph-attention one; this paper does not restate it.)  S_dst: [n, heads]; S_src: [n_kv, heads]. */
+void orc_attention_additive(int n, int d, int heads, double slope, const double* S_dst, const double* S_src,
+                            const double* V, const int32_t* nbr_ptr, const int32_t* nbr_idx, double* O, double* alpha) {
+    int dh = d / heads;
+#pragma omp parallel for schedule(static)
+    for (int v = 0; v < n; ++v) {
+        int lo = nbr_ptr[v], cnt = nbr_ptr[v + 1] - lo;
+        std::vector<double> e(cnt), a(cnt);
+        for (int h = 0; h < heads; ++h) {
+            for (int j = 0; j < cnt; ++j) {
+                int64_t u = nbr_idx[lo + j];
+                double x = S_src[u * heads + h] + S_dst[(int64_t)v * heads + h];
+                e[j] = x > 0.0 ? x : slope * x;
+            }
+            double m = e[0];
+            for (int j = 1; j < cnt; ++j) m = std::max(m, e[j]);
+            double z = 0.0;
+            for (int j = 0; j < cnt; ++j) { a[j] = std::exp(e[j] - m); z += a[j]; }
+            for (int j = 0; j < cnt; ++j) a[j] /= z;
+            for (int c = 0; c < dh; ++c) {
+                double acc = 0.0;
+                for (int j = 0; j < cnt; ++j) acc += a[j] * V[(int64_t)nbr_idx[lo + j] * d + h * dh + c];
+                O[(int64_t)v * d + h * dh + c] = acc;
+            }
             if (alpha) for (int j = 0; j < cnt; ++j) alpha[(int64_t)(lo + j) * heads + h] = a[j];
         }
     }

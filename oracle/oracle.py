@@ -47,6 +47,8 @@ def _load():
         lib.orc_class_order.argtypes = [c_int, _i32p, c_int, _i32p, _i32p, c_int, _i32p, _i32p]
         lib.orc_attention.restype = None
         lib.orc_attention.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, _i32p, _i32p, _f64p, _f64p]
+        lib.orc_attention_additive.restype = None
+        lib.orc_attention_additive.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, _i32p, _i32p, _f64p, _f64p]
         lib.orc_project.restype = None
         lib.orc_project.argtypes = [c_int, c_int, c_int, _f64p, _f64p, _f64p, _f64p]
         lib.orc_layer_parallel.restype = None
@@ -150,6 +152,21 @@ def attention(Q, K, V, nbr_ptr, nbr_idx, heads, scale, return_alpha=False):
     O = np.zeros((n, d), np.float64)
     alpha = np.zeros((nbr_idx.shape[0], heads), np.float64) if return_alpha else None
     _load().orc_attention(n, d, heads, float(scale), _d(Q), _d(K), _d(V), _i(nbr_ptr), _i(nbr_idx), _d(O), _d(alpha))
+    return (O, alpha) if return_alpha else O
+
+
+def attention_additive(S_dst, S_src, V, nbr_ptr, nbr_idx, slope=0.2, return_alpha=False):
+    """GAT-style additive scores: e = LeakyReLU(S_src[u,h] + S_dst[v,h]).  S_dst: [n, heads]; S_src: [n_kv, heads];
+    V: [n_kv, d]."""
+    S_dst, S_src, V = _f64(S_dst), _f64(S_src), _f64(V)
+    nbr_ptr, nbr_idx = _i32(nbr_ptr), _i32(nbr_idx)
+    n, heads = S_dst.shape
+    d = V.shape[1]
+    assert nbr_ptr.shape[0] == n + 1 and S_src.shape == (V.shape[0], heads)
+    O = np.zeros((n, d), np.float64)
+    alpha = np.zeros((nbr_idx.shape[0], heads), np.float64) if return_alpha else None
+    _load().orc_attention_additive(n, d, heads, float(slope), _d(S_dst), _d(S_src), _d(V), _i(nbr_ptr), _i(nbr_idx),
+                                   _d(O), _d(alpha))
     return (O, alpha) if return_alpha else O
 
 

@@ -423,3 +423,58 @@ def test_generated_circuits_have_the_stated_shape():
     g = synth.workload(4, 50).graph()
     w = synth.workload(4, 50)
     assert g.level.max() == w.n_levels
+
+
+# ----------------------------------------------------------------------------- additive (GAT-style) scores
+
+def _dense_additive(S_dst, S_src, V, mask, slope):
+    n, heads = S_dst.shape
+    d = V.shape[1]
+    dh = d // heads
+    e = torch.from_numpy(S_dst).T[:, :, None] + torch.from_numpy(S_src).T[:, None, :]       # [h, v, u]
+    e = torch.nn.functional.leaky_relu(e, slope).masked_fill(~torch.from_numpy(mask)[None], float("-inf"))
+    v = torch.from_numpy(V).view(-1, heads, dh).transpose(0, 1)
+    return (torch.softmax(e, dim=-1) @ v).transpose(0, 1).reshape(n, d).numpy()
+
+
+@pytest.mark.parametrize("hops,heads,slope", [(1, 4, 0.2), (2, 8, 0.2), (2, 2, 0.01)])
+def test_additive_attention_equals_dense_masked_gat(hops, heads, slope):
+    rng = np.random.default_rng(50 + hops + heads)
+    fanins = random_dag(rng, 6, 150, window=12)
+    n, d = len(fanins), 32
+    rp, ci = csr_from_fanins(fanins)
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    sd, ss, V = 2 * rng.standard_normal((n, heads)), 2 * rng.standard_normal((n, heads)), rng.standard_normal((n, d))
+    want = _dense_additive(sd, ss, V, _mask_from_nbr(ptr, idx, n), slope)
+    got, alpha = orc.attention_additive(sd, ss, V, ptr, idx, slope, return_alpha=True)
+    assert np.abs(got - want).max() < 1e-12
+    for v in range(n):
+        assert np.abs(alpha[ptr[v]:ptr[v + 1]].sum(0) - 1.0).max() < 1e-12
+
+
+def test_additive_attention_closed_forms():
+    rng = np.random.default_rng(60)
+    fanins, root, _ = binary_in_tree(2)
+    n, d, heads = len(fanins), 8, 2
+    rp, ci = csr_from_fanins(fanins)
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    V = rng.standard_normal((n, d))
+    sd = rng.standard_normal((n, heads))
+    # equal source terms: every score of a node is the same, so the output is the plain mean of the rows
+    O = orc.attention_additive(sd, np.zeros((n, heads)), V, ptr, idx, 0.2)
+    assert np.allclose(O[root], V.mean(0), atol=1e-14)
+    assert (O[:4] == V[:4]).all()                               # leaves see only themselves
+    # slope 1 makes the score linear, so the destination term shifts all scores of a node alike and drops out
+    ss = rng.standard_normal((n, heads))
+    a = orc.attention_additive(sd, ss, V, ptr, idx, 1.0)
+    b = orc.attention_additive(np.zeros_like(sd), ss, V, ptr, idx, 1.0)
+    assert np.abs(a - b).max() < 1e-12
+    # hand case: one head, scores LeakyReLU(ln 3 + 0) = ln 3 and LeakyReLU(-5 + 0) = -1 with slope 0.2:
+    # weights 3 / (3 + e^-1) and e^-1 / (3 + e^-1)
+    ptr2, idx2 = np.array([0, 1, 3], np.int32), np.array([0, 1, 0], np.int32)
+    V2 = np.array([[2.0, 0.0], [0.0, 4.0]])
+    ss2 = np.array([[-5.0], [np.log(3.0)]])
+    O2, al = orc.attention_additive(np.zeros((2, 1)), ss2, V2, ptr2, idx2, 0.2, return_alpha=True)
+    z = 3.0 + np.exp(-1.0)
+    assert np.allclose(al[1:, 0], [3.0 / z, np.exp(-1.0) / z], atol=1e-15)
+    assert np.allclose(O2[1], (3.0 / z) * V2[1] + (np.exp(-1.0) / z) * V2[0], atol=1e-15)
