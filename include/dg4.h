@@ -167,6 +167,19 @@ dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* desc,
                                const void* V, int64_t ldv, void* O, int64_t ldo, void* stream);
 
 /*
+ * The same fused attention with the additive score of graph-attention layers (the form the fused GAT kernels
+ * discussed in Sec. 2 and Sec. 3.7 aggregate with; the paper does not restate the formula): per head h
+ *     e_u = LeakyReLU(S_src[u,h] + S_dst[v,h]),  alpha = softmax over u in N(v),  O[v,h,:] = sum_u alpha_u V[u,h,:]
+ * with node-level scalars instead of key rows (a neighbour then costs one value row plus 4 bytes per head).
+ *   S_dst, S_src    device, [n, heads] fp32, contiguous
+ *   negative_slope  of the LeakyReLU (0.2 in the usual definition)
+ *   V, O            device, [n, d] of desc->dtype; O must not alias V.  desc->scale is not used.
+ */
+dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4_desc* desc,
+                                        const float* S_dst, const float* S_src, float negative_slope,
+                                        const void* V, int64_t ldv, void* O, int64_t ldo, void* stream);
+
+/*
  * Output projection: H_out = O * W_o^T (+ H_res if desc->flags has DG4_FLAG_RESIDUAL and H_res != NULL).
  *   O device [n, d] bf16;  W_o device [d, d] bf16 (output-major);  H_res device [n, d] bf16 or NULL;
  *   H_out device [n, d] bf16; may alias H_res (each row is read before it is written by the same thread).

@@ -78,12 +78,67 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(d
     }
 }
 
+// Additive (GAT-style) scores: e = LeakyReLU(S_src[u, head] + S_dst[v, head]) from node-level scalars, so a
+// neighbour costs one value row and one 4-byte scalar per head instead of a key row; same persistent walk.
+template <bool BF16, int LPH, int MAXN>
+__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive_kernel(dg4i_attn_args a) {
+    constexpr int G = BF16 ? 16 : 32;
+    constexpr int EPP = Elem<BF16>::kPerPiece;
+    constexpr int ES = BF16 ? 2 : 4;
+    constexpr int W = MAXN + 1;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane & (G - 1);
+    const int grp_base = lane - sub;
+    const unsigned mask = (G == 32) ? 0xffffffffu : (0xffffu << grp_base);
+    const int stride = (int)(gridDim.x * (blockDim.x / G));
+    int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) / G);
+    const size_t col = (size_t)sub * EPP * ES;
+    const int head = sub / LPH;                    // the head this lane's piece belongs to
+
+    int v_next = -1, pad_next = 0;
+    if (slot < a.count) {
+        v_next = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
+        if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+    }
+    for (; slot < a.count; slot += stride) {
+        const int v = v_next;
+        const int pad = pad_next;
+        {
+            const int s2 = slot + stride;
+            if (s2 < a.count) {
+                v_next = a.node_list ? a.node_list[a.first + s2] : a.first + s2;
+                if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+            }
+        }
+        const int cnt = __shfl_sync(mask, pad, grp_base);
+        Piece vq[MAXN];
+        float ss[MAXN];
+        int u[MAXN];
+        u[0] = v;
+#pragma unroll
+        for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(mask, pad, grp_base + j);
+#pragma unroll
+        for (int j = 0; j < MAXN; ++j) {
+            ss[j] = 0.f;
+            if (j < cnt) {
+                vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
+                if (cnt > 1) ss[j] = __ldg(a.s_src + (size_t)u[j] * a.heads + head);
+            }
+        }
+        const float sd = cnt > 1 ? __ldg(a.s_dst + (size_t)v * a.heads + head) : 0.f;
+        float acc[EPP];
+        attend_additive<BF16, MAXN>(sd, ss, vq, cnt, a.slope, acc);
+        st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
+    }
+}
+
 struct LaunchShape { int sm_count = 0; int blocks_per_sm = 0; };
 
-template <bool BF16, int LPH, int MAXN>
+template <bool BF16, int LPH, int MAXN, bool ADDITIVE>
 dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     const int threads = 256;
+    auto kern = ADDITIVE ? sparse_attn_additive_kernel<BF16, LPH, MAXN> : sparse_attn_kernel<BF16, LPH, MAXN>;
     static LaunchShape shape[64];
     int dev = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
@@ -91,7 +146,7 @@ dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
     if (shape[dev].sm_count == 0) {
         int sms = 0, per_sm = 0;
         DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sparse_attn_kernel<BF16, LPH, MAXN>, threads, 0));
+        DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0));
         shape[dev].blocks_per_sm = per_sm > 0 ? per_sm : 1;
         shape[dev].sm_count = sms;
     }
@@ -99,34 +154,40 @@ dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
     const int64_t needed = ((int64_t)a.count + nodes_per_block - 1) / nodes_per_block;
     const int64_t resident = (int64_t)shape[dev].sm_count * shape[dev].blocks_per_sm;
     const unsigned blocks = (unsigned)(needed < resident ? needed : resident);
-    sparse_attn_kernel<BF16, LPH, MAXN><<<blocks, threads, 0, st>>>(a);
+    kern<<<blocks, threads, 0, st>>>(a);
     dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
 
-template <bool BF16, int MAXN>
+template <bool BF16, int MAXN, bool ADDITIVE>
 dg4_status launch_for_heads(const dg4i_attn_args& a, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     switch (G / a.heads) {
-        case 1: return launch_one<BF16, 1, MAXN>(a, st);
-        case 2: return launch_one<BF16, 2, MAXN>(a, st);
-        case 4: return launch_one<BF16, 4, MAXN>(a, st);
-        case 8: return launch_one<BF16, 8, MAXN>(a, st);
-        case 16: return launch_one<BF16, 16, MAXN>(a, st);
-        case 32: if (G == 32) return launch_one<BF16, (G == 32 ? 32 : 16), MAXN>(a, st);
+        case 1: return launch_one<BF16, 1, MAXN, ADDITIVE>(a, st);
+        case 2: return launch_one<BF16, 2, MAXN, ADDITIVE>(a, st);
+        case 4: return launch_one<BF16, 4, MAXN, ADDITIVE>(a, st);
+        case 8: return launch_one<BF16, 8, MAXN, ADDITIVE>(a, st);
+        case 16: return launch_one<BF16, 16, MAXN, ADDITIVE>(a, st);
+        case 32: if (G == 32) return launch_one<BF16, (G == 32 ? 32 : 16), MAXN, ADDITIVE>(a, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
 }
 
 }  // namespace
 
-dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st) {
+namespace {
+template <bool ADDITIVE>
+dg4_status attn_dispatch(const dg4i_attn_args& a, cudaStream_t st) {
     if (a.count <= 0) return DG4_OK;
     const bool bf16 = a.dtype == DG4_BF16;
     const int G = bf16 ? 16 : 32;
     if (a.heads < 1 || a.heads > G || (G % a.heads) != 0)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must divide %d", a.heads, G);
-    if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3>(a, st) : launch_for_heads<false, 3>(a, st);
-    return bf16 ? launch_for_heads<true, 7>(a, st) : launch_for_heads<false, 7>(a, st);
+    if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3, ADDITIVE>(a, st) : launch_for_heads<false, 3, ADDITIVE>(a, st);
+    return bf16 ? launch_for_heads<true, 7, ADDITIVE>(a, st) : launch_for_heads<false, 7, ADDITIVE>(a, st);
 }
+}  // namespace
+
+dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st) { return attn_dispatch<false>(a, st); }
+dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, cudaStream_t st) { return attn_dispatch<true>(a, st); }

@@ -94,30 +94,10 @@ template <> struct Elem<false> {
     }
 };
 
-// Scores, softmax and weighted sum for one lane's piece of one node.  qp, kq[j], vq[j]: this lane's pieces
-// of the query row and of neighbour j's key / value rows (j < cnt; cnt >= 1).  `mask` names the lanes of this
-// node's group: they share cnt, so they take the same path and meet in the score-reduction shuffles; other
-// groups of the warp may be on a different path.
-template <bool BF16, int LPH, int MAXN>
-__device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const Piece* vq, int cnt, float scale,
-                                       unsigned mask, float* acc /*[kPerPiece]*/) {
+// Softmax over the scores s[0..cnt) (log2 units, maximum m) and the weighted sum of this lane's value pieces.
+template <bool BF16, int MAXN>
+__device__ __forceinline__ void softmax_weighted_sum(const float* s, float m, int cnt, const Piece* vq, float* acc) {
     constexpr int EPP = Elem<BF16>::kPerPiece;
-    if (cnt <= 1) {                                   // softmax over one element: weight exactly 1
-        Elem<BF16>::unpack(vq[0], acc);
-        return;
-    }
-    const float c = scale * 1.4426950408889634f;      // scores kept in log2 units
-    float s[MAXN];
-    float m = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < MAXN; ++j) {
-        float dot = 0.f;
-        if (j < cnt) dot = Elem<BF16>::dot(qp, kq[j]);
-#pragma unroll
-        for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
-        s[j] = (j < cnt) ? dot * c : -INFINITY;
-        m = fmaxf(m, s[j]);
-    }
     float z = 0.f;
 #pragma unroll
     for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
@@ -135,6 +115,53 @@ __device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const P
     const float inv = fast_rcp(z);
 #pragma unroll
     for (int i = 0; i < EPP; ++i) acc[i] *= inv;
+}
+
+// Scores, softmax and weighted sum for one lane's piece of one node.  qp, kq[j], vq[j]: this lane's pieces
+// of the query row and of neighbour j's key / value rows (j < cnt; cnt >= 1).  `mask` names the lanes of this
+// node's group: they share cnt, so they take the same path and meet in the score-reduction shuffles; other
+// groups of the warp may be on a different path.
+template <bool BF16, int LPH, int MAXN>
+__device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const Piece* vq, int cnt, float scale,
+                                       unsigned mask, float* acc /*[kPerPiece]*/) {
+    if (cnt <= 1) {                                   // softmax over one element: weight exactly 1
+        Elem<BF16>::unpack(vq[0], acc);
+        return;
+    }
+    const float c = scale * 1.4426950408889634f;      // scores kept in log2 units
+    float s[MAXN];
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < MAXN; ++j) {
+        float dot = 0.f;
+        if (j < cnt) dot = Elem<BF16>::dot(qp, kq[j]);
+#pragma unroll
+        for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(mask, dot, o);
+        s[j] = (j < cnt) ? dot * c : -INFINITY;
+        m = fmaxf(m, s[j]);
+    }
+    softmax_weighted_sum<BF16, MAXN>(s, m, cnt, vq, acc);
+}
+
+// Additive-score variant: this lane's head has the node-level scalars s_dst (of the destination) and s_src[j]
+// (of neighbour j); score = LeakyReLU(s_src[j] + s_dst).  No cross-lane traffic at all.
+template <bool BF16, int MAXN>
+__device__ __forceinline__ void attend_additive(float s_dst, const float* s_src, const Piece* vq, int cnt, float slope,
+                                                float* acc /*[kPerPiece]*/) {
+    if (cnt <= 1) {
+        Elem<BF16>::unpack(vq[0], acc);
+        return;
+    }
+    float s[MAXN];
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < MAXN; ++j) {
+        float x = s_src[j] + s_dst;
+        x = (x > 0.f ? x : slope * x) * 1.4426950408889634f;
+        s[j] = (j < cnt) ? x : -INFINITY;
+        m = fmaxf(m, s[j]);
+    }
+    softmax_weighted_sum<BF16, MAXN>(s, m, cnt, vq, acc);
 }
 
 }  // namespace attn

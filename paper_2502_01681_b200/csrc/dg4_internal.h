@@ -86,8 +86,13 @@ struct dg4i_attn_args {
     int32_t max_nbr;            // 3 or 7
     int32_t dtype;
     float scale;
+    // additive-score variant (dg4i_attn_additive_launch): node-level scalars [n, heads] fp32; Q and K unused
+    const float* s_dst = nullptr;
+    const float* s_src = nullptr;
+    float slope = 0.f;
 };
 dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st);
+dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, cudaStream_t st);
 
 // Y[r, 0:n_out] = A[r, 0:128] * W[0:n_out, 0:128]^T (+ R[r, :]) for rows r of a list (or 0..rows-1).
 // Output column block j (of 128) goes to out[j] with leading dimension ldo[j].

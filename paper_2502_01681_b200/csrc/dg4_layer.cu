@@ -140,6 +140,23 @@ extern "C" dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* de
     return dg4i_attn_launch(attn_args(g, desc, Q, ldq, K, ldk, V, ldv, O, ldo), (cudaStream_t)stream);
 }
 
+extern "C" dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4_desc* desc, const float* S_dst,
+                                                    const float* S_src, float negative_slope, const void* V,
+                                                    int64_t ldv, void* O, int64_t ldo, void* stream) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(check_desc(desc, false));
+    if (!S_dst || !S_src) DG4_FAIL(DG4_ERR_INVALID_ARG, "null score array");
+    if ((((uintptr_t)S_dst) | ((uintptr_t)S_src)) & 3u) DG4_FAIL(DG4_ERR_INVALID_ARG, "score arrays must be 4-byte aligned");
+    if (!(negative_slope == negative_slope)) DG4_FAIL(DG4_ERR_INVALID_ARG, "negative_slope is not a number");
+    const int es = desc->dtype == DG4_BF16 ? 2 : 4;
+    CHECK(check_tensor("V", V, ldv, es, 128));
+    CHECK(check_tensor("O", O, ldo, es, 128));
+    if (O == V) DG4_FAIL(DG4_ERR_INVALID_ARG, "O must not alias V");
+    dg4i_attn_args a = attn_args(g, desc, nullptr, 0, nullptr, 0, V, ldv, O, ldo);
+    a.s_dst = S_dst; a.s_src = S_src; a.slope = negative_slope;
+    return dg4i_attn_additive_launch(a, (cudaStream_t)stream);
+}
+
 extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, const void* O, int64_t ldo,
                                        const void* W_o, const void* H_res, int64_t ldh, void* H_out, int64_t ldho,
                                        void* stream) {

@@ -39,7 +39,7 @@ EXPORTS = [
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_poll_status", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
-    "dg4_selftest_bounded_wait",
+    "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd",
 ]
 
 
@@ -106,6 +106,8 @@ def load():
     lib.dg4_qkv_project.argtypes = [vp, dp, vp, i64, vp, vp, i64, vp, i64, vp, i64, vp]
     lib.dg4_sparse_attn_fwd.restype = ctypes.c_int
     lib.dg4_sparse_attn_fwd.argtypes = [vp, dp, vp, i64, vp, i64, vp, i64, vp, i64, vp]
+    lib.dg4_sparse_attn_additive_fwd.restype = ctypes.c_int
+    lib.dg4_sparse_attn_additive_fwd.argtypes = [vp, dp, vp, vp, ctypes.c_float, vp, i64, vp, i64, vp]
     lib.dg4_out_project.restype = ctypes.c_int
     lib.dg4_out_project.argtypes = [vp, dp, vp, i64, vp, vp, i64, vp, i64, vp]
     lib.dg4_layer_workspace_bytes.restype = ctypes.c_size_t
@@ -294,3 +296,9 @@ def dg4_layers_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, w
 
 def dg4_selftest_bounded_wait(device_status, stream=None):
     _check(load().dg4_selftest_bounded_wait(_ptr(device_status), _stream(stream)))
+
+
+def dg4_sparse_attn_additive_fwd(g: Graph, dsc: dg4_desc, S_dst, S_src, negative_slope, V, O, stream=None):
+    assert S_dst.is_contiguous() and S_src.is_contiguous()
+    _check(load().dg4_sparse_attn_additive_fwd(g.handle, ctypes.byref(dsc), _ptr(S_dst), _ptr(S_src),
+                                               float(negative_slope), _ptr(V), _ld(V), _ptr(O), _ld(O), _stream(stream)))

@@ -389,3 +389,35 @@ def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
                                        rounding="bf16")
     err = rel_row_err(host_f64_of_bf16(h), want)
     assert err.max() <= BF16_ROW_TOL, err.max()
+
+
+@pytest.mark.parametrize("dtype,hops,heads", [("f32", 1, 4), ("f32", 2, 8), ("bf16", 2, 8), ("bf16", 1, 1),
+                                              ("bf16", 2, 16), ("f32", 2, 32)])
+def test_additive_score_attention_matches_checker(dtype, hops, heads):
+    rng = np.random.default_rng(7000 + heads + hops)
+    fanins = random_dag(rng, 40, 5000, window=200)
+    rp, ci = csr_from_fanins(fanins)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, levels_of(fanins), hops, 0)
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    sd = synth.normal_f32(3, 80, (n, heads), 1.5)
+    ss = synth.normal_f32(3, 81, (n, heads), 1.5)
+    v32 = synth.normal_f32(3, 82, (n, 128), 1.0)
+    dsd, dss = torch.from_numpy(sd).cuda(), torch.from_numpy(ss).cuda()
+    if dtype == "f32":
+        dv = torch.from_numpy(v32).cuda()
+        o = torch.empty_like(dv)
+        dg4.dg4_sparse_attn_additive_fwd(g, dg4.desc(heads, dg4.DG4_F32, 1.0), dsd, dss, 0.2, dv, o)
+        torch.cuda.synchronize()
+        want = orc.attention_additive(sd, ss, v32, ptr, idx, 0.2)
+        assert np.abs(o.cpu().numpy().astype(np.float64) - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+    else:
+        vb = synth.f32_to_bf16_bits(v32)
+        dv = dev_bf16(vb)
+        o = torch.empty_like(dv)
+        dg4.dg4_sparse_attn_additive_fwd(g, dg4.desc(heads, dg4.DG4_BF16, 1.0), dsd, dss, 0.2, dv, o)
+        torch.cuda.synchronize()
+        want = orc.round_bf16(orc.attention_additive(sd, ss, f64_of_bits(vb), ptr, idx, 0.2))
+        assert rel_row_err(host_f64_of_bf16(o), want).max() <= BF16_ROW_TOL
+        pis = np.nonzero(np.diff(ptr) == 1)[0]
+        assert torch.equal(o[torch.from_numpy(pis).cuda()], dv[torch.from_numpy(pis).cuda()])    # weight exactly 1
