@@ -111,7 +111,11 @@ int64_t dg4_launch_count(void);
  *   row_ptr     host, [n_nodes+1], destination-sorted CSR of DIRECT fan-ins (no self entry)
  *   col_idx     host, [row_ptr[n_nodes]], source ids; any order inside a row; a repeated source is allowed
  *   level       host, [n_nodes]; any layering with level[u] < level[v] on every edge is accepted
- *   hops        1 (fan-ins + self) or 2 (2-hop fan-in cone + self)
+ *   hops        1 (fan-ins + self), 2 (2-hop fan-in cone + self), or 3 .. 8 (wider cones, the paper uses k = 8:
+ *               up to 2^(hops+1)-1 members).  For hops > 2 only the neighbourhood CSR and the level buckets are
+ *               built (no fixed-width table, no class orderings: exporting those returns DG4_ERR_UNSUPPORTED),
+ *               the lists must stay below 2^31 entries, dg4_graph_rebuild is not available, and the levelised
+ *               layer runs only with DG4_FLAG_LEVEL_LAUNCHES.
  *   perm_chunk  0 (one chunk) or a positive multiple of 1024
  *   device      CUDA ordinal; made current for the duration of the call and restored
  *   out         receives the handle; untouched on error

@@ -132,6 +132,124 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive
     }
 }
 
+// Wider cones (3 to 8 hops, up to 511 neighbours, Sec. 3.2 with the paper's k = 8): one warp per node, the
+// neighbour list in CSR form walked in chunks; for bf16 the two half-warps take alternate neighbours.  Each lane
+// keeps an online softmax (running maximum and sum, in log2 units) over the neighbours its half has seen and the
+// matching weighted sum of its value piece; the halves are merged at the end.  Four neighbours per half are in
+// flight at a time.
+template <bool BF16, int LPH>
+__global__ void __launch_bounds__(256) sparse_attn_wide_kernel(dg4i_attn_args a) {
+    constexpr int G = BF16 ? 16 : 32;              // lanes per row
+    constexpr int HALVES = 32 / G;                 // neighbours a warp handles side by side
+    constexpr int EPP = Elem<BF16>::kPerPiece;
+    constexpr int ES = BF16 ? 2 : 4;
+    constexpr int UN = 4;                          // neighbours in flight per half
+    const int lane = threadIdx.x & 31;
+    const int sub = lane & (G - 1);
+    const int half = lane / G;
+    const unsigned hmask = (G == 32) ? 0xffffffffu : (0xffffu << (lane - sub));
+    const size_t col = (size_t)sub * EPP * ES;
+    const int warps = (int)(gridDim.x * (blockDim.x >> 5));
+    const float c = a.scale * 1.4426950408889634f;
+    for (int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); slot < a.count; slot += warps) {
+        const int v = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
+        const int beg = a.nbr_ptr[v];
+        const int cnt = a.nbr_ptr[v + 1] - beg;
+        const Piece qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
+        float m = -INFINITY, z = 0.f, acc[EPP];
+#pragma unroll
+        for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
+        for (int base = 0; base < cnt; base += 32) {
+            const int my_u = (base + lane < cnt) ? a.nbr_idx[beg + base + lane] : -1;
+            const int chunk = cnt - base < 32 ? cnt - base : 32;
+            for (int t = 0; t < chunk; t += HALVES * UN) {
+                Piece kq[UN], vq[UN];
+                int u[UN];
+#pragma unroll
+                for (int i = 0; i < UN; ++i) {
+                    const int j = t + i * HALVES + half;                       // position inside the chunk
+                    u[i] = __shfl_sync(0xffffffffu, my_u, j & 31);
+                    if (j >= chunk) u[i] = -1;
+                }
+#pragma unroll
+                for (int i = 0; i < UN; ++i) {
+                    if (u[i] >= 0) {
+                        kq[i] = ld_piece_nc((const char*)a.K + (size_t)u[i] * a.ldk * ES + col);
+                        vq[i] = ld_piece_nc((const char*)a.V + (size_t)u[i] * a.ldv * ES + col);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < UN; ++i) {
+                    float dot = (u[i] >= 0) ? Elem<BF16>::dot(qp, kq[i]) : 0.f;
+#pragma unroll
+                    for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(hmask, dot, o);
+                    if (u[i] >= 0) {                                           // uniform inside a half
+                        const float s = dot * c;
+                        const float m_new = fmaxf(m, s);
+                        const float keep = fast_exp2(m - m_new);               // 0 on the first neighbour (m = -inf)
+                        const float p = fast_exp2(s - m_new);
+                        float vf[EPP];
+                        Elem<BF16>::unpack(vq[i], vf);
+                        z = z * keep + p;
+#pragma unroll
+                        for (int e = 0; e < EPP; ++e) acc[e] = fmaf(p, vf[e], acc[e] * keep);
+                        m = m_new;
+                    }
+                }
+            }
+        }
+        if (HALVES == 2) {                       // merge the two halves' partial softmaxes
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, 16);
+            const float z2 = __shfl_xor_sync(0xffffffffu, z, 16);
+            const float mm = fmaxf(m, m2);
+            const float w1 = fast_exp2(m - mm), w2 = (m2 == -INFINITY) ? 0.f : fast_exp2(m2 - mm);
+            z = z * w1 + z2 * w2;
+#pragma unroll
+            for (int e = 0; e < EPP; ++e) {
+                const float a2 = __shfl_xor_sync(0xffffffffu, acc[e], 16);
+                acc[e] = acc[e] * w1 + a2 * w2;
+            }
+        }
+        if (half == 0) {
+            if (cnt == 1) {                      // a single neighbour (v itself): weight exactly 1
+                // acc = 1 * V row, z = 1 already; nothing to normalise
+            } else {
+                const float inv = fast_rcp(z);
+#pragma unroll
+                for (int e = 0; e < EPP; ++e) acc[e] *= inv;
+            }
+            st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
+        }
+    }
+}
+
+template <bool BF16, int LPH>
+dg4_status launch_wide(const dg4i_attn_args& a, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    DG4_CUDA_TRY(cudaGetDevice(&dev));
+    DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int64_t needed = ((int64_t)a.count + 7) / 8;
+    const int64_t resident = (int64_t)sms * 4;
+    sparse_attn_wide_kernel<BF16, LPH><<<(unsigned)(needed < resident ? needed : resident), 256, 0, st>>>(a);
+    dg4i_count_launch();
+    DG4_CUDA_TRY(cudaGetLastError());
+    return DG4_OK;
+}
+
+template <bool BF16>
+dg4_status launch_wide_heads(const dg4i_attn_args& a, cudaStream_t st) {
+    constexpr int G = BF16 ? 16 : 32;
+    switch (G / a.heads) {
+        case 1: return launch_wide<BF16, 1>(a, st);
+        case 2: return launch_wide<BF16, 2>(a, st);
+        case 4: return launch_wide<BF16, 4>(a, st);
+        case 8: return launch_wide<BF16, 8>(a, st);
+        case 16: return launch_wide<BF16, 16>(a, st);
+        case 32: if (G == 32) return launch_wide<BF16, (G == 32 ? 32 : 16)>(a, st);
+    }
+    DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
+}
+
 struct LaunchShape { int sm_count = 0; int blocks_per_sm = 0; };
 
 template <bool BF16, int LPH, int MAXN, bool ADDITIVE>
@@ -184,6 +302,10 @@ dg4_status attn_dispatch(const dg4i_attn_args& a, cudaStream_t st) {
     const int G = bf16 ? 16 : 32;
     if (a.heads < 1 || a.heads > G || (G % a.heads) != 0)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must divide %d", a.heads, G);
+    if (a.max_nbr > 7) {
+        if (ADDITIVE) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the additive-score variant supports cones of at most two hops");
+        return bf16 ? launch_wide_heads<true>(a, st) : launch_wide_heads<false>(a, st);
+    }
     if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3, ADDITIVE>(a, st) : launch_for_heads<false, 3, ADDITIVE>(a, st);
     return bf16 ? launch_for_heads<true, 7, ADDITIVE>(a, st) : launch_for_heads<false, 7, ADDITIVE>(a, st);
 }

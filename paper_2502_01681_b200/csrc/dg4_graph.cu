@@ -287,6 +287,10 @@ dg4_status sort_by_level(dg4_graph* g, const int32_t* first, int32_t* dst, cudaS
 
 }  // namespace
 
+dg4_status dg4i_exclusive_scan(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t st) {
+    return exclusive_scan(in, out, n, block_sums, st);
+}
+
 // ------------------------------------------------------------------------------------------------
 // device pass (a2..a4).  first_time: stops after the neighbourhood sizes are known so that the caller can
 // size nbr_idx; it is then called again with first_time == false.
@@ -296,13 +300,15 @@ dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only
     const int tb = 256, nbk = (n + tb - 1) / tb;
     dg4_status s;
 
-    // neighbourhood sizes -> nbr_ptr
-    cone_count_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr);
-    dg4i_count_launch();
-    if ((s = exclusive_scan(g->nbr_ptr, g->nbr_ptr, (int64_t)n + 1, g->block_sums, st)) != DG4_OK) return s;
-    if (sizes_only) return DG4_OK;
-    cone_fill_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr, g->nbr_idx, g->pad_width, g->nbr_pad);
-    dg4i_count_launch();
+    if (!g->wide) {
+        // neighbourhood sizes -> nbr_ptr
+        cone_count_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr);
+        dg4i_count_launch();
+        if ((s = exclusive_scan(g->nbr_ptr, g->nbr_ptr, (int64_t)n + 1, g->block_sums, st)) != DG4_OK) return s;
+        if (sizes_only) return DG4_OK;
+        cone_fill_kernel<<<nbk, tb, 0, st>>>(n, g->row_ptr, g->col_idx, g->hops, g->nbr_ptr, g->nbr_idx, g->pad_width, g->nbr_pad);
+        dg4i_count_launch();
+    }
 
     // level buckets
     DG4_CUDA_TRY(cudaMemsetAsync(g->level_ptr, 0, ((size_t)g->n_levels + 1) * sizeof(int32_t), st));
@@ -310,6 +316,11 @@ dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only
     dg4i_count_launch();
     if ((s = exclusive_scan(g->level_ptr, g->level_ptr, (int64_t)g->n_levels + 1, g->block_sums, st)) != DG4_OK) return s;
     if ((s = sort_by_level(g, nullptr, g->level_nodes, st)) != DG4_OK) return s;
+
+    if (g->wide) {            // wider cones: lists come from dg4i_build_wide_cones; no class orderings
+        DG4_CUDA_TRY(cudaGetLastError());
+        return DG4_OK;
+    }
 
     // degree-class order inside id chunks
     const int mc1 = g->max_class + 1;
@@ -381,7 +392,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
                                         dg4_graph** out) {
     if (!row_ptr || !level || !out) DG4_FAIL(DG4_ERR_INVALID_ARG, "null pointer argument");
     if (n_nodes < 1) DG4_FAIL(DG4_ERR_INVALID_ARG, "n_nodes must be >= 1 (got %d)", n_nodes);
-    if (hops != 1 && hops != 2) DG4_FAIL(DG4_ERR_UNSUPPORTED, "hops must be 1 or 2 (got %d)", hops);
+    if (hops < 1 || hops > 8) DG4_FAIL(DG4_ERR_UNSUPPORTED, "hops must be between 1 and 8 (got %d)", hops);
     if (perm_chunk < 0 || (perm_chunk % kTile) != 0)
         DG4_FAIL(DG4_ERR_INVALID_ARG, "perm_chunk must be 0 or a positive multiple of %d (got %d)", kTile, perm_chunk);
 
@@ -448,7 +459,8 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     g->e = n_edges;
     g->hops = hops;
     g->max_class = (1 << (hops + 1)) - 1;
-    g->pad_width = g->max_class + 1;           // 4 or 8 int32: 16 or 32 bytes per node
+    g->wide = hops > 2;
+    g->pad_width = g->wide ? 0 : g->max_class + 1;   // 4 or 8 int32: 16 or 32 bytes per node
     g->n_levels = max_level + 1;
     g->perm_chunk = (perm_chunk >= n_nodes) ? 0 : perm_chunk;
     g->n_chunks = g->perm_chunk > 0 ? (n_nodes + g->perm_chunk - 1) / g->perm_chunk : 1;
@@ -456,7 +468,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     const int64_t n = n_nodes;
     const int64_t nb = (n + kTile - 1) / kTile;
     const int64_t bpc = g->perm_chunk > 0 ? g->perm_chunk / kTile : nb;
-    const int64_t mc1 = g->max_class + 1;
+    const int64_t mc1 = g->wide ? 1 : g->max_class + 1;   // no class arrays for wider cones
     int64_t hist_len = 256 * nb;
     if (hist_len < g->n_chunks * 8 * bpc) hist_len = g->n_chunks * 8 * bpc;
     g->hist_len = hist_len;
@@ -497,12 +509,16 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     if ((ce = cudaMemcpy(g->level, level, (size_t)n * 4, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(ce, "upload of level");
 
     // sizes first, so that nbr_idx can be allocated exactly
-    if ((s = dg4i_graph_device_pass(g, 0, true)) != DG4_OK) return fail(s);
-    int32_t total = 0;
-    if ((ce = cudaMemcpy(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
-    g->n_nbr = total;
-    TRY_ALLOC(g->nbr_idx, g->n_nbr);
-    TRY_ALLOC(g->nbr_pad, n * g->pad_width);
+    if (g->wide) {
+        if ((s = dg4i_build_wide_cones(g)) != DG4_OK) return fail(s);
+    } else {
+        if ((s = dg4i_graph_device_pass(g, 0, true)) != DG4_OK) return fail(s);
+        int32_t total = 0;
+        if ((ce = cudaMemcpy(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
+        g->n_nbr = total;
+        TRY_ALLOC(g->nbr_idx, g->n_nbr);
+        TRY_ALLOC(g->nbr_pad, n * g->pad_width);
+    }
 #undef TRY_ALLOC
     if ((s = dg4i_graph_device_pass(g, 0, false)) != DG4_OK) return fail(s);
 
@@ -516,6 +532,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
 
 extern "C" dg4_status dg4_graph_rebuild(dg4_graph* g, void* stream) {
     if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    if (g->wide) DG4_FAIL(DG4_ERR_UNSUPPORTED, "rebuild is available for cones of at most two hops");
     return dg4i_graph_device_pass(g, (cudaStream_t)stream, false);
 }
 
@@ -546,13 +563,13 @@ const int32_t* array_of(const dg4_graph* g, dg4_array_id which, int64_t* len) {
     switch (which) {
         case DG4_ARR_NBR_PTR: *len = (int64_t)g->n + 1; return g->nbr_ptr;
         case DG4_ARR_NBR_IDX: *len = g->n_nbr; return g->nbr_idx;
-        case DG4_ARR_NBR_PAD: *len = (int64_t)g->n * g->pad_width; return g->nbr_pad;
+        case DG4_ARR_NBR_PAD: *len = g->wide ? 0 : (int64_t)g->n * g->pad_width; return g->wide ? nullptr : g->nbr_pad;
         case DG4_ARR_LEVEL_PTR: *len = (int64_t)g->n_levels + 1; return g->level_ptr;
         case DG4_ARR_LEVEL_NODES: *len = g->n; return g->level_nodes;
-        case DG4_ARR_PERM: *len = g->n; return g->perm;
-        case DG4_ARR_CLASS_PTR: *len = g->n_chunks * mc1; return g->class_ptr;
-        case DG4_ARR_LEVEL_PERM: *len = g->n; return g->level_perm;
-        case DG4_ARR_LEVEL_CLASS_PTR: *len = g->n_levels * mc1; return g->level_class_ptr;
+        case DG4_ARR_PERM: *len = g->wide ? 0 : g->n; return g->wide ? nullptr : g->perm;
+        case DG4_ARR_CLASS_PTR: *len = g->wide ? 0 : g->n_chunks * mc1; return g->wide ? nullptr : g->class_ptr;
+        case DG4_ARR_LEVEL_PERM: *len = g->wide ? 0 : g->n; return g->wide ? nullptr : g->level_perm;
+        case DG4_ARR_LEVEL_CLASS_PTR: *len = g->wide ? 0 : g->n_levels * mc1; return g->wide ? nullptr : g->level_class_ptr;
     }
     *len = 0;
     return nullptr;
@@ -570,7 +587,8 @@ extern "C" dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, i
     if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
     int64_t len = 0;
     const int32_t* src = array_of(g, which, &len);
-    if (!src) DG4_FAIL(DG4_ERR_INVALID_ARG, "unknown array id %d", (int)which);
+    if (!src) DG4_FAIL(which >= 0 && which <= DG4_ARR_NBR_PAD ? DG4_ERR_UNSUPPORTED : DG4_ERR_INVALID_ARG,
+                       "array %d does not exist for this graph", (int)which);
     if (n_written) *n_written = len;
     if (!host_dst) return DG4_OK;
     if (capacity < len) DG4_FAIL(DG4_ERR_INVALID_ARG, "capacity %lld is below the array length %lld", (long long)capacity, (long long)len);

@@ -50,7 +50,8 @@ struct dg4_graph {
     int32_t* nbr_ptr = nullptr;          // [n+1]
     int32_t* nbr_idx = nullptr;          // [n_nbr]
     int32_t* nbr_pad = nullptr;          // [n, pad_width]: |N(v)|, then the members other than v (filler: v)
-    int32_t pad_width = 0;               // max_class + 1
+    int32_t pad_width = 0;               // max_class + 1 (0 for cones wider than two hops: no table)
+    bool wide = false;                   // hops > 2: CSR lists only, no fixed-width table, no class orderings
     int32_t* level_ptr = nullptr;        // [n_levels+1]
     int32_t* level_nodes = nullptr;      // [n]
     int32_t* perm = nullptr;             // [n]
@@ -72,13 +73,19 @@ struct dg4_graph {
 
 // ---- kernels' host launchers (each enqueues on `st` and returns) -----------------------------
 dg4_status dg4i_graph_device_pass(dg4_graph* g, cudaStream_t st, bool sizes_only);
+// exclusive prefix sum of n int32 values (in place allowed); block_sums: scratch of the graph handle
+dg4_status dg4i_exclusive_scan(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t st);
+// cones wider than two hops (graphs created with hops 3..8): fills nbr_ptr, allocates and fills nbr_idx
+dg4_status dg4i_build_wide_cones(dg4_graph* g);
 
 struct dg4i_attn_args {
     const void* Q; int64_t ldq;
     const void* K; int64_t ldk;
     const void* V; int64_t ldv;
     void* O; int64_t ldo;
-    const int32_t* nbr_pad;     // [n, max_nbr + 1] fixed-width neighbour table
+    const int32_t* nbr_pad;     // [n, max_nbr + 1] fixed-width neighbour table (cones of at most two hops)
+    const int32_t* nbr_ptr = nullptr;   // CSR lists, used for wider cones
+    const int32_t* nbr_idx = nullptr;
     const int32_t* node_list;   // nullable: node ids to process; else ids first..first+count-1
     int32_t first;
     int32_t count;

@@ -72,7 +72,7 @@ dg4i_attn_args attn_args(const dg4_graph* g, const dg4_desc* d, const void* Q, i
                          int64_t ldk, const void* V, int64_t ldv, void* O, int64_t ldo) {
     dg4i_attn_args a;
     a.Q = Q; a.ldq = ldq; a.K = K; a.ldk = ldk; a.V = V; a.ldv = ldv; a.O = O; a.ldo = ldo;
-    a.nbr_pad = g->nbr_pad; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.nbr_pad = g->nbr_pad; a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
     a.heads = d->heads; a.max_nbr = g->max_class; a.dtype = d->dtype; a.scale = d->scale;
     return a;
 }
@@ -239,6 +239,8 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
 
+    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layer needs DG4_FLAG_LEVEL_LAUNCHES");
     if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
         // one persistent kernel walks the levels
         int32_t* sync = (int32_t*)((char*)workspace + tensors_bytes(g->n));
@@ -303,6 +305,8 @@ extern "C" dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_des
                  layers_workspace_bytes(g, n_layers));
     cudaStream_t st = (cudaStream_t)stream;
 
+    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layers need DG4_FLAG_LEVEL_LAUNCHES");
     if (desc->flags & DG4_FLAG_LEVEL_LAUNCHES) {       // comparison driver: layer after layer, a launch group per level
         for (int k = 0; k < n_layers; ++k)
             CHECK(dg4_layer_fwd_levelised(g, desc, H, ldh, W_qkv[k], W_o[k], workspace, workspace_bytes_, device_status, stream));

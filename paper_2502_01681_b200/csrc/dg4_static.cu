@@ -97,7 +97,7 @@ extern "C" dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg
 
     dg4i_attn_args a;
     a.Q = Q; a.ldq = 128; a.K = KV; a.ldk = 256; a.V = KV + 128; a.ldv = 256; a.O = O; a.ldo = 128;
-    a.nbr_pad = g->nbr_pad; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.nbr_pad = g->nbr_pad; a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
     a.heads = desc->heads; a.max_nbr = g->max_class; a.dtype = DG4_BF16; a.scale = desc->scale;
     if ((s = dg4i_attn_launch(a, st)) != DG4_OK) return s;
 

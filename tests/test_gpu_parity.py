@@ -421,3 +421,73 @@ def test_additive_score_attention_matches_checker(dtype, hops, heads):
         assert rel_row_err(host_f64_of_bf16(o), want).max() <= BF16_ROW_TOL
         pis = np.nonzero(np.diff(ptr) == 1)[0]
         assert torch.equal(o[torch.from_numpy(pis).cuda()], dv[torch.from_numpy(pis).cuda()])    # weight exactly 1
+
+
+# ----------------------------------------------------------------------------- wider cones (3 to 8 hops)
+
+@pytest.mark.parametrize("hops", [3, 4, 6, 8])
+def test_wide_cone_lists_match_checker(hops):
+    rng = np.random.default_rng(hops)
+    cases = [binary_in_tree(8)[0], random_dag(rng, 30, 4000, window=64), [[]] + [[i - 1] for i in range(1, 300)],
+             [[], [], [0, 0], [2, 2], [1, 3], [3, 4]]]
+    for fanins in cases:
+        rp, ci = csr_from_fanins(fanins)
+        level = levels_of(fanins)
+        g = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+        ptr, idx = orc.neighbourhood(rp, ci, hops)
+        lptr, lnodes = orc.level_buckets(level)
+        assert (dg4.dg4_graph_export(g, dg4.DG4_ARR_NBR_PTR) == ptr).all()
+        assert (dg4.dg4_graph_export(g, dg4.DG4_ARR_NBR_IDX) == idx).all()
+        assert (dg4.dg4_graph_export(g, dg4.DG4_ARR_LEVEL_PTR) == lptr).all()
+        assert (dg4.dg4_graph_export(g, dg4.DG4_ARR_LEVEL_NODES) == lnodes).all()
+        info = dg4.dg4_graph_info(g)
+        assert info.max_class == 2 ** (hops + 1) - 1 and info.n_nbr == len(idx)
+        assert np.diff(ptr).max() <= info.max_class
+        with pytest.raises(dg4.Dg4Error) as e:
+            dg4.dg4_graph_export(g, dg4.DG4_ARR_PERM)
+        assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype,hops,heads", [("bf16", 3, 8), ("bf16", 8, 8), ("bf16", 5, 1), ("bf16", 4, 16),
+                                              ("f32", 3, 4), ("f32", 8, 8), ("f32", 6, 32)])
+def test_wide_cone_attention_matches_checker(dtype, hops, heads):
+    rng = np.random.default_rng(hops * 100 + heads)
+    fanins = random_dag(rng, 30, 3000, window=80)
+    rp, ci = csr_from_fanins(fanins)
+    scale = 1.0 / np.sqrt(128 // heads)
+    got, want = _attention_case(rp, ci, levels_of(fanins), hops, heads, dtype, scale, 1.5)
+    if dtype == "f32":
+        assert np.abs(got - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+    else:
+        assert rel_row_err(got, want).max() <= BF16_ROW_TOL
+
+
+def test_wide_cone_layers_parallel_and_level_launches():
+    rng = np.random.default_rng(31)
+    fanins = random_dag(rng, 30, 2500, window=60)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    n, hops, heads = len(fanins), 4, 8
+    gr = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+    xb = synth.normal_bf16_bits(8, 1, (n, 128), 1.0)
+    wqb, wq = bf16_weights(synth.normal_f32(8, 2, (384, 128), 0.05))
+    wob, wo = bf16_weights(synth.normal_f32(8, 3, (128, 128), 0.05))
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    lptr, lnodes = orc.level_buckets(level)
+    for mode in ("parallel", "level-launches"):
+        dsc = dg4.desc(heads, dg4.DG4_BF16, 0.25, residual=True, level_launches=(mode == "level-launches"))
+        ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+        h = dev_bf16(xb).clone()
+        if mode == "parallel":
+            dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wqb), dev_bf16(wob), h, ws)
+            want = orc.layer_parallel(f64_of_bits(xb), wq, wo, ptr, idx, heads, 0.25, residual=True, rounding="bf16")
+        else:
+            dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wqb), dev_bf16(wob), ws)
+            want = orc.layer_levelised(f64_of_bits(xb), wq, wo, ptr, idx, lptr, lnodes, heads, 0.25, residual=True,
+                                       rounding="bf16")
+        torch.cuda.synchronize()
+        assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL, mode
+    # the persistent level kernel holds at most 7 neighbours in registers: wider cones are refused, not mangled
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_layer_fwd_levelised(gr, dg4.desc(heads, dg4.DG4_BF16, 0.25), h, dev_bf16(wqb), dev_bf16(wob), ws)
+    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED

@@ -41,7 +41,8 @@ def test_status_strings():
     ([0, 0, 1], [1], [0, 1], 1, 0, dg4.DG4_ERR_BAD_LEVEL),             # self loop
     ([0, 0, 1], [5], [0, 1], 1, 0, dg4.DG4_ERR_BAD_LEVEL),             # source out of range
     ([0, 0, 1], [0], [-1, 1], 1, 0, dg4.DG4_ERR_BAD_LEVEL),
-    ([0, 0, 1], [0], [0, 1], 3, 0, dg4.DG4_ERR_UNSUPPORTED),
+    ([0, 0, 1], [0], [0, 1], 9, 0, dg4.DG4_ERR_UNSUPPORTED),
+    ([0, 0, 1], [0], [0, 1], 0, 0, dg4.DG4_ERR_UNSUPPORTED),
     ([0, 0, 1], [0], [0, 1], 1, 100, dg4.DG4_ERR_INVALID_ARG),         # chunk not a multiple of 1024
 ])
 def test_graph_create_rejects_malformed_circuits(row_ptr, col_idx, level, hops, chunk, status):
