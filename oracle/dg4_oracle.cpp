@@ -25,6 +25,7 @@
  *   orc_layer_levelised   the same layer applied level by level in topological order, each level
  *                         reading the rows already updated for earlier levels (Sec. 1 and Sec. 3.4:
  *                         each gate is computed once, in strict level order)
+ *   orc_partition_roots   Algorithm 1 (graph partition): which nodes' cones the partition collects
  *   orc_level_buckets / orc_class_order   index arrays of the graph-prep pass, from their definitions
  *
  * Pins (tests that do not restate these loops): dense masked softmax attention by a library routine on
@@ -153,6 +154,32 @@ int orc_class_order(int n, const int32_t* seq, int n_seg, const int32_t* seg_ptr
         }
     }
     return 0;
+}
+
+/* Algorithm 1 (graph partition): the roots whose cone_k the partition collects.  Taken step by step: levels
+ * l = k, k + delta, ... up to the maximum level contribute every node of that level, in the order the level's
+ * nodes are visited (ascending id); then every node without fan-out is added to the group of its own level.
+ * A node that qualifies both ways is kept once (the groups are treated as sets of cones).  Output: roots grouped
+ * by level, ascending id inside a group; group_ptr[l] = number of roots with level below l (n_levels + 1 entries).
+ * The cone of a root r is cone_k(r), i.e. its list in orc_neighbourhood(hops = k).  Returns the number of roots. */
+int orc_partition_roots(int n, const int32_t* row_ptr, const int32_t* col_idx, const int32_t* level, int n_levels,
+                        int k, int delta, int32_t* roots, int32_t* group_ptr) {
+    std::vector<int> out_degree(n, 0);
+    for (int e = 0; e < row_ptr[n]; ++e) out_degree[col_idx[e]] += 1;
+    std::vector<std::set<int>> cones(n_levels);              /* cones^l, as sets of root ids */
+    const int L = n_levels - 1;
+    for (int l = k; l <= L; l += delta)
+        for (int v = 0; v < n; ++v)
+            if (level[v] == l) cones[l].insert(v);
+    for (int v = 0; v < n; ++v)
+        if (out_degree[v] == 0) cones[level[v]].insert(v);
+    int total = 0;
+    for (int l = 0; l < n_levels; ++l) {
+        group_ptr[l] = total;
+        for (int v : cones[l]) roots[total++] = v;
+    }
+    group_ptr[n_levels] = total;
+    return total;
 }
 
 /* One node, one head of the restricted attention.  q: d_head values; krows[j], vrows[j]: the head's

@@ -45,6 +45,8 @@ def _load():
         lib.orc_level_buckets.argtypes = [c_int, _i32p, c_int, _i32p, _i32p]
         lib.orc_class_order.restype = c_int
         lib.orc_class_order.argtypes = [c_int, _i32p, c_int, _i32p, _i32p, c_int, _i32p, _i32p]
+        lib.orc_partition_roots.restype = c_int
+        lib.orc_partition_roots.argtypes = [c_int, _i32p, _i32p, _i32p, c_int, c_int, c_int, _i32p, _i32p]
         lib.orc_attention.restype = None
         lib.orc_attention.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, _i32p, _i32p, _f64p, _f64p]
         lib.orc_attention_additive.restype = None
@@ -133,6 +135,18 @@ def class_order(seq, seg_ptr, nbr_ptr, max_class):
     class_ptr = np.zeros((n_seg, max_class + 1), np.int32)
     _load().orc_class_order(n, _i(seq), n_seg, _i(seg_ptr), _i(nbr_ptr), max_class, _i(perm), _i(class_ptr))
     return perm, class_ptr
+
+
+def partition_roots(row_ptr, col_idx, level, k, delta):
+    """Algorithm 1: roots of the partition's cones, grouped by level.  Returns (roots, group_ptr[n_levels+1])."""
+    row_ptr, col_idx, level = _i32(row_ptr), _i32(col_idx), _i32(level)
+    n = level.shape[0]
+    n_levels = int(level.max()) + 1
+    roots = np.zeros(n, np.int32)
+    group_ptr = np.zeros(n_levels + 1, np.int32)
+    m = _load().orc_partition_roots(n, _i(row_ptr), _i(col_idx), _i(level), n_levels, int(k), int(delta), _i(roots),
+                                    _i(group_ptr))
+    return roots[:m].copy(), group_ptr
 
 
 def chunk_ptr(n, chunk):

@@ -478,3 +478,31 @@ def test_additive_attention_closed_forms():
     z = 3.0 + np.exp(-1.0)
     assert np.allclose(al[1:, 0], [3.0 / z, np.exp(-1.0) / z], atol=1e-15)
     assert np.allclose(O2[1], (3.0 / z) * V2[1] + (np.exp(-1.0) / z) * V2[0], atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- Algorithm 1 (graph partition)
+
+def test_partition_roots_match_hand_worked_fixture():
+    fanins, level, _ = _read_golden()
+    rp, ci = csr_from_fanins(fanins)
+    for (k, delta), want in (((2, 1), {1: [8], 2: [5], 3: [6, 7]}), ((1, 2), {1: [3, 4, 8], 3: [6, 7]}),
+                             ((3, 2), {1: [8], 3: [6, 7]})):
+        roots, gptr = orc.partition_roots(rp, ci, level, k, delta)
+        got = {l: roots[gptr[l]:gptr[l + 1]].tolist() for l in range(len(gptr) - 1) if gptr[l + 1] > gptr[l]}
+        assert got == want, (k, delta)
+
+
+def test_partition_roots_by_vectorised_selection():
+    rng = np.random.default_rng(77)
+    fanins = random_dag(rng, 10, 600, window=15)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    n = len(fanins)
+    out_degree = np.bincount(ci, minlength=n)
+    for k, delta in ((8, 6), (3, 2), (2, 1), (50, 1)):
+        on_stride = (level >= k) & ((level - k) % delta == 0)
+        sel = np.nonzero(on_stride | (out_degree == 0))[0]
+        want = sel[np.lexsort((sel, level[sel]))]
+        roots, gptr = orc.partition_roots(rp, ci, level, k, delta)
+        assert (roots == want).all()
+        assert (gptr == np.concatenate([[0], np.cumsum(np.bincount(level[want], minlength=level.max() + 1))])).all()
