@@ -140,6 +140,19 @@ dg4_status dg4_graph_info(const dg4_graph* g, dg4_graph_info_t* out);
 dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, int32_t* host_dst, int64_t capacity,
                             int64_t* n_written);
 
+/*
+ * Algorithm 1 (graph partition): the roots whose cones the partition collects, for cone depth k = the hops the
+ * handle was created with and stride delta.  Roots are the nodes on levels k, k + delta, ... and the nodes
+ * without fan-out (added to the group of their own level; a node that qualifies both ways appears once),
+ * grouped by level and ordered by id inside a level.  The cone of a root r is its list in DG4_ARR_NBR_IDX.
+ *   roots      device, capacity n_nodes int32; receives the root ids
+ *   group_ptr  device, n_levels + 1 int32; group_ptr[l] = number of roots on levels below l
+ *   n_roots    host; receives the number of roots
+ * The graph's device must be current.  Allocates scratch and synchronises (a graph-prep call, not a forward call).
+ */
+dg4_status dg4_graph_partition(const dg4_graph* g, int32_t delta, int32_t* roots, int32_t* group_ptr,
+                               int64_t* n_roots);
+
 /* Waits for the device to go idle and reads the handle's status word: DG4_OK, or DG4_ERR_TIMEOUT if a bounded
  * device-side wait of an earlier forward call ran out (that call's output is then incomplete). */
 dg4_status dg4_graph_poll_status(const dg4_graph* g, int32_t* out);

@@ -39,7 +39,7 @@ EXPORTS = [
     "dg4_graph_info", "dg4_graph_export", "dg4_graph_poll_status", "dg4_graph_device_array", "dg4_qkv_project", "dg4_sparse_attn_fwd",
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
-    "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd",
+    "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
 ]
 
 
@@ -98,6 +98,8 @@ def load():
     lib.dg4_graph_info.argtypes = [vp, ctypes.POINTER(dg4_graph_info_t)]
     lib.dg4_graph_export.restype = ctypes.c_int
     lib.dg4_graph_export.argtypes = [vp, ctypes.c_int, i32p, i64, ctypes.POINTER(i64)]
+    lib.dg4_graph_partition.restype = ctypes.c_int
+    lib.dg4_graph_partition.argtypes = [vp, ctypes.c_int32, vp, vp, ctypes.POINTER(i64)]
     lib.dg4_graph_poll_status.restype = ctypes.c_int
     lib.dg4_graph_poll_status.argtypes = [vp, i32p]
     lib.dg4_graph_device_array.restype = vp
@@ -302,3 +304,13 @@ def dg4_sparse_attn_additive_fwd(g: Graph, dsc: dg4_desc, S_dst, S_src, negative
     assert S_dst.is_contiguous() and S_src.is_contiguous()
     _check(load().dg4_sparse_attn_additive_fwd(g.handle, ctypes.byref(dsc), _ptr(S_dst), _ptr(S_src),
                                                float(negative_slope), _ptr(V), _ld(V), _ptr(O), _ld(O), _stream(stream)))
+
+
+def dg4_graph_partition(g: Graph, delta: int):
+    """Algorithm 1: returns (roots, group_ptr) as CUDA int32 tensors (roots trimmed to their number)."""
+    import torch
+    roots = torch.empty(g.n, dtype=torch.int32, device="cuda")
+    group_ptr = torch.empty(int(g.info.n_levels) + 1, dtype=torch.int32, device="cuda")
+    m = ctypes.c_int64(0)
+    _check(load().dg4_graph_partition(g.handle, int(delta), _ptr(roots), _ptr(group_ptr), ctypes.byref(m)))
+    return roots[: m.value], group_ptr

@@ -491,3 +491,16 @@ def test_wide_cone_layers_parallel_and_level_launches():
     with pytest.raises(dg4.Dg4Error) as e:
         dg4.dg4_layer_fwd_levelised(gr, dg4.desc(heads, dg4.DG4_BF16, 0.25), h, dev_bf16(wqb), dev_bf16(wob), ws)
     assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("hops,delta", [(8, 6), (3, 2), (2, 1), (1, 1)])
+def test_graph_partition_roots_match_checker(hops, delta):
+    rng = np.random.default_rng(hops * 10 + delta)
+    for fanins in (random_dag(rng, 20, 5000, window=25), binary_in_tree(9)[0], [[] for _ in range(7)]):
+        rp, ci = csr_from_fanins(fanins)
+        level = levels_of(fanins)
+        g = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+        roots, gptr = dg4.dg4_graph_partition(g, delta)
+        want_roots, want_gptr = orc.partition_roots(rp, ci, level, hops, delta)
+        assert (roots.cpu().numpy() == want_roots).all()
+        assert (gptr.cpu().numpy() == want_gptr).all()
