@@ -504,3 +504,30 @@ def test_graph_partition_roots_match_checker(hops, delta):
         want_roots, want_gptr = orc.partition_roots(rp, ci, level, hops, delta)
         assert (roots.cpu().numpy() == want_roots).all()
         assert (gptr.cpu().numpy() == want_gptr).all()
+
+
+def test_levelised_layers_with_empty_levels():
+    # any strictly increasing layering is accepted; here two of every three levels are empty
+    rng = np.random.default_rng(99)
+    fanins = random_dag(rng, 50, 3000, window=100)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins) * 3 + 1
+    n = len(fanins)
+    gr = dg4.dg4_graph_create(rp, ci, level, 2, 0)
+    xb = synth.normal_bf16_bits(11, 1, (n, 128), 1.0)
+    weights = [bf16_weights(synth.normal_f32(11, 10 + l, (384, 128), 0.05)) +
+               bf16_weights(synth.normal_f32(11, 20 + l, (128, 128), 0.05)) for l in range(3)]
+    dsc = dg4.desc(8, dg4.DG4_BF16, 0.25, residual=True)
+    ws = torch.empty(dg4.dg4_layers_workspace_bytes(gr, dsc, 3), dtype=torch.uint8, device="cuda")
+    h = dev_bf16(xb).clone()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dev_bf16(w_[0]) for w_ in weights], [dev_bf16(w_[2]) for w_ in weights],
+                                 ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    lptr, lnodes = orc.level_buckets(level)
+    want = f64_of_bits(xb)
+    for (_, wq, _, wo) in weights:
+        want = orc.layer_levelised(want, wq, wo, ptr, idx, lptr, lnodes, 8, 0.25, residual=True, rounding="bf16")
+    assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
