@@ -4,7 +4,9 @@
 // Q|K|V of every node from the layer's input once -- a node's own query, key and value always come from
 // its row as it was at the start of the layer -- and then, level by level, runs the attention for that
 // level's nodes, writes their new rows, and refreshes their K|V rows so that higher levels gather the
-// updated ones.
+// updated ones.  By default that walk is one persistent kernel (dg4_levelised.cu), which can also run several
+// layers as a wavefront; with DG4_FLAG_LEVEL_LAUNCHES it is one group of launches per level (kept for
+// comparison, and the only levelised driver for cones wider than two hops).
 
 #include "dg4_internal.h"
 
