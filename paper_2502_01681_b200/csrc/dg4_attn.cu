@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(d
 // Additive (GAT-style) scores: e = LeakyReLU(S_src[u, head] + S_dst[v, head]) from node-level scalars, so a
 // neighbour costs one value row and one 4-byte scalar per head instead of a key row; same persistent walk.
 template <bool BF16, int LPH, int MAXN>
-__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive_kernel(dg4i_attn_args a) {
+__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive_kernel(dg4i_attn_args a, dg4i_attn_more x) {
     constexpr int G = BF16 ? 16 : 32;
     constexpr int EPP = Elem<BF16>::kPerPiece;
     constexpr int ES = BF16 ? 2 : 4;
@@ -122,12 +122,12 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive
             ss[j] = 0.f;
             if (j < cnt) {
                 vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
-                if (cnt > 1) ss[j] = __ldg(a.s_src + (size_t)u[j] * a.heads + head);
+                if (cnt > 1) ss[j] = __ldg(x.s_src + (size_t)u[j] * a.heads + head);
             }
         }
-        const float sd = cnt > 1 ? __ldg(a.s_dst + (size_t)v * a.heads + head) : 0.f;
+        const float sd = cnt > 1 ? __ldg(x.s_dst + (size_t)v * a.heads + head) : 0.f;
         float acc[EPP];
-        attend_additive<BF16, MAXN>(sd, ss, vq, cnt, a.slope, acc);
+        attend_additive<BF16, MAXN>(sd, ss, vq, cnt, x.slope, acc);
         st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
     }
 }
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive
 // matching weighted sum of its value piece; the halves are merged at the end.  Four neighbours per half are in
 // flight at a time.
 template <bool BF16, int LPH>
-__global__ void __launch_bounds__(256) sparse_attn_wide_kernel(dg4i_attn_args a) {
+__global__ void __launch_bounds__(256) sparse_attn_wide_kernel(dg4i_attn_args a, dg4i_attn_more x) {
     constexpr int G = BF16 ? 16 : 32;              // lanes per row
     constexpr int HALVES = 32 / G;                 // neighbours a warp handles side by side
     constexpr int EPP = Elem<BF16>::kPerPiece;
@@ -153,14 +153,14 @@ __global__ void __launch_bounds__(256) sparse_attn_wide_kernel(dg4i_attn_args a)
     const float c = a.scale * 1.4426950408889634f;
     for (int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); slot < a.count; slot += warps) {
         const int v = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
-        const int beg = a.nbr_ptr[v];
-        const int cnt = a.nbr_ptr[v + 1] - beg;
+        const int beg = x.nbr_ptr[v];
+        const int cnt = x.nbr_ptr[v + 1] - beg;
         const Piece qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
         float m = -INFINITY, z = 0.f, acc[EPP];
 #pragma unroll
         for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
         for (int base = 0; base < cnt; base += 32) {
-            const int my_u = (base + lane < cnt) ? a.nbr_idx[beg + base + lane] : -1;
+            const int my_u = (base + lane < cnt) ? x.nbr_idx[beg + base + lane] : -1;
             const int chunk = cnt - base < 32 ? cnt - base : 32;
             for (int t = 0; t < chunk; t += HALVES * UN) {
                 Piece kq[UN], vq[UN];
@@ -224,28 +224,28 @@ __global__ void __launch_bounds__(256) sparse_attn_wide_kernel(dg4i_attn_args a)
 }
 
 template <bool BF16, int LPH>
-dg4_status launch_wide(const dg4i_attn_args& a, cudaStream_t st) {
+dg4_status launch_wide(const dg4i_attn_args& a, const dg4i_attn_more& x, cudaStream_t st) {
     int dev = 0, sms = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
     DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int64_t needed = ((int64_t)a.count + 7) / 8;
     const int64_t resident = (int64_t)sms * 4;
-    sparse_attn_wide_kernel<BF16, LPH><<<(unsigned)(needed < resident ? needed : resident), 256, 0, st>>>(a);
+    sparse_attn_wide_kernel<BF16, LPH><<<(unsigned)(needed < resident ? needed : resident), 256, 0, st>>>(a, x);
     dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
 
 template <bool BF16>
-dg4_status launch_wide_heads(const dg4i_attn_args& a, cudaStream_t st) {
+dg4_status launch_wide_heads(const dg4i_attn_args& a, const dg4i_attn_more& x, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     switch (G / a.heads) {
-        case 1: return launch_wide<BF16, 1>(a, st);
-        case 2: return launch_wide<BF16, 2>(a, st);
-        case 4: return launch_wide<BF16, 4>(a, st);
-        case 8: return launch_wide<BF16, 8>(a, st);
-        case 16: return launch_wide<BF16, 16>(a, st);
-        case 32: if (G == 32) return launch_wide<BF16, (G == 32 ? 32 : 16)>(a, st);
+        case 1: return launch_wide<BF16, 1>(a, x, st);
+        case 2: return launch_wide<BF16, 2>(a, x, st);
+        case 4: return launch_wide<BF16, 4>(a, x, st);
+        case 8: return launch_wide<BF16, 8>(a, x, st);
+        case 16: return launch_wide<BF16, 16>(a, x, st);
+        case 32: if (G == 32) return launch_wide<BF16, (G == 32 ? 32 : 16)>(a, x, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
 }
@@ -253,10 +253,9 @@ dg4_status launch_wide_heads(const dg4i_attn_args& a, cudaStream_t st) {
 struct LaunchShape { int sm_count = 0; int blocks_per_sm = 0; };
 
 template <bool BF16, int LPH, int MAXN, bool ADDITIVE>
-dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
+dg4_status launch_one(const dg4i_attn_args& a, const dg4i_attn_more* x, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     const int threads = 256;
-    auto kern = ADDITIVE ? sparse_attn_additive_kernel<BF16, LPH, MAXN> : sparse_attn_kernel<BF16, LPH, MAXN>;
     static LaunchShape shape[64];
     int dev = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
@@ -264,7 +263,8 @@ dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
     if (shape[dev].sm_count == 0) {
         int sms = 0, per_sm = 0;
         DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, 0));
+        if (ADDITIVE) DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sparse_attn_additive_kernel<BF16, LPH, MAXN>, threads, 0));
+        else DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sparse_attn_kernel<BF16, LPH, MAXN>, threads, 0));
         shape[dev].blocks_per_sm = per_sm > 0 ? per_sm : 1;
         shape[dev].sm_count = sms;
     }
@@ -272,22 +272,23 @@ dg4_status launch_one(const dg4i_attn_args& a, cudaStream_t st) {
     const int64_t needed = ((int64_t)a.count + nodes_per_block - 1) / nodes_per_block;
     const int64_t resident = (int64_t)shape[dev].sm_count * shape[dev].blocks_per_sm;
     const unsigned blocks = (unsigned)(needed < resident ? needed : resident);
-    kern<<<blocks, threads, 0, st>>>(a);
+    if (ADDITIVE) sparse_attn_additive_kernel<BF16, LPH, MAXN><<<blocks, threads, 0, st>>>(a, *x);
+    else sparse_attn_kernel<BF16, LPH, MAXN><<<blocks, threads, 0, st>>>(a);
     dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
 
 template <bool BF16, int MAXN, bool ADDITIVE>
-dg4_status launch_for_heads(const dg4i_attn_args& a, cudaStream_t st) {
+dg4_status launch_for_heads(const dg4i_attn_args& a, const dg4i_attn_more* x, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     switch (G / a.heads) {
-        case 1: return launch_one<BF16, 1, MAXN, ADDITIVE>(a, st);
-        case 2: return launch_one<BF16, 2, MAXN, ADDITIVE>(a, st);
-        case 4: return launch_one<BF16, 4, MAXN, ADDITIVE>(a, st);
-        case 8: return launch_one<BF16, 8, MAXN, ADDITIVE>(a, st);
-        case 16: return launch_one<BF16, 16, MAXN, ADDITIVE>(a, st);
-        case 32: if (G == 32) return launch_one<BF16, (G == 32 ? 32 : 16), MAXN, ADDITIVE>(a, st);
+        case 1: return launch_one<BF16, 1, MAXN, ADDITIVE>(a, x, st);
+        case 2: return launch_one<BF16, 2, MAXN, ADDITIVE>(a, x, st);
+        case 4: return launch_one<BF16, 4, MAXN, ADDITIVE>(a, x, st);
+        case 8: return launch_one<BF16, 8, MAXN, ADDITIVE>(a, x, st);
+        case 16: return launch_one<BF16, 16, MAXN, ADDITIVE>(a, x, st);
+        case 32: if (G == 32) return launch_one<BF16, (G == 32 ? 32 : 16), MAXN, ADDITIVE>(a, x, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
 }
@@ -296,7 +297,7 @@ dg4_status launch_for_heads(const dg4i_attn_args& a, cudaStream_t st) {
 
 namespace {
 template <bool ADDITIVE>
-dg4_status attn_dispatch(const dg4i_attn_args& a, cudaStream_t st) {
+dg4_status attn_dispatch(const dg4i_attn_args& a, const dg4i_attn_more* x, cudaStream_t st) {
     if (a.count <= 0) return DG4_OK;
     const bool bf16 = a.dtype == DG4_BF16;
     const int G = bf16 ? 16 : 32;
@@ -304,12 +305,17 @@ dg4_status attn_dispatch(const dg4i_attn_args& a, cudaStream_t st) {
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must divide %d", a.heads, G);
     if (a.max_nbr > 7) {
         if (ADDITIVE) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the additive-score variant supports cones of at most two hops");
-        return bf16 ? launch_wide_heads<true>(a, st) : launch_wide_heads<false>(a, st);
+        if (!x || !x->nbr_ptr || !x->nbr_idx) DG4_FAIL(DG4_ERR_INVALID_ARG, "wider cones need the CSR neighbour lists");
+        return bf16 ? launch_wide_heads<true>(a, *x, st) : launch_wide_heads<false>(a, *x, st);
     }
-    if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3, ADDITIVE>(a, st) : launch_for_heads<false, 3, ADDITIVE>(a, st);
-    return bf16 ? launch_for_heads<true, 7, ADDITIVE>(a, st) : launch_for_heads<false, 7, ADDITIVE>(a, st);
+    if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3, ADDITIVE>(a, x, st) : launch_for_heads<false, 3, ADDITIVE>(a, x, st);
+    return bf16 ? launch_for_heads<true, 7, ADDITIVE>(a, x, st) : launch_for_heads<false, 7, ADDITIVE>(a, x, st);
 }
 }  // namespace
 
-dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st) { return attn_dispatch<false>(a, st); }
-dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, cudaStream_t st) { return attn_dispatch<true>(a, st); }
+dg4_status dg4i_attn_launch(const dg4i_attn_args& a, const dg4i_attn_more* more, cudaStream_t st) {
+    return attn_dispatch<false>(a, more, st);
+}
+dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, const dg4i_attn_more& more, cudaStream_t st) {
+    return attn_dispatch<true>(a, &more, st);
+}

@@ -140,7 +140,24 @@ __device__ __forceinline__ void attend(const Piece& qp, const Piece* kq, const P
         s[j] = (j < cnt) ? dot * c : -INFINITY;
         m = fmaxf(m, s[j]);
     }
-    softmax_weighted_sum<BF16, MAXN>(s, m, cnt, vq, acc);
+    constexpr int EPP = Elem<BF16>::kPerPiece;
+    float z = 0.f;
+#pragma unroll
+    for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXN; ++j) {
+        if (j < cnt) {
+            float p = fast_exp2(s[j] - m);
+            z += p;
+            float vf[EPP];
+            Elem<BF16>::unpack(vq[j], vf);
+#pragma unroll
+            for (int i = 0; i < EPP; ++i) acc[i] = fmaf(p, vf[i], acc[i]);
+        }
+    }
+    const float inv = fast_rcp(z);
+#pragma unroll
+    for (int i = 0; i < EPP; ++i) acc[i] *= inv;
 }
 
 // Additive-score variant: this lane's head has the node-level scalars s_dst (of the destination) and s_src[j]

@@ -84,22 +84,26 @@ struct dg4i_attn_args {
     const void* V; int64_t ldv;
     void* O; int64_t ldo;
     const int32_t* nbr_pad;     // [n, max_nbr + 1] fixed-width neighbour table (cones of at most two hops)
-    const int32_t* nbr_ptr = nullptr;   // CSR lists, used for wider cones
-    const int32_t* nbr_idx = nullptr;
     const int32_t* node_list;   // nullable: node ids to process; else ids first..first+count-1
     int32_t first;
     int32_t count;
     int32_t heads;
-    int32_t max_nbr;            // 3 or 7
+    int32_t max_nbr;            // 3 or 7; larger for cones wider than two hops
     int32_t dtype;
     float scale;
-    // additive-score variant (dg4i_attn_additive_launch): node-level scalars [n, heads] fp32; Q and K unused
-    const float* s_dst = nullptr;
+};
+// What the less common kernels need on top (kept out of the struct above: the main kernel compiles to fewer
+// registers and instructions with the smaller parameter block).
+struct dg4i_attn_more {
+    const int32_t* nbr_ptr = nullptr;   // CSR lists, used for wider cones
+    const int32_t* nbr_idx = nullptr;
+    const float* s_dst = nullptr;       // additive-score variant: node-level scalars [n, heads] fp32
     const float* s_src = nullptr;
     float slope = 0.f;
 };
-dg4_status dg4i_attn_launch(const dg4i_attn_args& a, cudaStream_t st);
-dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, cudaStream_t st);
+// `more` may be null for graphs with cones of at most two hops
+dg4_status dg4i_attn_launch(const dg4i_attn_args& a, const dg4i_attn_more* more, cudaStream_t st);
+dg4_status dg4i_attn_additive_launch(const dg4i_attn_args& a, const dg4i_attn_more& more, cudaStream_t st);
 
 // Y[r, 0:n_out] = A[r, 0:128] * W[0:n_out, 0:128]^T (+ R[r, :]) for rows r of a list (or 0..rows-1).
 // Output column block j (of 128) goes to out[j] with leading dimension ldo[j].

@@ -70,11 +70,17 @@ Workspace carve(void* ws, int64_t n) {
     return w;
 }
 
+dg4i_attn_more attn_more(const dg4_graph* g) {
+    dg4i_attn_more m;
+    m.nbr_ptr = g->nbr_ptr; m.nbr_idx = g->nbr_idx;
+    return m;
+}
+
 dg4i_attn_args attn_args(const dg4_graph* g, const dg4_desc* d, const void* Q, int64_t ldq, const void* K,
                          int64_t ldk, const void* V, int64_t ldv, void* O, int64_t ldo) {
     dg4i_attn_args a;
     a.Q = Q; a.ldq = ldq; a.K = K; a.ldk = ldk; a.V = V; a.ldv = ldv; a.O = O; a.ldo = ldo;
-    a.nbr_pad = g->nbr_pad; a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.nbr_pad = g->nbr_pad; a.node_list = nullptr; a.first = 0; a.count = g->n;
     a.heads = d->heads; a.max_nbr = g->max_class; a.dtype = d->dtype; a.scale = d->scale;
     return a;
 }
@@ -139,7 +145,8 @@ extern "C" dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* de
     CHECK(check_tensor("V", V, ldv, es, 128));
     CHECK(check_tensor("O", O, ldo, es, 128));
     if (O == K || O == V) DG4_FAIL(DG4_ERR_INVALID_ARG, "O must not alias K or V");
-    return dg4i_attn_launch(attn_args(g, desc, Q, ldq, K, ldk, V, ldv, O, ldo), (cudaStream_t)stream);
+    const dg4i_attn_more more = attn_more(g);
+    return dg4i_attn_launch(attn_args(g, desc, Q, ldq, K, ldk, V, ldv, O, ldo), &more, (cudaStream_t)stream);
 }
 
 extern "C" dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4_desc* desc, const float* S_dst,
@@ -155,8 +162,9 @@ extern "C" dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4
     CHECK(check_tensor("O", O, ldo, es, 128));
     if (O == V) DG4_FAIL(DG4_ERR_INVALID_ARG, "O must not alias V");
     dg4i_attn_args a = attn_args(g, desc, nullptr, 0, nullptr, 0, V, ldv, O, ldo);
-    a.s_dst = S_dst; a.s_src = S_src; a.slope = negative_slope;
-    return dg4i_attn_additive_launch(a, (cudaStream_t)stream);
+    dg4i_attn_more more = attn_more(g);
+    more.s_dst = S_dst; more.s_src = S_src; more.slope = negative_slope;
+    return dg4i_attn_additive_launch(a, more, (cudaStream_t)stream);
 }
 
 extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, const void* O, int64_t ldo,
@@ -215,7 +223,8 @@ extern "C" dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc*
     p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
 
-    CHECK(dg4i_attn_launch(attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128), st));
+    const dg4i_attn_more more = attn_more(g);
+    CHECK(dg4i_attn_launch(attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128), &more, st));
 
     dg4i_proj_args o;
     o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
@@ -260,7 +269,8 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
         if (count <= 0) continue;
         dg4i_attn_args a = attn_args(g, desc, w.Q, 128, w.KV, 256, w.KV + 128, 256, w.O, 128);
         a.node_list = g->level_nodes; a.first = first; a.count = count;
-        CHECK(dg4i_attn_launch(a, st));
+        const dg4i_attn_more more = attn_more(g);
+        CHECK(dg4i_attn_launch(a, &more, st));
 
         dg4i_proj_args o;
         o.A = w.O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;

@@ -97,9 +97,11 @@ extern "C" dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg
 
     dg4i_attn_args a;
     a.Q = Q; a.ldq = 128; a.K = KV; a.ldk = 256; a.V = KV + 128; a.ldv = 256; a.O = O; a.ldo = 128;
-    a.nbr_pad = g->nbr_pad; a.nbr_ptr = g->nbr_ptr; a.nbr_idx = g->nbr_idx; a.node_list = nullptr; a.first = 0; a.count = g->n;
+    a.nbr_pad = g->nbr_pad; a.node_list = nullptr; a.first = 0; a.count = g->n;
     a.heads = desc->heads; a.max_nbr = g->max_class; a.dtype = DG4_BF16; a.scale = desc->scale;
-    if ((s = dg4i_attn_launch(a, st)) != DG4_OK) return s;
+    dg4i_attn_more more;
+    more.nbr_ptr = g->nbr_ptr; more.nbr_idx = g->nbr_idx;
+    if ((s = dg4i_attn_launch(a, &more, st)) != DG4_OK) return s;
 
     dg4i_proj_args o;
     o.A = O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
