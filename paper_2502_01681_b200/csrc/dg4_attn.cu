@@ -16,7 +16,7 @@
 
 // resident blocks per SM the compiler must allow for (caps registers per thread)
 #ifndef DG4_ATTN_MIN_BLOCKS
-#define DG4_ATTN_MIN_BLOCKS 2
+#define DG4_ATTN_MIN_BLOCKS 3
 #endif
 
 namespace {
@@ -63,15 +63,14 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(d
         u[0] = v;
 #pragma unroll
         for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(mask, pad, grp_base + j);
+        // The filler entries of the table repeat v, so every slot names a valid row: all 2 * MAXN + 1 loads are
+        // issued without predicates (slots beyond cnt re-read the node's own row, a cache hit), which saves the
+        // branches and lets the kernel fit three blocks per SM; the arithmetic below still stops at cnt.
+        qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
 #pragma unroll
-        for (int j = 0; j < MAXN; ++j)
-            if (j < cnt) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
-        if (cnt > 1) {
-            qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
+        for (int j = 0; j < MAXN; ++j) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
 #pragma unroll
-            for (int j = 0; j < MAXN; ++j)
-                if (j < cnt) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
-        }
+        for (int j = 0; j < MAXN; ++j) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
         float acc[EPP];
         attend<BF16, LPH, MAXN>(qp, kq, vq, cnt, a.scale, mask, acc);
         st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
