@@ -15,6 +15,9 @@
 #include "dg4_attn_core.cuh"
 
 // resident blocks per SM the compiler must allow for (caps registers per thread)
+#ifndef DG4_ATTN_THREADS
+#define DG4_ATTN_THREADS 256
+#endif
 #ifndef DG4_ATTN_MIN_BLOCKS
 #define DG4_ATTN_MIN_BLOCKS 3
 #endif
@@ -29,7 +32,7 @@ using namespace attn;
 // fixed-width neighbour entry of the NEXT node is fetched while the current node's rows are in flight, which
 // takes the index lookup off the per-node dependency chain (one memory round trip per node instead of three).
 template <bool BF16, int LPH, int MAXN>
-__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(dg4i_attn_args a) {
+__global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(dg4i_attn_args a) {
     constexpr int G = BF16 ? 16 : 32;              // lanes per node
     constexpr int EPP = Elem<BF16>::kPerPiece;     // elements per 16-byte piece
     constexpr int ES = BF16 ? 2 : 4;
@@ -80,7 +83,7 @@ __global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_kernel(d
 // Additive (GAT-style) scores: e = LeakyReLU(S_src[u, head] + S_dst[v, head]) from node-level scalars, so a
 // neighbour costs one value row and one 4-byte scalar per head instead of a key row; same persistent walk.
 template <bool BF16, int LPH, int MAXN>
-__global__ void __launch_bounds__(256, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive_kernel(dg4i_attn_args a, dg4i_attn_more x) {
+__global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_attn_additive_kernel(dg4i_attn_args a, dg4i_attn_more x) {
     constexpr int G = BF16 ? 16 : 32;
     constexpr int EPP = Elem<BF16>::kPerPiece;
     constexpr int ES = BF16 ? 2 : 4;
@@ -254,7 +257,7 @@ struct LaunchShape { int sm_count = 0; int blocks_per_sm = 0; };
 template <bool BF16, int LPH, int MAXN, bool ADDITIVE>
 dg4_status launch_one(const dg4i_attn_args& a, const dg4i_attn_more* x, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
-    const int threads = 256;
+    const int threads = DG4_ATTN_THREADS;
     static LaunchShape shape[64];
     int dev = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
