@@ -404,7 +404,7 @@ def run_ours(args, w):
 
 # DRAM bytes (read + write) of one sparse_attn_kernel launch on the full workload, from the ncu capture
 # summarised under profiles/; None while no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = 14.19e9   # 3.547 GB at a quarter of the nodes (profiles/), scaled by the node count
+TRAFFIC_BYTES_PER_LAUNCH = 16.60e9   # 4.149 GB at a quarter of the nodes (profiles/), scaled by the node count
 
 
 def main():
