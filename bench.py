@@ -9,6 +9,7 @@ gates, log-uniform locality window, 2-hop cones, d = 128, 8 heads, bf16):
 The metric is AIG nodes per second per sparse-attention layer: nodes x layer passes / time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--shrink S]
+    python bench.py --per-config [--configs 1,2,3] [--cpu-only --cpu-threads T]    (a table, see run_per_config)
 
 With N > 1 (under torchrun) every rank runs its own circuit of the same shape (weak scaling, no collective
 on the data path); the reported time is the maximum over ranks.
@@ -402,6 +403,149 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------------
+# --per-config: the attention step on each of the five workloads (a table, not the benchmark line)
+# --------------------------------------------------------------------------------------------------
+
+def run_per_config(args):
+    """Times the fused sparse-attention kernel on each workload: 20 repetitions back to back (warm L2) and 20
+    with a 512 MB scratch write in between (cold L2), median and minimum; the layer and the levelised mode
+    where the workload has them; the CPU checker's attention on the same circuit beside it.  Prints a
+    markdown table."""
+    cfgs = [int(c) for c in args.configs.split(",")]
+    rows = []
+    if not args.cpu_only:
+        import torch
+        from paper_2502_01681_b200 import dg4
+        if not torch.cuda.is_available():
+            raise RuntimeError("bench.py needs a CUDA device: the product has no CPU path")
+        torch.cuda.set_device(0)
+        stream = torch.cuda.current_stream()
+        scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    from paper_2502_01681_b200 import synth
+    peak, peak_kind = measured_hbm_peak()
+
+    def timed(fn, reps, between=None):
+        import torch
+        ts = []
+        for _ in range(reps):
+            if between is not None:
+                between()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts)), float(np.min(ts))
+
+    for cfg in cfgs:
+        w = synth.workload(cfg)
+        g = w.graph()
+        n = g.n
+        r = {"cfg": cfg, "name": w.name, "n": n, "dtype": w.dtype}
+        esz = 4 if w.dtype == "f32" else 2
+        if not args.cpu_only:
+            import torch
+            t0 = time.perf_counter()
+            gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, 0)
+            torch.cuda.synchronize()
+            r["create_ms"] = (time.perf_counter() - t0) * 1e3
+            r["prep_ms"] = timed(lambda: dg4.dg4_graph_rebuild(gr), 5)[0]
+            info = gr.info
+            r["n_nbr"], r["levels"] = int(info.n_nbr), int(info.n_levels)
+            tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+            dsc = dg4.desc(w.heads, dg4.DG4_F32 if w.dtype == "f32" else dg4.DG4_BF16, w.scale, residual=w.residual)
+
+            def dev(bits):
+                return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+            if w.with_projection:
+                x = dev(w.x_bf16_bits())
+                wq = [dev(synth.f32_to_bf16_bits(w.w_qkv_f32(l))) for l in range(w.layers)]
+                wo = [dev(synth.f32_to_bf16_bits(w.w_o_f32(l))) for l in range(w.layers)]
+                q, k, v = (torch.empty_like(x) for _ in range(3))
+                dg4.dg4_qkv_project(gr, dsc, x, wq[0], q, k, v)
+            elif w.dtype == "f32":
+                q, k, v = (torch.from_numpy(t).cuda() for t in w.qkv_f32())
+            else:
+                q, k, v = (dev(t) for t in w.qkv_bf16_bits())
+            o = torch.empty_like(q)
+            attn = lambda: dg4.dg4_sparse_attn_fwd(gr, dsc, q, k, v, o)
+            for _ in range(3):
+                attn()
+            r["warm"] = timed(attn, 20)
+            r["cold"] = timed(attn, 20, between=lambda: scratch.zero_())
+            r["bytes"] = (2 * w.d * esz + 4) * n + (2 * w.d * esz + 4) * r["n_nbr"]
+            if w.with_projection:
+                ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc),
+                                     dg4.dg4_layers_workspace_bytes(gr, dsc, w.layers)),
+                                 dtype=torch.uint8, device="cuda")
+                status = torch.zeros(1, dtype=torch.int32, device="cuda")
+                h = torch.empty_like(x)
+                if "parallel" in w.modes:
+                    par = lambda: dg4.dg4_layer_fwd_parallel(gr, dsc, x, wq[0], wo[0], h, ws)
+                    for _ in range(3):
+                        par()
+                    r["layer"] = timed(par, 20)
+                if "levelised" in w.modes:
+                    lev = lambda: dg4.dg4_layers_fwd_levelised(gr, dsc, h, wq, wo, ws, status)
+                    h.copy_(x)
+                    lev()
+                    r["lev"] = timed(lev, 5, between=lambda: h.copy_(x))
+                    dsl = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, level_launches=True)
+                    r["lev_launches"] = timed(lambda: dg4.dg4_layer_fwd_levelised(gr, dsl, h, wq[0], wo[0], ws, status),
+                                              2, between=lambda: h.copy_(x))
+                    assert int(status.item()) == 0
+                del ws, h
+            dg4.dg4_graph_destroy(gr)
+            del q, k, v, o
+            torch.cuda.empty_cache()
+        if not args.no_cpu_baseline:
+            from oracle import oracle as orc
+            wc = synth.workload(cfg, 10) if cfg == 5 else w       # the 10M-node circuit: a tenth of it
+            gc = wc.graph() if cfg == 5 else g
+            ptr, idx = orc.neighbourhood(gc.row_ptr, gc.col_idx, w.hops)
+            if w.dtype == "f32":
+                qc, kc, vc = (t.astype(np.float64) for t in wc.qkv_f32())
+            else:
+                qc, kc, vc = (synth.bf16_bits_to_f32(t).astype(np.float64) for t in wc.qkv_bf16_bits())
+            t0 = time.perf_counter()
+            orc.attention(qc, kc, vc, ptr, idx, w.heads, w.scale)
+            r["cpu_s"], r["cpu_n"], r["cpu_threads"] = time.perf_counter() - t0, gc.n, orc.num_threads()
+        rows.append(r)
+
+    print(f"HBM peak used: {peak:.0f} GB/s ({peak_kind}); nominal 8000 GB/s.  Times in ms as median / minimum.")
+    if not args.cpu_only:
+        print("\n| cfg | nodes | neighbour entries | levels | graph create (host+device) | device prep | attention, warm L2 "
+              "| attention, cold L2 | nodes/s (cold median) | algorithmic GB/s | of measured | of 8000 |")
+        print("|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|")
+        for r in rows:
+            t = r["cold"][0] * 1e-3
+            gbs = r["bytes"] / t / 1e9
+            print(f"| {r['cfg']} {r['name']} ({r['dtype']}) | {r['n']} | {r['n_nbr']} | {r['levels']} | {r['create_ms']:.2f} "
+                  f"| {r['prep_ms']:.3f} | {r['warm'][0]:.4f} / {r['warm'][1]:.4f} | {r['cold'][0]:.4f} / {r['cold'][1]:.4f} "
+                  f"| {r['n'] / t:.3e} | {gbs:.0f} | {100 * gbs / peak:.0f} % | {100 * gbs / 8000:.0f} % |")
+        print("\n| cfg | parallel layer (QKV + attention + output) | levelised, all layers in one launch | per layer "
+              "| us per wavefront step (levels + layers - 1 steps) | levelised, one layer as per-level launches |")
+        print("|---|---:|---:|---:|---:|---:|")
+        for r in rows:
+            if "layer" in r or "lev" in r:
+                L = synth.workload(r["cfg"]).layers
+                lay = f"{r['layer'][0]:.3f} / {r['layer'][1]:.3f}" if "layer" in r else "-"
+                if "lev" in r:
+                    lev = (f"{r['lev'][0]:.2f} / {r['lev'][1]:.2f} | {r['lev'][0] / L:.2f} "
+                           f"| {1e3 * r['lev'][0] / (r['levels'] + L - 1):.2f} | {r['lev_launches'][0]:.1f}")
+                else:
+                    lev = "- | - | - | -"
+                print(f"| {r['cfg']} | {lay} | {lev} |")
+    if not args.no_cpu_baseline:
+        print("\n| cfg | CPU checker, attention only: nodes | threads | seconds | nodes/s |")
+        print("|---|---:|---:|---:|---:|")
+        for r in rows:
+            print(f"| {r['cfg']} | {r['cpu_n']} | {r['cpu_threads']} | {r['cpu_s']:.3f} | {r['cpu_n'] / r['cpu_s']:.3e} |")
+
+
 # DRAM bytes (read + write) of one sparse_attn_kernel launch on the full workload, from the ncu capture
 # summarised under profiles/; None while no capture of the current kernel exists.
 TRAFFIC_BYTES_PER_LAUNCH = 16.60e9   # 4.149 GB at a quarter of the nodes (profiles/), scaled by the node count
@@ -418,7 +562,18 @@ def main():
     ap.add_argument("--no-levelised", action="store_true",
                     help="profiling only: leave the levelised layers out of the step (the printed value is then "
                          "not a benchmark result)")
+    ap.add_argument("--per-config", action="store_true",
+                    help="time the attention step on each of the five workloads and print a table instead of "
+                         "the benchmark line")
+    ap.add_argument("--configs", default="1,2,3,4,5", help="with --per-config: which workloads")
+    ap.add_argument("--cpu-only", action="store_true", help="with --per-config: only the CPU checker's column")
+    ap.add_argument("--cpu-threads", type=int, default=0, help="with --per-config: OpenMP threads of the CPU checker")
     args = ap.parse_args()
+    if args.cpu_threads > 0:
+        os.environ["OMP_NUM_THREADS"] = str(args.cpu_threads)
+    if args.per_config:
+        run_per_config(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.shrink == 1 else args.warmup
     from paper_2502_01681_b200 import synth
     w = synth.workload(5, args.shrink)
