@@ -21,6 +21,8 @@
  *   orc_attention_additive  the same restricted attention with the additive LeakyReLU score of GAT layers
  *                         (node-level scalars), the form the kernels of Sec. 3.7 aggregate with
  *   orc_project           the dense projections of the Transformer block kept around the attention
+ *   orc_layernorm / orc_ffn   the rest of that block (Sec. 3.5 keeps the original Transformer structure): row
+ *                         normalisation and the position-wise feed-forward sub-layer with residual, post-norm
  *   orc_layer_parallel    QKV projection -> attention -> output projection (+ residual), all nodes at once
  *   orc_layer_levelised   the same layer applied level by level in topological order, each level
  *                         reading the rows already updated for earlier levels (Sec. 1 and Sec. 3.4:
@@ -298,6 +300,53 @@ void orc_layer_parallel(int n, int d, int heads, double scale, const double* X, 
     round_all(O.data(), nd, rounding);
     orc_project(n, d, d, O.data(), W_o, residual ? X : nullptr, H_out);
     round_all(H_out, nd, rounding);
+}
+
+/* Row-wise layer normalisation as in the Transformer block the paper keeps around its attention (Sec. 3.5:
+ * only the attention module is replaced, the rest of the block stays): y = (x - mean) / sqrt(var + eps) * gamma
+ * + beta, mean and (biased) variance over the d features of the row. */
+void orc_layernorm(int n, int d, const double* X, const double* gamma, const double* beta, double eps, double* Y) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < n; ++i) {
+        const double* x = X + (int64_t)i * d;
+        double mean = 0.0;
+        for (int c = 0; c < d; ++c) mean += x[c];
+        mean /= d;
+        double var = 0.0;
+        for (int c = 0; c < d; ++c) var += (x[c] - mean) * (x[c] - mean);
+        var /= d;
+        double rstd = 1.0 / std::sqrt(var + eps);
+        for (int c = 0; c < d; ++c) Y[(int64_t)i * d + c] = (x[c] - mean) * rstd * gamma[c] + beta[c];
+    }
+}
+
+/* Position-wise feed-forward sub-layer of that block, with its residual connection and the normalisation
+ * that follows it (post-norm, as in the original Transformer):
+ *     U = max(0, X W1^T + b1)      W1: [d_ff, d]
+ *     Y = LayerNorm(X + U W2^T + b2)   W2: [d, d_ff]
+ * rounding: 0 none; 1 = U (the hidden activations handed to the second product) and Y are rounded to
+ * bfloat16, the places where an implementation with 16-bit storage has to round. */
+void orc_ffn(int n, int d, int d_ff, const double* X, const double* W1, const double* b1, const double* W2,
+             const double* b2, const double* gamma, const double* beta, double eps, int rounding, double* Y) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < n; ++i) {
+        const double* x = X + (int64_t)i * d;
+        std::vector<double> u(d_ff), z(d);
+        for (int h = 0; h < d_ff; ++h) {
+            double acc = b1[h];
+            for (int c = 0; c < d; ++c) acc += x[c] * W1[(int64_t)h * d + c];
+            acc = acc > 0.0 ? acc : 0.0;
+            u[h] = store_round(acc, rounding);
+        }
+        for (int o = 0; o < d; ++o) {
+            double acc = b2[o];
+            for (int h = 0; h < d_ff; ++h) acc += u[h] * W2[(int64_t)o * d_ff + h];
+            z[o] = x[o] + acc;
+        }
+        double* y = Y + (int64_t)i * d;
+        orc_layernorm(1, d, z.data(), gamma, beta, eps, y);
+        for (int o = 0; o < d; ++o) y[o] = store_round(y[o], rounding);
+    }
 }
 
 /* Levelised layer, in place on H.  Buckets l = 0..n_levels-1 are processed in order; a node v of bucket l

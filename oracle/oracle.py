@@ -53,6 +53,10 @@ def _load():
         lib.orc_attention_additive.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, _i32p, _i32p, _f64p, _f64p]
         lib.orc_project.restype = None
         lib.orc_project.argtypes = [c_int, c_int, c_int, _f64p, _f64p, _f64p, _f64p]
+        lib.orc_layernorm.restype = None
+        lib.orc_layernorm.argtypes = [c_int, c_int, _f64p, _f64p, _f64p, c_dbl, _f64p]
+        lib.orc_ffn.restype = None
+        lib.orc_ffn.argtypes = [c_int, c_int, c_int, _f64p, _f64p, _f64p, _f64p, _f64p, _f64p, _f64p, c_dbl, c_int, _f64p]
         lib.orc_layer_parallel.restype = None
         lib.orc_layer_parallel.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, c_int, _i32p, _i32p,
                                            c_int, _f64p]
@@ -191,6 +195,27 @@ def project(X, W, R=None):
     d_out = W.shape[0]
     Y = np.zeros((n, d_out), np.float64)
     _load().orc_project(n, d_in, d_out, _d(X), _d(W), _d(R), _d(Y))
+    return Y
+
+
+def layernorm(X, gamma, beta, eps=1e-5):
+    """Row-wise layer normalisation (biased variance over the features of a row)."""
+    X, gamma, beta = _f64(X), _f64(gamma), _f64(beta)
+    n, d = X.shape
+    Y = np.zeros((n, d), np.float64)
+    _load().orc_layernorm(n, d, _d(X), _d(gamma), _d(beta), float(eps), _d(Y))
+    return Y
+
+
+def ffn(X, W1, b1, W2, b2, gamma, beta, eps=1e-5, rounding=None):
+    """LayerNorm(X + max(0, X W1^T + b1) W2^T + b2); W1 [d_ff, d], W2 [d, d_ff]."""
+    X, W1, b1, W2, b2, gamma, beta = (_f64(a) for a in (X, W1, b1, W2, b2, gamma, beta))
+    n, d = X.shape
+    d_ff = W1.shape[0]
+    assert W1.shape == (d_ff, d) and W2.shape == (d, d_ff) and b1.shape == (d_ff,) and b2.shape == (d,)
+    Y = np.zeros((n, d), np.float64)
+    _load().orc_ffn(n, d, d_ff, _d(X), _d(W1), _d(b1), _d(W2), _d(b2), _d(gamma), _d(beta), float(eps),
+                    ROUND[rounding], _d(Y))
     return Y
 
 

@@ -17,7 +17,9 @@
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
 // to layers round-robin; each keeps its layer's W_o, W_k, W_v and the next layer's W_q, W_k, W_v resident in
-// shared memory (one TMA load each).  With n layers the dependent chain is n_levels + n - 1 tile steps long
+// TENSOR memory (six blocks of 128 lanes x 64 columns beside the accumulators) and issues its MMAs with the A
+// operand read from there, so the weights are never re-read from shared memory and shared memory holds only the
+// node-side tiles.  With n layers the dependent chain is n_levels + n - 1 tile steps long
 // instead of n * n_levels, while computing exactly what n successive level-by-level sweeps compute.
 //
 // Levels are separated by counters in global memory instead of kernel launches: every (layer, level) has an
@@ -41,35 +43,37 @@ using namespace attn;
 
 constexpr int kTile = 16;                    // nodes per tile
 constexpr int kThreads = kTile * 16;         // 16 lanes per node
-constexpr int kWBlock = 2 * 128 * 128;       // one 128 x 128 bf16 weight block: two K-halves of 16 KiB
 constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
-constexpr int kTmemCols = 128;               // six accumulators of kTile columns
+constexpr int kTmemCols = 512;               // six accumulators of kTile columns, then six weight blocks of 64 columns
+constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks W_o | W_k | W_v | next W_q | W_k | W_v
+constexpr int kWCols = 64;                   // a 128 x 128 bf16 block: 128 lanes x 64 columns of two elements
 constexpr int kStageRow = 1280;              // staging per node: K|V of this layer 512, Q of the next 256, its K|V 512
 
-constexpr int kOffW = 0;                          // W_o | W_k | W_v | next W_q | W_k | W_v : 192 KiB
-constexpr int kOffO = 6 * kWBlock;                // attention tile (operand layout)
+constexpr int kOffO = 0;                          // attention tile (operand layout)
 constexpr int kOffHp = kOffO + 2 * kBHalf;        // new rows (operand layout)
 constexpr int kOffHres = kOffHp + 2 * kBHalf;     // residual rows, plain [kTile][256 B]
 constexpr int kOffStage = kOffHres + kTile * 256; // output staging, plain [kTile][kStageRow]
 constexpr int kOffMisc = kOffStage + kTile * kStageRow;
 constexpr int kSmemBytes = kOffMisc + 256 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
+static_assert(kWCol0 + 6 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
+// Every CTA allocates all of its SM's tensor memory, so two CTAs must never share an SM (the second one's
+// allocation would wait for the first, which waits for the second's levels): the launch asks for more than half
+// of an SM's shared memory, which rules that out.
+constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
 struct Misc {
-    uint64_t w_full, mma1, mma2;
+    uint64_t mma1, mma2;
     uint32_t tmem_base;
     int32_t go, go2;
     int32_t node[kTile];
 };
 
-struct LayerMaps {
-    CUtensorMap wo[DG4I_MAX_LAYERS];
-    CUtensorMap wqkv[DG4I_MAX_LAYERS];
-};
-
 struct LevParams {
     __nv_bfloat16* Q[DG4I_MAX_LAYERS];     // [n, 128] per layer
     __nv_bfloat16* KV[DG4I_MAX_LAYERS];    // [n, 256] per layer
+    const __nv_bfloat16* Wo[DG4I_MAX_LAYERS];    // [128, 128] per layer, out x in
+    const __nv_bfloat16* Wqkv[DG4I_MAX_LAYERS];  // [384, 128] per layer
     __nv_bfloat16* H;                      // [n, ldh], updated in place by every layer in turn
     int64_t ldh;
     const int32_t* nbr_pad;                // [n, pad_width]
@@ -109,11 +113,6 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t* r) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr) : "memory");
-}
 __device__ __forceinline__ uint16_t bf16_bits(float x) {
     __nv_bfloat16 h = __float2bfloat16_rn(x);
     return *reinterpret_cast<uint16_t*>(&h);
@@ -141,18 +140,18 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
 
 template <int LPH, int MAXN>
 __global__ void __launch_bounds__(kThreads, 1)
-levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
+levelised_kernel(LevParams p) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int W = MAXN + 1;                          // width of a neighbour-table entry
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
-    const uint32_t sW = base + kOffW, sO = base + kOffO, sHp = base + kOffHp, sHres = base + kOffHres, sSt = base + kOffStage;
+    const uint32_t sO = base + kOffO, sHp = base + kOffHp, sHres = base + kOffHres, sSt = base + kOffStage;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid >> 4, sub = tid & 15;          // node slot of the tile and lane within the node
     const int grp_base = lane - sub;
     const unsigned gmask = 0xffffu << grp_base;
-    const uint32_t bar_w = smem_u32(&misc->w_full), bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
+    const uint32_t bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
 
     // this CTA's layer, its rank among the CTAs of that layer, and how many CTAs each layer has
     const int layer = (int)blockIdx.x % p.n_layers;
@@ -163,37 +162,46 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
     const int n_acc = has_next ? 5 : 2;                  // accumulators of the second MMA group
 
     if (tid == 0) {
-        mbar_init(bar_w, 1);
         mbar_init(bar1, 1);
         mbar_init(bar2, 1);
         misc->go = 1;
         misc->go2 = 1;
         mbar_fence_init();
-        tma_prefetch_desc(&maps.wo[layer]);
-        tma_prefetch_desc(&maps.wqkv[layer]);
-        mbar_expect_tx(bar_w, (uint32_t)((has_next ? 6 : 3) * kWBlock));
-        for (int h = 0; h < 2; ++h) {
-            tma_load_2d(sW + h * (kWBlock / 2), &maps.wo[layer], h * 64, 0, bar_w);
-            tma_load_2d(sW + kWBlock + h * (kWBlock / 2), &maps.wqkv[layer], h * 64, 128, bar_w);
-            tma_load_2d(sW + 2 * kWBlock + h * (kWBlock / 2), &maps.wqkv[layer], h * 64, 256, bar_w);
-            if (has_next)
-                for (int b = 0; b < 3; ++b)
-                    tma_load_2d(sW + (3 + b) * kWBlock + h * (kWBlock / 2), &maps.wqkv[layer + 1], h * 64, b * 128, bar_w);
-        }
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc->tmem_base;
-    if (!mbar_wait(bar_w, 0) && tid == 0) give_up(p);
+    static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
+    const int q4 = warp & 3, cg = warp >> 2;             // TMEM lane quadrant of the warp; which half of the columns it takes
+    const int feat = q4 * 32 + lane;                     // output feature (TMEM lane) this thread holds
+    // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
+    // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
+    // half a row (128 bytes) of every block of its layer.
+    {
+        const int n_blocks = has_next ? 6 : 3;
+        for (int blk = 0; blk < n_blocks; ++blk) {
+            const __nv_bfloat16* wb = blk == 0 ? p.Wo[layer]
+                                     : blk < 3 ? p.Wqkv[layer] + (size_t)blk * 128 * 128
+                                               : p.Wqkv[layer + 1] + (size_t)(blk - 3) * 128 * 128;
+            const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint4 lo = src[2 * c], hi = src[2 * c + 1];
+                const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                tmem_st_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kWCol0 + blk * kWCols + cg * 32 + c * 8), r);
+            }
+        }
+        tmem_st_wait();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
 
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
-    // matrix descriptors of the resident operands; stepping along K or to another block only adds to the address field
-    const uint64_t dW = smem_desc_sw128(sW), dO = smem_desc_sw128(sO), dHp = smem_desc_sw128(sHp);
-    static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
-    const int q4 = warp & 3, cg = warp >> 2;             // epilogue: TMEM lane quadrant and group of 8 node columns
-    const int feat = q4 * 32 + lane;                     // output feature this thread holds in the epilogues
+    // matrix descriptors of the node-side operands; stepping along K only adds to the address field
+    const uint64_t dO = smem_desc_sw128(sO), dHp = smem_desc_sw128(sHp);
     uint32_t ph1 = 0, ph2 = 0;
     int last_nonempty = -1, last_participants = 0;
     bool alive = true;
@@ -208,23 +216,25 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
     // any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
     // level-to-level critical path: while level l is processed, the node id of this CTA's first tile of level
     // l+2 and the table entry for level l+1 are in flight.
-    auto level_first = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv] : 0; };
-    auto level_size = [&](int lv) { return lv < p.n_levels ? p.level_ptr[lv + 1] - p.level_ptr[lv] : 0; };
-    auto stage_node = [&](int lv) -> int {            // node of (first tile of this CTA, this slot) at level lv
-        const int n_lv = level_size(lv);
+    // The level offsets run four levels ahead in registers: every acquire of a counter drops the L1 contents,
+    // so a plain load at the top of a level would cost a trip to L2 on the level-to-level chain.
+    auto lp_at = [&](int lv) { return p.level_ptr[lv < p.n_levels ? lv : p.n_levels]; };
+    auto stage_node = [&](int lv_first, int lv_end) -> int {   // node of (first tile of this CTA, this slot) of a level
         const int r = bid * kTile + slot;
-        return (r < n_lv) ? p.level_nodes[level_first(lv) + r] : -1;
+        return (r < lv_end - lv_first) ? p.level_nodes[lv_first + r] : -1;
     };
+    int lp0 = lp_at(0), lp1 = lp_at(1), lp2 = lp_at(2), lp3 = lp_at(3);
     auto pad_of = [&](int v) -> int { return (v >= 0 && sub < W) ? p.nbr_pad[(size_t)v * W + sub] : 0; };
-    int v0 = stage_node(0);                            // level l  : node id and this lane's table word
+    int v0 = stage_node(lp0, lp1);                     // level l  : node id and this lane's table word
     int pad0 = pad_of(v0);
-    int vC = stage_node(1);                            // level l+1: node id
+    int vC = stage_node(lp1, lp2);                     // level l+1: node id
 
     for (int l = 0; l < p.n_levels && alive; ++l) {
-        const int first = p.level_ptr[l];
-        const int n_l = p.level_ptr[l + 1] - first;
+        const int first = lp0;
+        const int n_l = lp1 - lp0;
         // issue the next load of every pipelined chain; the results are first used one level later
-        const int vB = stage_node(l + 2);
+        const int lp4 = lp_at(l + 4);
+        const int vB = stage_node(lp2, lp3);
         const int padC = pad_of(vC);
         const int tiles = (n_l + kTile - 1) / kTile;
         if (n_l > 0 && bid < tiles) {
@@ -298,9 +308,8 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t a_off = (uint32_t)((ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
                         const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                        mma_bf16(tmem, dW + (a_off >> 4), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                        mma_bf16_ta(tmem, tmem + (uint32_t)(kWCol0 + ks * 8), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
                     }
                     mma_commit(bar1);
                 }
@@ -326,15 +335,17 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
                 // ---- from the new rows, transposed: this layer's K | V refresh and the next layer's Q | K | V
                 if (tid == 0) {
                     tc_fence_after();
+                    // K-step outermost: consecutive instructions accumulate into different accumulators, so none
+                    // has to wait for the one before it
 #pragma unroll
-                    for (int blk = 0; blk < 5; ++blk) {
-                        if (blk < n_acc) {
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
 #pragma unroll
-                            for (int ks = 0; ks < 8; ++ks) {
-                                const uint32_t a_off = (uint32_t)((1 + blk) * kWBlock + (ks >> 2) * (kWBlock / 2) + (ks & 3) * 32);
-                                const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                                mma_bf16(tmem + (uint32_t)(kTile * (1 + blk)), dW + (a_off >> 4), dHp + (b_off >> 4), idesc,
-                                         ks > 0 ? 1u : 0u);
+                        for (int blk = 0; blk < 5; ++blk) {
+                            if (blk < n_acc) {
+                                mma_bf16_ta(tmem + (uint32_t)(kTile * (1 + blk)),
+                                            tmem + (uint32_t)(kWCol0 + (1 + blk) * kWCols + ks * 8), dHp + (b_off >> 4), idesc,
+                                            ks > 0 ? 1u : 0u);
                             }
                         }
                     }
@@ -392,7 +403,9 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
             }
             if (!alive) break;
             // ---- this CTA's part of (layer, level l) is in global memory: arrive on its counter (release)
-            if (tid == 0) red_release_add(my_arrive + l, 1);
+            // (by a thread that does not poll: the release waits for the CTA's outstanding stores, and the pollers
+            // should already be watching the next level's counters meanwhile)
+            if (tid == 64) red_release_add(my_arrive + l, 1);
         }
         if (n_l > 0) {
             last_nonempty = l;
@@ -401,6 +414,7 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
         // rotate the pipeline by one level
         v0 = vC; pad0 = padC;
         vC = vB;
+        lp0 = lp1; lp1 = lp2; lp2 = lp3; lp3 = lp4;
     }
 
     tc_fence_before();
@@ -412,62 +426,32 @@ levelised_kernel(const __grid_constant__ LayerMaps maps, LevParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 std::mutex g_mu;
-EncodeTiledFn g_encode = nullptr;
 int g_sm_count[64] = {};
 int g_coop[64] = {};
 bool g_dev_known[64] = {};
 
-dg4_status make_weight_map(CUtensorMap* m, const void* base, int64_t rows) {
-    {
-        std::lock_guard<std::mutex> lock(g_mu);
-        if (!g_encode) {
-            void* fn = nullptr;
-            cudaDriverEntryPointQueryResult q;
-            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
-            if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
-                cudaGetLastError();
-                DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-            }
-            g_encode = (EncodeTiledFn)fn;
-        }
-    }
-    cuuint64_t dims[2] = {128, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {256};
-    cuuint32_t box[2] = {64, 128};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    return DG4_OK;
-}
-
 template <int LPH, int MAXN>
-dg4_status launch(const LayerMaps& maps, const LevParams& p, int grid, cudaStream_t st) {
+dg4_status launch(const LevParams& p, int grid, cudaStream_t st) {
     auto kern = levelised_kernel<LPH, MAXN>;
-    DG4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    DG4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLaunchSmemBytes));
     int per_sm = 0;
-    DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
-    if (per_sm < 1) DG4_FAIL(DG4_ERR_CUDA, "the levelised kernel does not fit on this device");
-    void* args[] = {(void*)&maps, (void*)&p};
-    DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, kSmemBytes, st));
+    DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kLaunchSmemBytes));
+    if (per_sm != 1) DG4_FAIL(DG4_ERR_CUDA, "the levelised kernel needs exactly one CTA per SM on this device (got %d)", per_sm);
+    void* args[] = {(void*)&p};
+    DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, kLaunchSmemBytes, st));
     dg4i_count_launch();
     return DG4_OK;
 }
 
 template <int MAXN>
-dg4_status launch_heads(int heads, const LayerMaps& maps, const LevParams& p, int grid, cudaStream_t st) {
+dg4_status launch_heads(int heads, const LevParams& p, int grid, cudaStream_t st) {
     switch (16 / heads) {
-        case 1: return launch<1, MAXN>(maps, p, grid, st);
-        case 2: return launch<2, MAXN>(maps, p, grid, st);
-        case 4: return launch<4, MAXN>(maps, p, grid, st);
-        case 8: return launch<8, MAXN>(maps, p, grid, st);
-        case 16: return launch<16, MAXN>(maps, p, grid, st);
+        case 1: return launch<1, MAXN>(p, grid, st);
+        case 2: return launch<2, MAXN>(p, grid, st);
+        case 4: return launch<4, MAXN>(p, grid, st);
+        case 8: return launch<8, MAXN>(p, grid, st);
+        case 16: return launch<16, MAXN>(p, grid, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported", heads);
 }
@@ -497,13 +481,11 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     }
     if (!g_coop[dev]) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device %d cannot launch cooperative kernels", dev);
     if (g_sm_count[dev] < n_layers) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer SMs than layers");
-    LayerMaps maps;
     LevParams p;
-    dg4_status s;
     for (int k = 0; k < DG4I_MAX_LAYERS; ++k) {
         const int kk = k < n_layers ? k : 0;           // unused slots repeat layer 0 (never read)
-        if ((s = make_weight_map(&maps.wo[k], W_o[kk], 128)) != DG4_OK) return s;
-        if ((s = make_weight_map(&maps.wqkv[k], W_qkv[kk], 384)) != DG4_OK) return s;
+        p.Wo[k] = W_o[kk];
+        p.Wqkv[k] = W_qkv[kk];
         p.Q[k] = Q[kk];
         p.KV[k] = KV[kk];
     }
@@ -514,6 +496,6 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status;
     const int grid = g_sm_count[dev];
-    if (g->max_class <= 3) return launch_heads<3>(desc->heads, maps, p, grid, st);
-    return launch_heads<7>(desc->heads, maps, p, grid, st);
+    if (g->max_class <= 3) return launch_heads<3>(desc->heads, p, grid, st);
+    return launch_heads<7>(desc->heads, p, grid, st);
 }

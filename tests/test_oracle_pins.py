@@ -506,3 +506,90 @@ def test_partition_roots_by_vectorised_selection():
         roots, gptr = orc.partition_roots(rp, ci, level, k, delta)
         assert (roots == want).all()
         assert (gptr == np.concatenate([[0], np.cumsum(np.bincount(level[want], minlength=level.max() + 1))])).all()
+
+
+# ----------------------------------------------------------------------------- rest of the block: LayerNorm, FFN
+
+def _read_ffn_golden():
+    out = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "ffn_tiny.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        name, body = [t.strip() for t in line.split("|")]
+        rows = [[float(t) for t in r.split()] for r in body.split(";")]
+        out[name] = np.array(rows if len(rows) > 1 else rows[0], np.float64)
+    return out
+
+
+def test_ffn_matches_hand_worked_fixture():
+    g = _read_ffn_golden()
+    y = orc.ffn(g["x"][None, :], g["W1"], g["b1"], g["W2"], g["b2"], g["gamma"], g["beta"], eps=0.0)
+    assert np.allclose(y[0], g["y"], rtol=0, atol=1e-12)
+
+
+def test_layernorm_closed_forms_and_invariants():
+    one, zero = np.ones(4), np.zeros(4)
+    # 1,2,3,4: mean 2.5, biased variance 1.25
+    y = orc.layernorm(np.array([[1.0, 2.0, 3.0, 4.0]]), one, zero, eps=0.0)
+    assert np.allclose(y[0], np.array([-1.5, -0.5, 0.5, 1.5]) / np.sqrt(1.25), atol=1e-14)
+    # a constant row has nothing to normalise: beta comes out
+    beta = np.array([0.5, -1.0, 2.0, 0.0])
+    assert np.allclose(orc.layernorm(np.full((1, 4), 7.0), np.array([3.0, 1.0, 2.0, 5.0]), beta, eps=1e-5)[0], beta, atol=1e-12)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((6, 128))
+    y = orc.layernorm(x, np.ones(128), np.zeros(128), eps=0.0)
+    assert np.allclose(y.mean(1), 0, atol=1e-13) and np.allclose(y.var(1), 1, atol=1e-12)
+    # shift and positive scaling of the input leave the result alone (eps = 0)
+    assert np.allclose(orc.layernorm(3.5 * x + 11.0, np.ones(128), np.zeros(128), eps=0.0), y, atol=1e-11)
+    # eps enters under the root: a row of variance v comes out with variance v / (v + eps)
+    y2 = orc.layernorm(x, np.ones(128), np.zeros(128), eps=0.25)
+    assert np.allclose(y2.var(1), x.var(1) / (x.var(1) + 0.25), atol=1e-12)
+    # gamma and beta act per feature, after the normalisation
+    gam, bet = rng.standard_normal(128), rng.standard_normal(128)
+    assert np.allclose(orc.layernorm(x, gam, bet, eps=0.0), y * gam + bet, atol=1e-12)
+
+
+def test_ffn_closed_forms():
+    rng = np.random.default_rng(6)
+    d = 16
+    x = rng.standard_normal((9, d))
+    eye, one, zero = np.eye(d), np.ones(d), np.zeros(d)
+    # W1 = [I; -I], W2 = [I, -I]: max(0, x) - max(0, -x) = x, so the sub-layer returns LayerNorm(2 x) = LayerNorm(x)
+    y = orc.ffn(x, np.vstack([eye, -eye]), np.zeros(2 * d), np.hstack([eye, -eye]), zero, one, zero, eps=0.0)
+    assert np.allclose(y, orc.layernorm(x, one, zero, eps=0.0), atol=1e-12)
+    # a bias that switches every hidden unit off leaves LayerNorm(x + b2)
+    W1, W2, b2 = rng.standard_normal((40, d)), rng.standard_normal((d, 40)), rng.standard_normal(d)
+    y = orc.ffn(x, W1, np.full(40, -1e6), W2, b2, one, zero, eps=1e-5)
+    assert np.allclose(y, orc.layernorm(x + b2, one, zero, eps=1e-5), atol=1e-12)
+    # a bias that keeps every hidden unit on makes the sub-layer affine: x + (x W1^T + b1) W2^T + b2
+    b1 = np.full(40, 1e3)
+    y = orc.ffn(x, W1, b1, W2, b2, one, zero, eps=1e-5)
+    z = x + x @ (W2 @ W1).T + W2 @ b1 + b2
+    assert np.allclose(y, orc.layernorm(z, one, zero, eps=1e-5), atol=1e-9)
+
+
+@pytest.mark.parametrize("n,d,d_ff", [(1, 8, 32), (33, 128, 512), (7, 24, 10)])
+def test_ffn_equals_dense_library_algebra(n, d, d_ff):
+    rng = np.random.default_rng(n + d)
+    x, W1, b1 = rng.standard_normal((n, d)), rng.standard_normal((d_ff, d)) * 0.3, rng.standard_normal(d_ff)
+    W2, b2 = rng.standard_normal((d, d_ff)) * 0.3, rng.standard_normal(d)
+    gam, bet = rng.standard_normal(d), rng.standard_normal(d)
+    t = lambda a: torch.from_numpy(a)
+    z = t(x) + torch.relu(t(x) @ t(W1).T + t(b1)) @ t(W2).T + t(b2)
+    ref = torch.nn.functional.layer_norm(z, (d,), t(gam), t(bet), eps=1e-5).numpy()
+    assert np.allclose(orc.ffn(x, W1, b1, W2, b2, gam, bet, eps=1e-5), ref, atol=1e-11)
+
+
+def test_ffn_rounding_points():
+    # with 16-bit storage the hidden activations and the result are rounded, nothing else
+    rng = np.random.default_rng(8)
+    d, d_ff = 8, 16
+    x = orc.round_bf16(rng.standard_normal((5, d)))
+    W1, W2 = orc.round_bf16(rng.standard_normal((d_ff, d))), orc.round_bf16(rng.standard_normal((d, d_ff)))
+    b1, b2, gam, bet = rng.standard_normal(d_ff), rng.standard_normal(d), rng.standard_normal(d), rng.standard_normal(d)
+    u = orc.round_bf16(np.maximum(0.0, x @ W1.T + b1))
+    z = x + u @ W2.T + b2
+    ref = orc.round_bf16(orc.layernorm(z, gam, bet, eps=1e-5))
+    got = orc.ffn(x, W1, b1, W2, b2, gam, bet, eps=1e-5, rounding="bf16")
+    assert np.allclose(got, ref, atol=1e-12)
