@@ -275,6 +275,41 @@ dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, vo
                                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream);
 
 /*
+ * The rest of the Transformer block around the attention (Sec. 3.5: only the multi-head attention module is
+ * replaced, the structure of the original Transformer layer is kept; that layer is post-norm with a two-matrix
+ * ReLU feed-forward sub-layer; the paper's figure of the block is not part of its text, so this reading is the
+ * library's stated choice).  bf16 rows, fp32 arithmetic, d = 128.  All pointers are device pointers; rows have
+ * 128 valid elements and leading dimensions ldx / ldy in elements (multiples of 8); gamma, beta, b1, b2 are fp32
+ * vectors, 16-byte aligned.  eps >= 0 enters under the square root.  Asynchronous on `stream`; the number of rows
+ * is the handle's node count.  Errors: DG4_ERR_INVALID_ARG (null, misaligned, bad eps), DG4_ERR_UNSUPPORTED
+ * (d != 128, dtype != bf16, d_ff != 512), DG4_ERR_CUDA; a device-side wait that runs out records DG4_ERR_TIMEOUT
+ * in the handle's status word (dg4_graph_poll_status).
+ *
+ * dg4_layernorm_fwd: Y[i,:] = (X[i,:] - mean_i) / sqrt(var_i + eps) * gamma + beta, mean and biased variance over
+ * the 128 features of row i.  Y may be X.
+ *
+ * dg4_ffn_fwd: Y = LayerNorm(X + max(0, X W1^T + b1) W2^T + b2) with W1 [d_ff, 128] and W2 [128, d_ff] row-major
+ * bf16 (out x in), d_ff = 512.  The hidden activations are rounded to bf16 between the two products and are never
+ * written to global memory.  Y may be X.
+ *
+ * dg4_block_fwd_parallel: one whole block on all nodes at once:
+ *     H1 = LayerNorm_1(H_in + Attention(H_in) W_o^T),   H_out = LayerNorm_2(H1 + FFN(H1)),
+ * Attention being dg4_qkv_project + dg4_sparse_attn_fwd on the handle's neighbourhoods (desc gives heads and
+ * scale; the residual connections are always on).  workspace: dg4_layer_workspace_bytes() bytes, 256-byte aligned,
+ * owned by the caller; the library allocates nothing.  H_out may be H_in.
+ */
+dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
+                             const float* gamma, const float* beta, float eps, void* Y, int64_t ldy, void* stream);
+dg4_status dg4_ffn_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx, const void* W1,
+                       const float* b1, const void* W2, const float* b2, const float* gamma, const float* beta,
+                       float eps, int32_t d_ff, void* Y, int64_t ldy, void* stream);
+dg4_status dg4_block_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, const void* H_in, int64_t ldh,
+                                  const void* W_qkv, const void* W_o, const float* ln1_gamma, const float* ln1_beta,
+                                  const void* W1, const float* b1, const void* W2, const float* b2,
+                                  const float* ln2_gamma, const float* ln2_beta, float eps, int32_t d_ff,
+                                  void* H_out, int64_t ldho, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Diagnostic (the paper has no counterpart): launches one small CTA that waits, with the same bounded wait the
  * pipelines of this library use, on a barrier nothing ever arrives on.  The wait gives up after its poll limit
  * (about a second) and the kernel writes DG4_ERR_TIMEOUT to *device_status (device int32) and returns normally:

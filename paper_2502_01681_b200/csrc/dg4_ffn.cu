@@ -1,0 +1,470 @@
+// The rest of the Transformer block around the sparse attention (Sec. 3.5 replaces only the attention module
+// and keeps the block's structure; the block itself is the original post-norm Transformer layer):
+//   row-wise layer normalisation, and the position-wise feed-forward sub-layer with residual and the
+//   normalisation that follows it:
+//       U = max(0, X W1^T + b1),  W1 [512, 128];     Y = LayerNorm(X + U W2^T + b2),  W2 [128, 512].
+//
+// ffn_kernel: one persistent CTA per SM, a tile = 128 rows.  The hidden activations never leave the SM.
+//   * W1 stays in TENSOR memory for the whole kernel (4 blocks of 128 hidden units x 128 inputs = 4 x 64 columns)
+//     and is the A operand of the first product, computed TRANSPOSED per block q of 128 hidden units:
+//         D1^T[hidden, row] = W1_q (tensor memory) * X^T (the X tile in shared memory, K-major, as B operand);
+//   * the epilogue of block q (thread = hidden unit, registers = rows) adds b1, applies the ReLU, rounds to
+//     bf16 and scatters the values into shared memory as the K-major, 128-byte-swizzled A operand of the
+//     second product: A2[row, hidden of block q];
+//   * second product, accumulated over the four blocks: D2[row, out] += A2 * W2_q^T with W2 resident in shared
+//     memory (4 chunks of 128 outputs x 128 hidden units, 128 KiB, loaded once by TMA);
+//   * final epilogue (thread = row, two threads per row): + b2 + the X row (still in shared memory), mean and
+//     variance of the row combined from the two half-rows, gamma / beta, bf16, staged in shared memory and
+//     written with a TMA store (the last tile is clipped by the tensor map).
+//   The X tile of the next tile is prefetched by TMA while the current one is processed.
+// No cluster multicast anywhere.  Every wait is bounded; after a timeout the kernel records DG4_ERR_TIMEOUT and
+// the CTA leaves its tile loop.
+#include "dg4_internal.h"
+#include "dg4_sm100.cuh"
+
+#include <algorithm>
+#include <mutex>
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kTileM = 128;                 // rows per tile
+constexpr int kThreads = 256;
+constexpr int kHalf = 128 * 128;            // bytes of one K-half (64 bf16 columns) of a 128-row operand tile
+constexpr int kTileBytes = 2 * kHalf;       // 32 KiB: a 128 x 128 bf16 operand tile
+constexpr int kOffW2 = 0;                   // 4 chunks of W2
+constexpr int kOffX = 4 * kTileBytes;       // 2 stages of X tiles
+constexpr int kOffA2 = kOffX + 2 * kTileBytes;   // hidden activations of one block; later the output staging
+constexpr int kOffMisc = kOffA2 + kTileBytes;
+constexpr int kSmemBytes = kOffMisc + 1024 + 128;
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
+constexpr int kColD1 = 0, kColD2 = 128, kColW1 = 256, kTmemCols = 512;
+
+struct Misc {
+    uint64_t bar_w, bar_x[2], bar_mma;
+    uint32_t tmem_base;
+};
+
+struct FfnParams {
+    const __nv_bfloat16* W1;
+    const float* b1;
+    const float* b2;
+    const float* gamma;
+    const float* beta;
+    float eps;
+    int32_t n_tiles;
+    int32_t* status;
+};
+
+__device__ __forceinline__ void st_shared_b16(uint32_t addr, uint16_t v) {
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t* r) {
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void st_shared_f2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void ld_shared_f2(uint32_t addr, float& a, float& b) {
+    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ uint16_t bf16_bits(float x) {
+    __nv_bfloat16 h = __float2bfloat16_rn(x);
+    return *reinterpret_cast<uint16_t*>(&h);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
+}
+// byte offset of element k (0..127) of row `row` in a 128-row operand tile (two K-halves, 128-byte swizzle)
+__device__ __forceinline__ uint32_t operand_offset(int row, int k) {
+    return (uint32_t)((k >> 6) * kHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
+}
+// descriptor address increment of K-step ks (16 elements) inside an operand tile
+__device__ __forceinline__ uint64_t kstep(int ks) { return (uint64_t)(((ks >> 2) * kHalf + (ks & 3) * 32) >> 4); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w2,
+           const __grid_constant__ CUtensorMap map_y, FfnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
+    const uint32_t sW2 = base + kOffW2, sX = base + kOffX, sA2 = base + kOffA2;
+    const uint32_t bar_w = smem_u32(&misc->bar_w), bar_mma = smem_u32(&misc->bar_mma);
+    const uint32_t bar_x[2] = {smem_u32(&misc->bar_x[0]), smem_u32(&misc->bar_x[1])};
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int q4 = warp & 3, cg = warp >> 2;             // TMEM lane quadrant of the warp; which half of the columns it takes
+    const int ln = q4 * 32 + lane;                       // TMEM lane of this thread: a hidden unit, later a row
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+
+    const int first_tile = (int)blockIdx.x;
+    if (tid == 0) {
+        mbar_init(bar_w, 1);
+        mbar_init(bar_x[0], 1);
+        mbar_init(bar_x[1], 1);
+        mbar_init(bar_mma, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_w2);
+        tma_prefetch_desc(&map_y);
+        if (first_tile < p.n_tiles) {
+            mbar_expect_tx(bar_w, 4 * kTileBytes);
+            for (int q = 0; q < 4; ++q)
+                for (int h = 0; h < 2; ++h)
+                    tma_load_2d(sW2 + q * kTileBytes + h * kHalf, &map_w2, q * 128 + h * 64, 0, bar_w);
+            mbar_expect_tx(bar_x[0], kTileBytes);
+            for (int h = 0; h < 2; ++h) tma_load_2d(sX + h * kHalf, &map_x, h * 64, first_tile * kTileM, bar_x[0]);
+        }
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc->tmem_base;
+
+    // W1 into tensor memory: hidden unit `ln` of block q in lane `ln`, two consecutive inputs per 32-bit column
+    // (the bytes as they lie in global memory); each thread copies half a row (128 bytes) of every block.
+    float b1v[4];
+    for (int q = 0; q < 4; ++q) {
+        const uint4* src = reinterpret_cast<const uint4*>(p.W1 + (size_t)(q * 128 + ln) * 128 + cg * 64);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint4 lo = src[2 * c], hi = src[2 * c + 1];
+            const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+            tmem_st_32x8(tmem + lane_base + (uint32_t)(kColW1 + q * 64 + cg * 32 + c * 8), r);
+        }
+        b1v[q] = p.b1[q * 128 + ln];
+    }
+    tmem_st_wait();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const uint32_t idesc = idesc_bf16_f32(128, 128);
+    const uint64_t dA2 = smem_desc_sw128(sA2);
+    uint32_t ph_mma = 0;
+    bool failed = false;
+    if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0);
+
+    int it = 0;
+    for (int tile = first_tile; tile < p.n_tiles; tile += (int)gridDim.x, ++it) {
+        const int s = it & 1;
+        const uint32_t sXs = sX + s * kTileBytes;
+        const uint64_t dX = smem_desc_sw128(sXs);
+        if (tid == 0) {
+            const int next = tile + (int)gridDim.x;      // prefetch the next tile's rows into the other stage
+            if (next < p.n_tiles) {
+                mbar_expect_tx(bar_x[s ^ 1], kTileBytes);
+                for (int h = 0; h < 2; ++h)
+                    tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
+            }
+        }
+        failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u);
+
+        auto issue_g1 = [&](int q) {     // D1^T = W1_q * X^T
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                mma_bf16_ta(tmem + kColD1, tmem + (uint32_t)(kColW1 + q * 64 + ks * 8), dX + kstep(ks), idesc, ks > 0 ? 1u : 0u);
+        };
+        if (tid == 0) {
+            tc_fence_after();
+            issue_g1(0);
+            mma_commit(bar_mma);
+        }
+
+        for (int q = 0; q < 4; ++q) {
+            failed |= !mbar_wait(bar_mma, ph_mma);       // D1^T of block q is complete (and so is everything before it)
+            ph_mma ^= 1u;
+            tc_fence_after();
+            if (q == 0) {                                // the previous tile's store must have read the staging buffer
+                if (tid == 0) bulk_wait_read0();
+                __syncthreads();
+            }
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + half * 32), d);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int row = cg * 64 + half * 32 + j;
+                    const float u = fmaxf(__uint_as_float(d[j]) + b1v[q], 0.0f);
+                    st_shared_b16(sA2 + operand_offset(row, ln), bf16_bits(u));
+                }
+            }
+            tc_fence_before();
+            fence_proxy_async_smem();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                const uint64_t dW2 = smem_desc_sw128(sW2 + q * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)           // D2 += A2 * W2_q^T
+                    mma_bf16(tmem + kColD2, dA2 + kstep(ks), dW2 + kstep(ks), idesc, (q > 0 || ks > 0) ? 1u : 0u);
+                if (q < 3) issue_g1(q + 1);
+                mma_commit(bar_mma);
+            }
+        }
+        failed |= !mbar_wait(bar_mma, ph_mma);           // D2 is complete; the activation buffer is free
+        ph_mma ^= 1u;
+        tc_fence_after();
+
+        // ---- final epilogue: thread = row `ln`, columns cg*64 .. cg*64+63
+        {
+            float y[64];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64 + half * 32), d);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) y[half * 32 + j] = __uint_as_float(d[j]);
+            }
+            tc_fence_before();
+            const float4* b2v = reinterpret_cast<const float4*>(p.b2 + cg * 64);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {                // + b2 + the row of X (K-half cg of the X tile)
+                uint32_t w[4];
+                ld_shared_v4(sXs + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
+                const float4 ba = __ldg(b2v + 2 * c), bb = __ldg(b2v + 2 * c + 1);
+                y[c * 8 + 0] += __uint_as_float(w[0] << 16) + ba.x;
+                y[c * 8 + 1] += __uint_as_float(w[0] & 0xffff0000u) + ba.y;
+                y[c * 8 + 2] += __uint_as_float(w[1] << 16) + ba.z;
+                y[c * 8 + 3] += __uint_as_float(w[1] & 0xffff0000u) + ba.w;
+                y[c * 8 + 4] += __uint_as_float(w[2] << 16) + bb.x;
+                y[c * 8 + 5] += __uint_as_float(w[2] & 0xffff0000u) + bb.y;
+                y[c * 8 + 6] += __uint_as_float(w[3] << 16) + bb.z;
+                y[c * 8 + 7] += __uint_as_float(w[3] & 0xffff0000u) + bb.w;
+            }
+            // mean and sum of squared deviations of the half-row, merged with the other half-row's
+            float m = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) m += y[j];
+            m *= (1.0f / 64.0f);
+            float m2 = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) m2 += (y[j] - m) * (y[j] - m);
+            st_shared_f2(sA2 + (uint32_t)((ln * 2 + cg) * 8), m, m2);
+            __syncthreads();
+            float mo, m2o;
+            ld_shared_f2(sA2 + (uint32_t)((ln * 2 + (cg ^ 1)) * 8), mo, m2o);
+            __syncthreads();
+            const float mean = 0.5f * (m + mo);
+            const float var = (m2 + m2o + 32.0f * (m - mo) * (m - mo)) * (1.0f / 128.0f);
+            const float rstd = rsqrtf(var + p.eps);
+            const float4* gv = reinterpret_cast<const float4*>(p.gamma + cg * 64);
+            const float4* bv = reinterpret_cast<const float4*>(p.beta + cg * 64);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 ga = __ldg(gv + 2 * c), gb = __ldg(gv + 2 * c + 1);
+                const float4 ba = __ldg(bv + 2 * c), bb = __ldg(bv + 2 * c + 1);
+                uint32_t w[4];
+                w[0] = pack_bf16((y[c * 8 + 0] - mean) * rstd * ga.x + ba.x, (y[c * 8 + 1] - mean) * rstd * ga.y + ba.y);
+                w[1] = pack_bf16((y[c * 8 + 2] - mean) * rstd * ga.z + ba.z, (y[c * 8 + 3] - mean) * rstd * ga.w + ba.w);
+                w[2] = pack_bf16((y[c * 8 + 4] - mean) * rstd * gb.x + bb.x, (y[c * 8 + 5] - mean) * rstd * gb.y + bb.y);
+                w[3] = pack_bf16((y[c * 8 + 6] - mean) * rstd * gb.z + bb.z, (y[c * 8 + 7] - mean) * rstd * gb.w + bb.w);
+                st_shared_v4(sA2 + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
+            }
+        }
+        fence_proxy_async_smem();
+        const bool stop = __syncthreads_or(failed ? 1 : 0) != 0;   // also: the X stage may be refilled from here on
+        if (tid == 0 && !stop) {
+            tma_store_2d(&map_y, 0, tile * kTileM, sA2);
+            tma_store_2d(&map_y, 64, tile * kTileM, sA2 + kHalf);
+            bulk_commit();
+        }
+        if (stop) {
+            if (tid == 0 && p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
+            break;
+        }
+    }
+    if (tid == 0) bulk_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ---- row-wise layer normalisation: one warp per row, four columns per lane -------------------------
+__global__ void __launch_bounds__(256)
+layernorm_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, float eps, __nv_bfloat16* __restrict__ Y, int64_t ldy, int n) {
+    const int lane = threadIdx.x & 31;
+    const int warps = (int)((gridDim.x * blockDim.x) >> 5);
+    const float4 g4 = __ldg(reinterpret_cast<const float4*>(gamma) + lane);
+    const float4 b4 = __ldg(reinterpret_cast<const float4*>(beta) + lane);
+    for (int row = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); row < n; row += warps) {
+        const uint2 w = *reinterpret_cast<const uint2*>(X + (size_t)row * ldx + lane * 4);
+        float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
+        float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
+        float sum = x0 + x1 + x2 + x3;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float mean = sum * (1.0f / 128.0f);
+        x0 -= mean; x1 -= mean; x2 -= mean; x3 -= mean;
+        float sq = x0 * x0 + x1 * x1 + x2 * x2 + x3 * x3;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        const float rstd = rsqrtf(sq * (1.0f / 128.0f) + eps);
+        uint2 out;
+        out.x = pack_bf16(x0 * rstd * g4.x + b4.x, x1 * rstd * g4.y + b4.y);
+        out.y = pack_bf16(x2 * rstd * g4.z + b4.z, x3 * rstd * g4.w + b4.w);
+        *reinterpret_cast<uint2*>(Y + (size_t)row * ldy + lane * 4) = out;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+std::mutex g_mu;
+EncodeTiledFn g_encode = nullptr;
+bool g_attr_set[64] = {};
+int g_sm_count[64] = {};
+
+// [rows, cols] bf16 row-major with leading dimension ld; box = 64 columns x 128 rows, 128-byte swizzle
+dg4_status make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+            if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+                cudaGetLastError();
+                DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+            }
+            g_encode = (EncodeTiledFn)fn;
+        }
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)(ld * 2)};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) DG4_FAIL(DG4_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return DG4_OK;
+}
+
+bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+
+dg4_status check_rows(const char* name, const void* p, int64_t ld) {
+    if (!p) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is null", name);
+    if (!aligned16(p)) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    if (ld < 128) DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimension of %s (%lld) is below 128", name, (long long)ld);
+    if ((ld * 2) % 16 != 0)
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimension of %s (%lld elements) is not a multiple of 16 bytes", name, (long long)ld);
+    return DG4_OK;
+}
+
+dg4_status check_vec(const char* name, const float* p) {
+    if (!p) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is null", name);
+    if (!aligned16(p)) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    return DG4_OK;
+}
+
+dg4_status check_common(const dg4_graph* g, const dg4_desc* desc, float eps) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    if (!desc) DG4_FAIL(DG4_ERR_INVALID_ARG, "null descriptor");
+    if (desc->d != 128) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d = %d: only d = 128 is supported", desc->d);
+    if (desc->dtype != DG4_BF16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the block's dense parts are bf16 only");
+    if (!(eps >= 0.0f) || eps > 3.0e38f) DG4_FAIL(DG4_ERR_INVALID_ARG, "eps must be finite and not negative");
+    return DG4_OK;
+}
+
+#define CHECK(expr) do { dg4_status _s = (expr); if (_s != DG4_OK) return _s; } while (0)
+
+}  // namespace
+
+extern "C" dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
+                                         const float* gamma, const float* beta, float eps, void* Y, int64_t ldy,
+                                         void* stream) {
+    CHECK(check_common(g, desc, eps));
+    CHECK(check_rows("X", X, ldx));
+    CHECK(check_rows("Y", Y, ldy));
+    CHECK(check_vec("gamma", gamma));
+    CHECK(check_vec("beta", beta));
+    if (g->n == 0) return DG4_OK;
+    const int blocks = (int)std::min<int64_t>(((int64_t)g->n + 7) / 8, 148 * 8);
+    layernorm_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, ldx, gamma, beta, eps,
+                                                                (__nv_bfloat16*)Y, ldy, g->n);
+    DG4_CUDA_TRY(cudaGetLastError());
+    dg4i_count_launch();
+    return DG4_OK;
+}
+
+extern "C" dg4_status dg4_ffn_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx, const void* W1,
+                                   const float* b1, const void* W2, const float* b2, const float* gamma,
+                                   const float* beta, float eps, int32_t d_ff, void* Y, int64_t ldy, void* stream) {
+    CHECK(check_common(g, desc, eps));
+    if (d_ff != 512) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d_ff = %d: only d_ff = 4 d = 512 is supported", d_ff);
+    CHECK(check_rows("X", X, ldx));
+    CHECK(check_rows("Y", Y, ldy));
+    if (!W1 || !W2) DG4_FAIL(DG4_ERR_INVALID_ARG, "null weight matrix");
+    if (!aligned16(W1) || !aligned16(W2)) DG4_FAIL(DG4_ERR_INVALID_ARG, "weight matrices must be 16-byte aligned");
+    CHECK(check_vec("b1", b1));
+    CHECK(check_vec("b2", b2));
+    CHECK(check_vec("gamma", gamma));
+    CHECK(check_vec("beta", beta));
+    if (g->n == 0) return DG4_OK;
+    int dev = 0;
+    DG4_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_attr_set[dev]) {
+            DG4_CUDA_TRY(cudaFuncSetAttribute(ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            DG4_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+            g_attr_set[dev] = true;
+        }
+    }
+    CUtensorMap map_x, map_w2, map_y;
+    CHECK(make_map(&map_x, X, g->n, 128, ldx));
+    CHECK(make_map(&map_w2, W2, 128, 512, 512));
+    CHECK(make_map(&map_y, Y, g->n, 128, ldy));
+    FfnParams p;
+    p.W1 = (const __nv_bfloat16*)W1; p.b1 = b1; p.b2 = b2; p.gamma = gamma; p.beta = beta; p.eps = eps;
+    p.n_tiles = (g->n + kTileM - 1) / kTileM;
+    p.status = g->dev_status;
+    const int grid = std::min(p.n_tiles, g_sm_count[dev]);
+    ffn_kernel<<<grid, kThreads, kSmemBytes, (cudaStream_t)stream>>>(map_x, map_w2, map_y, p);
+    DG4_CUDA_TRY(cudaGetLastError());
+    dg4i_count_launch();
+    return DG4_OK;
+}
+
+extern "C" dg4_status dg4_block_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, const void* H_in, int64_t ldh,
+                                              const void* W_qkv, const void* W_o, const float* ln1_gamma,
+                                              const float* ln1_beta, const void* W1, const float* b1, const void* W2,
+                                              const float* b2, const float* ln2_gamma, const float* ln2_beta, float eps,
+                                              int32_t d_ff, void* H_out, int64_t ldho, void* workspace,
+                                              size_t workspace_bytes, void* stream) {
+    CHECK(check_common(g, desc, eps));
+    if (!workspace) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
+    if ((((uintptr_t)workspace) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+    if (workspace_bytes < dg4_layer_workspace_bytes(g, desc))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", workspace_bytes,
+                 dg4_layer_workspace_bytes(g, desc));
+    if (d_ff != 512) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d_ff = %d: only d_ff = 4 d = 512 is supported", d_ff);
+    // workspace rows: Q [n,128] | K|V [n,256] | O [n,128]; the Q table is free once the attention has run and
+    // then holds the attention sub-layer's output
+    __nv_bfloat16* Q = (__nv_bfloat16*)workspace;
+    __nv_bfloat16* KV = Q + (size_t)g->n * 128;
+    __nv_bfloat16* O = Q + (size_t)g->n * 384;
+    __nv_bfloat16* H1 = Q;
+    dg4_desc with_res = *desc;
+    with_res.flags |= DG4_FLAG_RESIDUAL;     // the block always has its residual connections
+    CHECK(dg4_qkv_project(g, desc, H_in, ldh, W_qkv, Q, 128, KV, 256, KV + 128, 256, stream));
+    CHECK(dg4_sparse_attn_fwd(g, desc, Q, 128, KV, 256, KV + 128, 256, O, 128, stream));
+    CHECK(dg4_out_project(g, &with_res, O, 128, W_o, H_in, ldh, H1, 128, stream));
+    CHECK(dg4_layernorm_fwd(g, desc, H1, 128, ln1_gamma, ln1_beta, eps, H1, 128, stream));
+    return dg4_ffn_fwd(g, desc, H1, 128, W1, b1, W2, b2, ln2_gamma, ln2_beta, eps, d_ff, H_out, ldho, stream);
+}

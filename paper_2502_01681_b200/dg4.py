@@ -40,6 +40,7 @@ EXPORTS = [
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
     "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
+    "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel",
 ]
 
 
@@ -129,6 +130,14 @@ def load():
     lib.dg4_layer_fwd_parallel_static.argtypes = [vp, dp, vp, i64, vp, vp, vp, i64, vp]
     lib.dg4_static_max_nodes.restype = ctypes.c_int64
     lib.dg4_static_max_nodes.argtypes = []
+    cf = ctypes.c_float
+    lib.dg4_layernorm_fwd.restype = ctypes.c_int
+    lib.dg4_layernorm_fwd.argtypes = [vp, dp, vp, i64, vp, vp, cf, vp, i64, vp]
+    lib.dg4_ffn_fwd.restype = ctypes.c_int
+    lib.dg4_ffn_fwd.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32, vp, i64, vp]
+    lib.dg4_block_fwd_parallel.restype = ctypes.c_int
+    lib.dg4_block_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
+                                           vp, i64, vp, ctypes.c_size_t, vp]
     _lib = lib
     return lib
 
@@ -304,6 +313,28 @@ def dg4_sparse_attn_additive_fwd(g: Graph, dsc: dg4_desc, S_dst, S_src, negative
     assert S_dst.is_contiguous() and S_src.is_contiguous()
     _check(load().dg4_sparse_attn_additive_fwd(g.handle, ctypes.byref(dsc), _ptr(S_dst), _ptr(S_src),
                                                float(negative_slope), _ptr(V), _ld(V), _ptr(O), _ld(O), _stream(stream)))
+
+
+def dg4_layernorm_fwd(g: Graph, dsc: dg4_desc, X, gamma, beta, eps, Y, stream=None):
+    _check(load().dg4_layernorm_fwd(g.handle, ctypes.byref(dsc), _ptr(X), _ld(X), _ptr(gamma), _ptr(beta),
+                                    ctypes.c_float(eps), _ptr(Y), _ld(Y), _stream(stream)))
+
+
+def dg4_ffn_fwd(g: Graph, dsc: dg4_desc, X, W1, b1, W2, b2, gamma, beta, eps, Y, stream=None):
+    """Y = LayerNorm(X + max(0, X W1^T + b1) W2^T + b2); W1 [512, 128] and W2 [128, 512] bf16, vectors fp32."""
+    _check(load().dg4_ffn_fwd(g.handle, ctypes.byref(dsc), _ptr(X), _ld(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
+                              _ptr(gamma), _ptr(beta), ctypes.c_float(eps), int(W1.shape[0]), _ptr(Y), _ld(Y),
+                              _stream(stream)))
+
+
+def dg4_block_fwd_parallel(g: Graph, dsc: dg4_desc, H_in, W_qkv, W_o, ln1_gamma, ln1_beta, W1, b1, W2, b2, ln2_gamma,
+                           ln2_beta, eps, H_out, workspace, stream=None):
+    """One whole block (attention sub-layer, LayerNorm, feed-forward sub-layer, LayerNorm) on all nodes at once."""
+    _check(load().dg4_block_fwd_parallel(g.handle, ctypes.byref(dsc), _ptr(H_in), _ld(H_in), _ptr(W_qkv), _ptr(W_o),
+                                         _ptr(ln1_gamma), _ptr(ln1_beta), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
+                                         _ptr(ln2_gamma), _ptr(ln2_beta), ctypes.c_float(eps), int(W1.shape[0]),
+                                         _ptr(H_out), _ld(H_out), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def dg4_graph_partition(g: Graph, delta: int):
