@@ -349,6 +349,31 @@ def run_ours(args, w):
         add_bytes = (256.0 + 4 * w.heads + 36.0) * n + (256.0 + 4 * w.heads) * info.n_nbr
         extras = {"attn_additive_ms": add_ms, "attn_additive_algorithmic_gbs": add_bytes / (add_ms * 1e-3) / 1e9}
         del s_dst, s_src
+        # the rest of the Transformer block on the same rows: feed-forward sub-layer (fused, tensor cores) and LayerNorm
+        w1 = (torch.randn(512, 128, device="cuda") * 0.05).to(torch.bfloat16)
+        w2 = (torch.randn(128, 512, device="cuda") * 0.05).to(torch.bfloat16)
+        b1, b2 = torch.randn(512, device="cuda") * 0.1, torch.randn(128, device="cuda") * 0.1
+        gam, bet = torch.ones(128, device="cuda"), torch.zeros(128, device="cuda")
+
+        def timed3(fn):
+            for _ in range(2):
+                fn()
+            t0, t1 = ev(), ev()
+            t0.record(stream)
+            for _ in range(3):
+                fn()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / 3
+
+        ffn_ms = timed3(lambda: dg4.dg4_ffn_fwd(gr, dsc, x_dev, w1, b1, w2, b2, gam, bet, 1e-5, o_v))
+        ln_ms = timed3(lambda: dg4.dg4_layernorm_fwd(gr, dsc, x_dev, gam, bet, 1e-5, o_v))
+        blk_ms = timed3(lambda: dg4.dg4_block_fwd_parallel(gr, dsc, x_dev, wq[0], wo[0], gam, bet, w1, b1, w2, b2, gam,
+                                                           bet, 1e-5, h_par, ws))
+        extras.update({"ffn_ms": ffn_ms, "ffn_tflops": 4.0 * 128 * 512 * n / (ffn_ms * 1e-3) / 1e12,
+                       "layernorm_ms": ln_ms, "layernorm_gbs": 512.0 * n / (ln_ms * 1e-3) / 1e9,
+                       "block_parallel_ms": blk_ms})
+        del w1, w2
 
     # ---- end to end through the C ABI from host buffers -----------------------------------------
     e2e_steps = max(1, min(2, args.steps))

@@ -42,7 +42,7 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr int kColD1 = 0, kColD2 = 128, kColW1 = 256, kTmemCols = 512;
 
 struct Misc {
-    uint64_t bar_w, bar_x[2], bar_mma;
+    uint64_t bar_w, bar_x[2], bar_g1, bar_g2;
     uint32_t tmem_base;
 };
 
@@ -57,9 +57,6 @@ struct FfnParams {
     int32_t* status;
 };
 
-__device__ __forceinline__ void st_shared_b16(uint32_t addr, uint16_t v) {
-    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
 }
@@ -79,6 +76,16 @@ __device__ __forceinline__ uint16_t bf16_bits(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
 }
+// max(0, lo) and max(0, hi) rounded to bf16 in one conversion, stored as two 16-bit values
+__device__ __forceinline__ void relu_pack_store2(uint32_t addr_lo, uint32_t addr_hi, float lo, float hi) {
+    asm volatile(
+        "{\n\t.reg .b32 pk;\n\t.reg .b16 l, h;\n\t"
+        "cvt.rn.relu.bf16x2.f32 pk, %3, %2;\n\t"
+        "mov.b32 {l, h}, pk;\n\t"
+        "st.shared.b16 [%0], l;\n\t"
+        "st.shared.b16 [%1], h;\n\t}"
+        ::"r"(addr_lo), "r"(addr_hi), "f"(lo), "f"(hi) : "memory");
+}
 // byte offset of element k (0..127) of row `row` in a 128-row operand tile (two K-halves, 128-byte swizzle)
 __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
     return (uint32_t)((k >> 6) * kHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
@@ -94,7 +101,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
     const uint32_t sW2 = base + kOffW2, sX = base + kOffX, sA2 = base + kOffA2;
-    const uint32_t bar_w = smem_u32(&misc->bar_w), bar_mma = smem_u32(&misc->bar_mma);
+    const uint32_t bar_w = smem_u32(&misc->bar_w), bar_g1 = smem_u32(&misc->bar_g1), bar_g2 = smem_u32(&misc->bar_g2);
     const uint32_t bar_x[2] = {smem_u32(&misc->bar_x[0]), smem_u32(&misc->bar_x[1])};
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int q4 = warp & 3, cg = warp >> 2;             // TMEM lane quadrant of the warp; which half of the columns it takes
@@ -106,7 +113,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         mbar_init(bar_w, 1);
         mbar_init(bar_x[0], 1);
         mbar_init(bar_x[1], 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_g1, 1);
+        mbar_init(bar_g2, 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w2);
@@ -145,8 +153,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
     tc_fence_after();
 
     const uint32_t idesc = idesc_bf16_f32(128, 128);
+    uint32_t a2_base[8];                                 // where this thread's hidden unit lies in rows cg*64 + (0..7)
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a2_base[k] = sA2 + operand_offset(cg * 64 + k, ln) - (uint32_t)(k * 128);
     const uint64_t dA2 = smem_desc_sw128(sA2);
-    uint32_t ph_mma = 0;
+    uint32_t ph_g1 = 0, ph_g2 = 0;
     bool failed = false;
     if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0);
 
@@ -173,30 +184,39 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         if (tid == 0) {
             tc_fence_after();
             issue_g1(0);
-            mma_commit(bar_mma);
+            mma_commit(bar_g1);
         }
 
+        // Per block q of hidden units: the accumulator is read into registers, the next block's first product is
+        // issued at once (it runs while the values are scattered into the operand buffer), then the second
+        // product of this block.  The tensor pipe executes in issue order: G1(0) G1(1) G2(0) G1(2) G2(1) ...
         for (int q = 0; q < 4; ++q) {
-            failed |= !mbar_wait(bar_mma, ph_mma);       // D1^T of block q is complete (and so is everything before it)
-            ph_mma ^= 1u;
+            failed |= !mbar_wait(bar_g1, ph_g1);         // D1^T of block q is complete
+            ph_g1 ^= 1u;
             tc_fence_after();
-            if (q == 0) {                                // the previous tile's store must have read the staging buffer
-                if (tid == 0) bulk_wait_read0();
-                __syncthreads();
-            }
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t d[32];
-                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + half * 32), d);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int row = cg * 64 + half * 32 + j;
-                    const float u = fmaxf(__uint_as_float(d[j]) + b1v[q], 0.0f);
-                    st_shared_b16(sA2 + operand_offset(row, ln), bf16_bits(u));
-                }
-            }
+            uint32_t d[64];
+            tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64), d);
+            tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + 32), d + 32);
+            tmem_ld_wait();
             tc_fence_before();
+            if (q == 0 && tid == 0) bulk_wait_read0();   // the previous tile's store has read the staging buffer
+            __syncthreads();                             // every thread holds its part of D1^T
+            if (tid == 0 && q < 3) {
+                tc_fence_after();
+                issue_g1(q + 1);
+                mma_commit(bar_g1);
+            }
+            if (q > 0) {                                 // the previous block's second product has read the buffer
+                failed |= !mbar_wait(bar_g2, ph_g2);
+                ph_g2 ^= 1u;
+            }
+            // rows cg*64 + j: element `ln` of row j lies at a2_base[j & 7] + 128 j (the swizzle depends on j & 7
+            // only, because cg*64 is a multiple of 8); two rows per conversion, ReLU folded into it
+            const float bq = b1v[q];
+#pragma unroll
+            for (int j = 0; j < 64; j += 2)
+                relu_pack_store2(a2_base[j & 7] + (uint32_t)(j * 128), a2_base[(j + 1) & 7] + (uint32_t)((j + 1) * 128),
+                                 __uint_as_float(d[j]) + bq, __uint_as_float(d[j + 1]) + bq);
             fence_proxy_async_smem();
             __syncthreads();
             if (tid == 0) {
@@ -205,12 +225,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)           // D2 += A2 * W2_q^T
                     mma_bf16(tmem + kColD2, dA2 + kstep(ks), dW2 + kstep(ks), idesc, (q > 0 || ks > 0) ? 1u : 0u);
-                if (q < 3) issue_g1(q + 1);
-                mma_commit(bar_mma);
+                mma_commit(bar_g2);
             }
         }
-        failed |= !mbar_wait(bar_mma, ph_mma);           // D2 is complete; the activation buffer is free
-        ph_mma ^= 1u;
+        failed |= !mbar_wait(bar_g2, ph_g2);             // D2 is complete; the activation buffer is free
+        ph_g2 ^= 1u;
         tc_fence_after();
 
         // ---- final epilogue: thread = row `ln`, columns cg*64 .. cg*64+63
@@ -291,31 +310,51 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
     }
 }
 
-// ---- row-wise layer normalisation: one warp per row, four columns per lane -------------------------
+// ---- row-wise layer normalisation: half a warp per row, eight columns (16 bytes) per lane -----------
 __global__ void __launch_bounds__(256)
-layernorm_kernel(const __nv_bfloat16* __restrict__ X, int64_t ldx, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, float eps, __nv_bfloat16* __restrict__ Y, int64_t ldy, int n) {
-    const int lane = threadIdx.x & 31;
-    const int warps = (int)((gridDim.x * blockDim.x) >> 5);
-    const float4 g4 = __ldg(reinterpret_cast<const float4*>(gamma) + lane);
-    const float4 b4 = __ldg(reinterpret_cast<const float4*>(beta) + lane);
-    for (int row = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); row < n; row += warps) {
-        const uint2 w = *reinterpret_cast<const uint2*>(X + (size_t)row * ldx + lane * 4);
-        float x0 = __uint_as_float(w.x << 16), x1 = __uint_as_float(w.x & 0xffff0000u);
-        float x2 = __uint_as_float(w.y << 16), x3 = __uint_as_float(w.y & 0xffff0000u);
-        float sum = x0 + x1 + x2 + x3;
+layernorm_kernel(const __nv_bfloat16* X, int64_t ldx, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, float eps, __nv_bfloat16* Y, int64_t ldy, int n) {   // Y may be X
+    const int sub = threadIdx.x & 15;
+    const int groups = (int)((gridDim.x * blockDim.x) >> 4);
+    const float4 ga = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * sub), gb = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * sub + 1);
+    const float4 ba = __ldg(reinterpret_cast<const float4*>(beta) + 2 * sub), bb = __ldg(reinterpret_cast<const float4*>(beta) + 2 * sub + 1);
+    const int first = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 4);
+    // whole warps stay in the loop together (the shuffles name all 32 lanes): rows are dealt two per warp, and
+    // every half-warp keeps four rows in flight
+    const int hw = (threadIdx.x >> 4) & 1;
+    for (int base_row = first - hw; base_row < n; base_row += 4 * groups) {
+        uint4 w[4];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        const float mean = sum * (1.0f / 128.0f);
-        x0 -= mean; x1 -= mean; x2 -= mean; x3 -= mean;
-        float sq = x0 * x0 + x1 * x1 + x2 * x2 + x3 * x3;
+        for (int i = 0; i < 4; ++i) {
+            const int row = base_row + hw + i * groups;
+            w[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (row < n) w[i] = *reinterpret_cast<const uint4*>(X + (size_t)row * ldx + sub * 8);
+        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-        const float rstd = rsqrtf(sq * (1.0f / 128.0f) + eps);
-        uint2 out;
-        out.x = pack_bf16(x0 * rstd * g4.x + b4.x, x1 * rstd * g4.y + b4.y);
-        out.y = pack_bf16(x2 * rstd * g4.z + b4.z, x3 * rstd * g4.w + b4.w);
-        *reinterpret_cast<uint2*>(Y + (size_t)row * ldy + lane * 4) = out;
+        for (int i = 0; i < 4; ++i) {
+            const int row = base_row + hw + i * groups;
+            float x[8] = {__uint_as_float(w[i].x << 16), __uint_as_float(w[i].x & 0xffff0000u), __uint_as_float(w[i].y << 16),
+                          __uint_as_float(w[i].y & 0xffff0000u), __uint_as_float(w[i].z << 16), __uint_as_float(w[i].z & 0xffff0000u),
+                          __uint_as_float(w[i].w << 16), __uint_as_float(w[i].w & 0xffff0000u)};
+            float sum = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sum += x[j];
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const float mean = sum * (1.0f / 128.0f);
+            float sq = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { x[j] -= mean; sq += x[j] * x[j]; }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+            const float rstd = rsqrtf(sq * (1.0f / 128.0f) + eps);
+            uint4 out;
+            out.x = pack_bf16(x[0] * rstd * ga.x + ba.x, x[1] * rstd * ga.y + ba.y);
+            out.y = pack_bf16(x[2] * rstd * ga.z + ba.z, x[3] * rstd * ga.w + ba.w);
+            out.z = pack_bf16(x[4] * rstd * gb.x + bb.x, x[5] * rstd * gb.y + bb.y);
+            out.w = pack_bf16(x[6] * rstd * gb.z + bb.z, x[7] * rstd * gb.w + bb.w);
+            if (row < n) *reinterpret_cast<uint4*>(Y + (size_t)row * ldy + sub * 8) = out;
+        }
     }
 }
 
@@ -393,7 +432,7 @@ extern "C" dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc
     CHECK(check_vec("gamma", gamma));
     CHECK(check_vec("beta", beta));
     if (g->n == 0) return DG4_OK;
-    const int blocks = (int)std::min<int64_t>(((int64_t)g->n + 7) / 8, 148 * 8);
+    const int blocks = (int)std::min<int64_t>(((int64_t)g->n + 15) / 16, 148 * 8);
     layernorm_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, ldx, gamma, beta, eps,
                                                                 (__nv_bfloat16*)Y, ldy, g->n);
     DG4_CUDA_TRY(cudaGetLastError());
