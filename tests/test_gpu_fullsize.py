@@ -147,3 +147,38 @@ def test_config4_full_size_levelised_prefix():
     g = w.graph()
     assert int(g.level.max()) + 1 == 501
     _levelised_prefix_check(w, g, g.n_pi + 12 * w.gates_per_level, w.layers)
+
+
+def test_block_dense_parts_at_full_size_sampled_rows():
+    """The feed-forward kernel and the LayerNorm kernel on the 10M-row workload, in the launch configuration the
+    benchmark's extras time.  Rows are independent, so the checker recomputes a sample of them: the first and last
+    rows of the first, a middle and the (ragged) last tile, and 2 000 rows drawn at random."""
+    w = synth.workload(5)
+    n = w.n
+    rp = np.zeros(n + 1, np.int32)
+    g = dg4.dg4_graph_create(rp, np.zeros(0, np.int32), np.zeros(n, np.int32), 1, 0)
+    dsc = dg4.desc(8, dg4.DG4_BF16, 0.25)
+    x = torch.randn(n, 128, device="cuda", generator=torch.Generator(device="cuda").manual_seed(5)).to(torch.bfloat16)
+    w1_bits, w1 = bf16_weights(synth.normal_f32(41, 1, (512, 128), 0.08))
+    w2_bits, w2 = bf16_weights(synth.normal_f32(41, 2, (128, 512), 0.08))
+    vec = [synth.normal_f32(41, 3 + i, (k,), 0.3).astype(np.float32) for i, k in enumerate((512, 128, 128, 128))]
+    vec[2] = vec[2] + np.float32(1.0)
+    b1, b2, gam, bet = vec
+    dv = [torch.from_numpy(v).cuda() for v in vec]
+    y = torch.empty_like(x)
+    dg4.dg4_ffn_fwd(g, dsc, x, dev_bf16(w1_bits), dv[0], dev_bf16(w2_bits), dv[1], dv[2], dv[3], 1e-5, y)
+    z = torch.empty_like(x)
+    dg4.dg4_layernorm_fwd(g, dsc, x, dv[2], dv[3], 1e-5, z)
+    torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(g) == 0
+    rng = np.random.default_rng(17)
+    last_tile = (n - 1) // 128 * 128
+    rows = np.unique(np.concatenate([[0, 127, 128, 5_000_063, 5_000_064, last_tile, n - 1], rng.integers(0, n, 2000)]))
+    idx = torch.from_numpy(rows).cuda()
+    xs = host_f64_of_bf16(x[idx])
+    want = orc.ffn(xs, w1, b1, w2, b2, gam, bet, eps=1e-5, rounding="bf16")
+    assert rel_row_err(host_f64_of_bf16(y[idx]), want).max() <= BF16_ROW_TOL
+    want_ln = orc.round_bf16(orc.layernorm(xs, gam, bet, 1e-5))
+    assert rel_row_err(host_f64_of_bf16(z[idx]), want_ln).max() <= BF16_ROW_TOL
+    # every row was written: a LayerNorm output row is never all zero with these beta
+    assert bool((z.abs().amax(dim=1) > 0).all()) and bool((y.abs().amax(dim=1) > 0).all())
