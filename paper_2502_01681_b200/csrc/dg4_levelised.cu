@@ -239,14 +239,17 @@ levelised_kernel(LevParams p) {
         const int tiles = (n_l + kTile - 1) / kTile;
         if (n_l > 0 && bid < tiles) {
             bool waited = false;
+            int v_nx = -1, pad_nx = 0;           // index chain of this CTA's next tile in a wide level
             for (int tile = bid; tile < tiles; tile += nctas) {
                 int v, pad;
                 if (tile == bid) {
                     v = v0; pad = pad0;
-                } else {                         // further tiles of a wide level: plain dependent loads
-                    const int r = tile * kTile + slot;
-                    v = (r < n_l) ? p.level_nodes[first + r] : -1;
-                    pad = pad_of(v);
+                } else {                         // further tiles of a wide level: fetched during the tile before
+                    v = v_nx; pad = pad_nx;
+                }
+                {
+                    const int r = (tile + nctas) * kTile + slot;
+                    v_nx = (tile + nctas < tiles && r < n_l) ? p.level_nodes[first + r] : -1;
                 }
                 const bool valid = v >= 0;
 
@@ -294,6 +297,7 @@ levelised_kernel(LevParams p) {
                 }
                 if (!valid || !p.residual) hres.w[0] = hres.w[1] = hres.w[2] = hres.w[3] = 0u;
                 attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, gmask, acc);
+                pad_nx = pad_of(v_nx);           // its node id has arrived by now; the entry is used by the next tile
                 {
                     Piece o = Elem<true>::pack(acc);
                     st_shared_v4(sO + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), o.w);
