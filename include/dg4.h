@@ -120,7 +120,9 @@ int64_t dg4_launch_count(void);
  *   device      CUDA ordinal; made current for the duration of the call and restored
  *   out         receives the handle; untouched on error
  *
- * Allocates device memory and synchronises; not for use inside a timed or captured region.
+ * Allocates device memory and returns when the handle is complete; not for use inside a captured region.  Its
+ * uploads and kernels run on a stream of their own: the call neither waits for nor delays work the caller has in
+ * flight on other streams (cones of more than two hops are the exception: that path synchronises the device).
  * Errors: INVALID_ARG, NOT_SORTED, BAD_DEGREE, BAD_LEVEL, UNSUPPORTED, ALLOC, CUDA.
  */
 dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, const int32_t* col_idx,

@@ -496,7 +496,15 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     TRY_ALLOC(g->hist, g->hist_len);
     TRY_ALLOC(g->block_sums, g->block_sums_len);
     TRY_ALLOC(g->dev_status, 1);
-    if (cudaMemset(g->dev_status, 0, sizeof(int32_t)) != cudaSuccess) { dg4_set_error("cudaMemset failed"); return fail(DG4_ERR_CUDA); }
+    // Uploads and the prep kernels run on a stream of their own that does not wait for (or hold up) the work the
+    // caller has in flight on other streams; it is drained before the handle is returned.
+    struct PrepStream {
+        cudaStream_t st = nullptr;
+        ~PrepStream() { if (st) cudaStreamDestroy(st); }
+    } prep;
+    if (cudaStreamCreateWithFlags(&prep.st, cudaStreamNonBlocking) != cudaSuccess) { dg4_set_error("cudaStreamCreate failed"); return fail(DG4_ERR_CUDA); }
+    const cudaStream_t st = prep.st;
+    if (cudaMemsetAsync(g->dev_status, 0, sizeof(int32_t), st) != cudaSuccess) { dg4_set_error("cudaMemset failed"); return fail(DG4_ERR_CUDA); }
 
     auto cuda_fail = [&](cudaError_t e, const char* what) {
         dg4_set_error("%s failed: %s", what, cudaGetErrorString(e));
@@ -504,28 +512,31 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
         return DG4_ERR_CUDA;
     };
     cudaError_t ce;
-    if ((ce = cudaMemcpy(g->row_ptr, row_ptr, (size_t)(n + 1) * 4, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(ce, "upload of row_ptr");
-    if (n_edges > 0 && (ce = cudaMemcpy(g->col_idx, col_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(ce, "upload of col_idx");
-    if ((ce = cudaMemcpy(g->level, level, (size_t)n * 4, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(ce, "upload of level");
+    if ((ce = cudaMemcpyAsync(g->row_ptr, row_ptr, (size_t)(n + 1) * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "upload of row_ptr");
+    if (n_edges > 0 && (ce = cudaMemcpyAsync(g->col_idx, col_idx, (size_t)n_edges * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "upload of col_idx");
+    if ((ce = cudaMemcpyAsync(g->level, level, (size_t)n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "upload of level");
 
     // sizes first, so that nbr_idx can be allocated exactly
     if (g->wide) {
+        if ((ce = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ce, "upload");
         if ((s = dg4i_build_wide_cones(g)) != DG4_OK) return fail(s);
     } else {
-        if ((s = dg4i_graph_device_pass(g, 0, true)) != DG4_OK) return fail(s);
+        if ((s = dg4i_graph_device_pass(g, st, true)) != DG4_OK) return fail(s);
         int32_t total = 0;
-        if ((ce = cudaMemcpy(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
+        if ((ce = cudaMemcpyAsync(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
+        if ((ce = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ce, "neighbourhood sizes");
         g->n_nbr = total;
         TRY_ALLOC(g->nbr_idx, g->n_nbr);
         TRY_ALLOC(g->nbr_pad, n * g->pad_width);
     }
 #undef TRY_ALLOC
-    if ((s = dg4i_graph_device_pass(g, 0, false)) != DG4_OK) return fail(s);
+    if ((s = dg4i_graph_device_pass(g, g->wide ? (cudaStream_t)0 : st, false)) != DG4_OK) return fail(s);
 
     g->h_level_ptr = (int32_t*)malloc(((size_t)g->n_levels + 1) * sizeof(int32_t));
     if (!g->h_level_ptr) { dg4_set_error("host allocation failed"); return fail(DG4_ERR_ALLOC); }
-    if ((ce = cudaMemcpy(g->h_level_ptr, g->level_ptr, ((size_t)g->n_levels + 1) * 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(ce, "read of level_ptr");
-    if ((ce = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(ce, "graph prep");
+    if (g->wide && (ce = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(ce, "graph prep");
+    if ((ce = cudaMemcpyAsync(g->h_level_ptr, g->level_ptr, ((size_t)g->n_levels + 1) * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "read of level_ptr");
+    if ((ce = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ce, "graph prep");
     *out = g;
     return DG4_OK;
 }
