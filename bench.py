@@ -385,42 +385,48 @@ def run_ours(args, w):
     d2h = out_host.numel() * 2
     up, down = torch.cuda.Stream(), torch.cuda.Stream()
     out_hosts = [out_host, torch.empty_like(out_host).pin_memory()]
-    keep = []                                             # graphs and tensors stay alive until the pipeline has drained
+    x_slots = [torch.empty_like(x_dev), torch.empty_like(x_dev)]      # device buffers of two steps in flight
+    hp = torch.empty_like(x_dev)
+    drained = [None, None]                                # read-back of the step that last used a slot
 
-    def stage_in():
+    def stage_in(i):
         with torch.cuda.stream(up):
-            x2 = x_host.cuda(non_blocking=True).view(torch.bfloat16)
+            if drained[i % 2] is not None:
+                up.wait_event(drained[i % 2])
+            x_slots[i % 2].view(torch.int16).copy_(x_host, non_blocking=True)
             arrived = torch.cuda.Event()
             arrived.record(up)
         gr2 = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local)
-        return x2, gr2, arrived
+        return x_slots[i % 2], gr2, arrived
 
+    # one untimed round fills the library's memory pool, as a serving loop's first request would
+    for gr2 in [dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local) for _ in range(2)]:
+        dg4.dg4_graph_destroy_async(gr2, stream)
     barrier()
     t0 = time.perf_counter()
-    staged = stage_in()
+    staged = stage_in(0)
     for i in range(e2e_steps):
         x2, gr2, arrived = staged
         stream.wait_event(arrived)
-        hp = x2.clone()
+        hp.copy_(x2)
         for l in range(w.layers):
             dg4.dg4_layer_fwd_parallel(gr2, dsc, hp, wq[l], wo[l], hp, ws)
         if not args.no_levelised:
             dg4.dg4_layers_fwd_levelised(gr2, dsc, x2, wq, wo, ws, status)
         done = torch.cuda.Event()
         done.record(stream)
+        dg4.dg4_graph_destroy_async(gr2, stream)          # freed once this step's kernels have run
         with torch.cuda.stream(down):
             down.wait_event(done)
             out_hosts[i % 2].copy_(x2.view(torch.int16), non_blocking=True)
-        keep.append((x2, hp, gr2))
+            drained[i % 2] = torch.cuda.Event()
+            drained[i % 2].record(down)
         if i + 1 < e2e_steps:
-            staged = stage_in()
+            staged = stage_in(i + 1)
     torch.cuda.synchronize()
     barrier()
     e2e_total_s, e2e_units = reduce_over_ranks(dist, "cuda", time.perf_counter() - t0,
                                                float(n) * layer_passes * e2e_steps)
-    for _, _, gr2 in keep:
-        dg4.dg4_graph_destroy(gr2)
-    del keep
     e2e_s = e2e_total_s / e2e_steps
     e2e_value = e2e_units / e2e_total_s
 

@@ -134,7 +134,20 @@ dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, const int32
  * The arrays are unchanged in content; this entry exists so the device pass can be timed on its own. */
 dg4_status dg4_graph_rebuild(dg4_graph* g, void* stream);
 
-dg4_status dg4_graph_destroy(dg4_graph* g);     /* NULL is accepted */
+/* Frees the handle and its device memory; waits for the device (kernels still using the handle finish first).
+ * NULL is accepted. */
+dg4_status dg4_graph_destroy(dg4_graph* g);
+
+/* The same without waiting (the paper has no counterpart): the handle's device memory is released in the order
+ * of `stream`, i.e. after the work enqueued there so far, and goes back to the library's pool, from which later
+ * dg4_graph_create calls are served without a call into the driver that would wait for running kernels.  The
+ * caller guarantees that no other stream still uses the handle.  Handles of cones of more than two hops are freed
+ * as by dg4_graph_destroy.  NULL is accepted. */
+dg4_status dg4_graph_destroy_async(dg4_graph* g, void* stream);
+
+/* Gives the unused part of the library's memory pool on `device` back to the driver (freed handles leave their
+ * memory in the pool for later dg4_graph_create calls).  Waits for the device.  The paper has no counterpart. */
+dg4_status dg4_memory_trim(int32_t device);
 dg4_status dg4_graph_info(const dg4_graph* g, dg4_graph_info_t* out);
 
 /* Copies one index array to the host (synchronises the device).  host_dst may be NULL to query the

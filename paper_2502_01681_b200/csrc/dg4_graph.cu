@@ -9,6 +9,7 @@
 
 #include "dg4_internal.h"
 
+#include <mutex>
 #include <new>
 #include <thread>
 #include <vector>
@@ -361,25 +362,56 @@ struct DeviceGuard {
     }
 };
 
-void free_graph(dg4_graph* g) {
+// Frees the handle.  With `ordered` set, pooled device memory is released in the order of `st` (work enqueued
+// there before may still use it) and nothing waits; otherwise every buffer is released with cudaFree, which
+// waits for the device.
+void free_graph(dg4_graph* g, bool ordered = false, cudaStream_t st = nullptr) {
     if (!g) return;
     int32_t* bufs[] = {g->nbr_pad, g->row_ptr, g->col_idx, g->level, g->nbr_ptr, g->nbr_idx, g->level_ptr, g->level_nodes,
                        g->perm, g->class_ptr, g->level_perm, g->level_class_ptr, g->seq_a, g->seq_b, g->hist,
                        g->block_sums, g->dev_status};
-    for (int32_t* b : bufs)
-        if (b) cudaFree(b);
+    for (int32_t* b : bufs) {
+        if (!b) continue;
+        if (ordered && g->pooled) cudaFreeAsync(b, st);
+        else cudaFree(b);
+    }
     free(g->h_level_ptr);
     delete g;
 }
 
+// The library's own memory pool of a device (handles of cones up to two hops allocate from it in stream order).
+// Freed memory stays in the pool, so that creating a handle while kernels run does not have to ask the driver for
+// new memory (which would wait for them).
+std::mutex g_pool_mu;
+cudaMemPool_t g_pool[64] = {};
+dg4_status device_pool(int dev, cudaMemPool_t* out) {
+    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
+    std::lock_guard<std::mutex> lock(g_pool_mu);
+    if (!g_pool[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t pool = nullptr;
+        DG4_CUDA_TRY(cudaMemPoolCreate(&pool, &props));
+        uint64_t keep = UINT64_MAX;
+        DG4_CUDA_TRY(cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep));
+        g_pool[dev] = pool;
+    }
+    *out = g_pool[dev];
+    return DG4_OK;
+}
+
 template <typename T>
-dg4_status dalloc(T** p, int64_t count) {
+dg4_status dalloc(T** p, int64_t count, cudaMemPool_t pool, cudaStream_t st) {
     if (count < 1) count = 1;
-    cudaError_t e = cudaMalloc((void**)p, (size_t)count * sizeof(T));
+    const size_t bytes = (size_t)count * sizeof(T);
+    cudaError_t e = pool ? cudaMallocFromPoolAsync((void**)p, bytes, pool, st) : cudaMalloc((void**)p, bytes);
     if (e != cudaSuccess) {
         *p = nullptr;
         cudaGetLastError();
-        dg4_set_error("cudaMalloc of %lld bytes failed: %s", (long long)(count * (int64_t)sizeof(T)), cudaGetErrorString(e));
+        dg4_set_error("device allocation of %lld bytes failed: %s", (long long)bytes, cudaGetErrorString(e));
         return DG4_ERR_ALLOC;
     }
     return DG4_OK;
@@ -480,7 +512,21 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
 
     dg4_status s = DG4_OK;
     auto fail = [&](dg4_status code) { free_graph(g); return code; };
-#define TRY_ALLOC(ptr, cnt) if ((s = dalloc(&(ptr), (cnt))) != DG4_OK) return fail(s)
+    // Uploads and the prep kernels run on a stream of their own that does not wait for (or hold up) the work the
+    // caller has in flight on other streams; it is drained before the handle is returned.  Device memory comes
+    // from the library's pool in the order of that stream (plain cudaMalloc for cones of more than two hops).
+    struct PrepStream {
+        cudaStream_t st = nullptr;
+        ~PrepStream() { if (st) cudaStreamDestroy(st); }
+    } prep;
+    if (cudaStreamCreateWithFlags(&prep.st, cudaStreamNonBlocking) != cudaSuccess) { dg4_set_error("cudaStreamCreate failed"); return fail(DG4_ERR_CUDA); }
+    const cudaStream_t st = prep.st;
+    cudaMemPool_t pool = nullptr;
+    if (!g->wide) {
+        if ((s = device_pool(device, &pool)) != DG4_OK) return fail(s);
+        g->pooled = true;
+    }
+#define TRY_ALLOC(ptr, cnt) if ((s = dalloc(&(ptr), (cnt), pool, st)) != DG4_OK) return fail(s)
     TRY_ALLOC(g->row_ptr, n + 1);
     TRY_ALLOC(g->col_idx, n_edges);
     TRY_ALLOC(g->level, n);
@@ -496,14 +542,6 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     TRY_ALLOC(g->hist, g->hist_len);
     TRY_ALLOC(g->block_sums, g->block_sums_len);
     TRY_ALLOC(g->dev_status, 1);
-    // Uploads and the prep kernels run on a stream of their own that does not wait for (or hold up) the work the
-    // caller has in flight on other streams; it is drained before the handle is returned.
-    struct PrepStream {
-        cudaStream_t st = nullptr;
-        ~PrepStream() { if (st) cudaStreamDestroy(st); }
-    } prep;
-    if (cudaStreamCreateWithFlags(&prep.st, cudaStreamNonBlocking) != cudaSuccess) { dg4_set_error("cudaStreamCreate failed"); return fail(DG4_ERR_CUDA); }
-    const cudaStream_t st = prep.st;
     if (cudaMemsetAsync(g->dev_status, 0, sizeof(int32_t), st) != cudaSuccess) { dg4_set_error("cudaMemset failed"); return fail(DG4_ERR_CUDA); }
 
     auto cuda_fail = [&](cudaError_t e, const char* what) {
@@ -551,6 +589,27 @@ extern "C" dg4_status dg4_graph_destroy(dg4_graph* g) {
     if (!g) return DG4_OK;
     DeviceGuard guard(g->device);
     free_graph(g);
+    return DG4_OK;
+}
+
+extern "C" dg4_status dg4_graph_destroy_async(dg4_graph* g, void* stream) {
+    if (!g) return DG4_OK;
+    DeviceGuard guard(g->device);
+    free_graph(g, true, (cudaStream_t)stream);
+    return DG4_OK;
+}
+
+extern "C" dg4_status dg4_memory_trim(int32_t device) {
+    if (device < 0 || device >= 64) DG4_FAIL(DG4_ERR_INVALID_ARG, "device ordinal %d is out of range", device);
+    cudaMemPool_t pool = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_pool_mu);
+        pool = g_pool[device];
+    }
+    if (!pool) return DG4_OK;                 // nothing was ever allocated on this device
+    DeviceGuard guard(device);
+    DG4_CUDA_TRY(cudaDeviceSynchronize());
+    DG4_CUDA_TRY(cudaMemPoolTrimTo(pool, 0));
     return DG4_OK;
 }
 

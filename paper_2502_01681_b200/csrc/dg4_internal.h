@@ -52,6 +52,7 @@ struct dg4_graph {
     int32_t* nbr_pad = nullptr;          // [n, pad_width]: |N(v)|, then the members other than v (filler: v)
     int32_t pad_width = 0;               // max_class + 1 (0 for cones wider than two hops: no table)
     bool wide = false;                   // hops > 2: CSR lists only, no fixed-width table, no class orderings
+    bool pooled = false;                 // device buffers come from the library's stream-ordered pool
     int32_t* level_ptr = nullptr;        // [n_levels+1]
     int32_t* level_nodes = nullptr;      // [n]
     int32_t* perm = nullptr;             // [n]

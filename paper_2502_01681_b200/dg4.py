@@ -40,7 +40,7 @@ EXPORTS = [
     "dg4_out_project", "dg4_layer_workspace_bytes", "dg4_layer_fwd_parallel", "dg4_layer_fwd_levelised",
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
     "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
-    "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel",
+    "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel", "dg4_graph_destroy_async", "dg4_memory_trim",
 ]
 
 
@@ -95,6 +95,10 @@ def load():
     lib.dg4_graph_rebuild.argtypes = [vp, vp]
     lib.dg4_graph_destroy.restype = ctypes.c_int
     lib.dg4_graph_destroy.argtypes = [vp]
+    lib.dg4_graph_destroy_async.restype = ctypes.c_int
+    lib.dg4_graph_destroy_async.argtypes = [vp, vp]
+    lib.dg4_memory_trim.restype = ctypes.c_int
+    lib.dg4_memory_trim.argtypes = [ctypes.c_int32]
     lib.dg4_graph_info.restype = ctypes.c_int
     lib.dg4_graph_info.argtypes = [vp, ctypes.POINTER(dg4_graph_info_t)]
     lib.dg4_graph_export.restype = ctypes.c_int
@@ -156,7 +160,7 @@ def _stream(stream):
     if stream is None:
         import torch
         return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
-    return ctypes.c_void_p(int(stream))
+    return ctypes.c_void_p(int(getattr(stream, "cuda_stream", stream)))     # a raw handle or a torch stream
 
 
 def _ptr(t):
@@ -217,6 +221,17 @@ def dg4_graph_destroy(g: Graph):
     if g.handle:
         _check(load().dg4_graph_destroy(g.handle))
         g.handle = None
+
+
+def dg4_graph_destroy_async(g: Graph, stream=None):
+    """Frees the handle in the order of `stream` (work enqueued there before may still use it); does not wait."""
+    if g.handle:
+        _check(load().dg4_graph_destroy_async(g.handle, _stream(stream)))
+        g.handle = None
+
+
+def dg4_memory_trim(device: int = 0):
+    _check(load().dg4_memory_trim(device))
 
 
 def dg4_graph_info(g: Graph) -> dg4_graph_info_t:

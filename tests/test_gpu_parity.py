@@ -531,3 +531,33 @@ def test_levelised_layers_with_empty_levels():
     for (_, wq, _, wo) in weights:
         want = orc.layer_levelised(want, wq, wo, ptr, idx, lptr, lnodes, 8, 0.25, residual=True, rounding="bf16")
     assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
+
+
+def test_stream_ordered_destroy_and_pooled_create():
+    """A handle freed in stream order right after its kernels were enqueued: the kernels still see intact arrays,
+    and handles created afterwards (served from the library's pool) give the same results."""
+    w = synth.workload(5, 400)
+    g = w.graph()
+    xb = w.x_bf16_bits()
+    wq_bits, _ = bf16_weights(w.w_qkv_f32(0))
+    wo_bits, _ = bf16_weights(w.w_o_f32(0))
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True)
+    outs = []
+    for rep in range(4):
+        gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+        ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+        h = dev_bf16(xb).clone()
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), h, ws)
+        dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), ws, st)
+        dg4.dg4_graph_destroy_async(gr)                    # no wait: the two layers are still queued or running
+        assert gr.handle is None
+        outs.append((h, st))
+    torch.cuda.synchronize()
+    for h, st in outs:
+        assert int(st.item()) == 0
+        assert torch.equal(h, outs[0][0])
+    dg4.dg4_memory_trim(0)                                 # the pool gives its free memory back; later creates still work
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+    assert (dg4.dg4_graph_export(gr, dg4.DG4_ARR_NBR_PTR) == orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)[0]).all()
+    dg4.dg4_graph_destroy(gr)
