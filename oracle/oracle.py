@@ -31,7 +31,9 @@ def build(force: bool = False) -> str:
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
+        # DG4_ORACLE_LIB: used only by tests/test_oracle_mutants.py, which checks that the pins reject deliberately
+        # broken builds of the checker
+        lib = ctypes.CDLL(os.environ.get("DG4_ORACLE_LIB") or build())
         c_int, c_dbl = ctypes.c_int, ctypes.c_double
         lib.orc_round_bf16.restype = c_dbl
         lib.orc_round_bf16.argtypes = [c_dbl]

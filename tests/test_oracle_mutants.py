@@ -1,0 +1,71 @@
+"""Do the pins bite?  Each case plants one plausible mistake in a COPY of the CPU checker's source (a dropped term,
+a wrong sign or index, a transposed operand, a wrong rounding or ordering rule), builds it, and runs the pins that
+are meant to catch that kind of mistake against the broken build: they must fail.  The mistakes are planted in the
+checker, on the CPU; nothing here touches a GPU or the CUDA library."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "dg4_oracle.cpp")
+
+# (name, text in the checker's source, what replaces it, -k expression selecting the pins expected to object)
+MUTANTS = [
+    ("level_without_plus_one", "lv = std::max(lv, level[u] + 1);", "lv = std::max(lv, level[u]);",
+     "levels or fixture or generated"),
+    ("cone_one_hop_short", "for (int step = 0; step < hops; ++step) {", "for (int step = 0; step + 1 < hops; ++step) {",
+     "cones or fixture or neighbourhood or binary"),
+    ("cone_without_self", "total += 1 + (int64_t)cone.size();", "total += (int64_t)cone.size();",
+     "cones or fixture or neighbourhood or binary"),
+    ("cone_only_last_frontier", "for (int u : next) cone.insert(u);", "cone = next;",
+     "cones or fixture or neighbourhood or binary"),
+    ("buckets_descending", "return level[a] < level[b]; });", "return level[a] > level[b]; });", "bucket or level"),
+    ("class_order_ties_by_descending_id", "            return a < b;\n        });", "            return a > b;\n        });",
+     "class"),
+    ("partition_stride_off_by_one", "for (int l = k; l <= L; l += delta)", "for (int l = k; l <= L; l += delta + 1)",
+     "partition"),
+    ("partition_forgets_fanout_free_nodes", "if (out_degree[v] == 0) cones[level[v]].insert(v);", ";", "partition"),
+    ("score_without_scale", "s[j] = scale * dot;", "s[j] = dot;", "attention or closed or dense"),
+    ("score_sign", "s[j] = scale * dot;", "s[j] = -scale * dot;", "attention or closed or dense"),
+    ("softmax_not_normalised", "for (int j = 0; j < cnt; ++j) a[j] /= z;\n    for (int c = 0; c < d_head; ++c) {",
+     "for (int c = 0; c < d_head; ++c) {", "attention or closed or sum"),
+    ("head_slices_of_key_ignored", "kr[j] = K + u * d + h * dh;", "kr[j] = K + u * d;", "attention or dense or heads"),
+    ("value_of_the_destination", "vr[j] = V + u * d + h * dh;", "vr[j] = V + (int64_t)v * d + h * dh;",
+     "attention or closed or dense"),
+    ("additive_without_leaky_slope", "e[j] = x > 0.0 ? x : slope * x;", "e[j] = x;", "additive"),
+    ("projection_transposed", "acc += x[c] * W[(int64_t)o * d_in + c];", "acc += x[c] * W[(int64_t)c * d_out + o];",
+     "project or layer"),
+    ("projection_without_residual", "if (r) acc += r[o];", "", "project or layer or residual"),
+    ("levelised_in_reverse_order", "for (int l = 0; l < n_levels; ++l) {\n        int lo = level_ptr[l], hi = level_ptr[l + 1];",
+     "for (int l = n_levels - 1; l >= 0; --l) {\n        int lo = level_ptr[l], hi = level_ptr[l + 1];", "levelised"),
+    ("bf16_by_truncation", "double r = std::nearbyint(x / q) * q;", "double r = std::trunc(x / q) * q;", "bf16 or rounding"),
+    ("layernorm_unbiased_variance", "        var /= d;\n", "        var /= (d - 1);\n", "layernorm or ffn"),
+    ("layernorm_eps_outside_root", "double rstd = 1.0 / std::sqrt(var + eps);", "double rstd = 1.0 / (std::sqrt(var) + eps);",
+     "layernorm or ffn"),
+    ("layernorm_gamma_beta_swapped", "(x[c] - mean) * rstd * gamma[c] + beta[c];", "(x[c] - mean) * rstd * beta[c] + gamma[c];",
+     "layernorm or ffn"),
+    ("ffn_without_first_bias", "double acc = b1[h];", "double acc = 0.0;", "ffn"),
+    ("ffn_without_relu", "acc = acc > 0.0 ? acc : 0.0;", "", "ffn"),
+    ("ffn_without_residual", "z[o] = x[o] + acc;", "z[o] = acc;", "ffn"),
+    ("ffn_second_matrix_transposed", "acc += u[h] * W2[(int64_t)o * d_ff + h];", "acc += u[h] * W2[(int64_t)h * d + o];", "ffn"),
+]
+
+
+@pytest.fixture(scope="module")
+def source():
+    return open(SRC).read()
+
+
+@pytest.mark.parametrize("name,old,new,pins", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_pins_reject_broken_checker(tmp_path, source, name, old, new, pins):
+    assert source.count(old) == 1, f"the text to replace must occur exactly once ({name})"
+    src = tmp_path / "mutant.cpp"
+    src.write_text(source.replace(old, new))
+    lib = tmp_path / "mutant.so"
+    subprocess.check_call(["g++", "-O1", "-fopenmp", "-shared", "-fPIC", "-w", "-o", str(lib), str(src)])
+    env = dict(os.environ, DG4_ORACLE_LIB=str(lib))
+    run = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"), "-x", "-q",
+                          "-p", "no:cacheprovider", "-k", pins], cwd=ROOT, env=env, capture_output=True, text=True)
+    assert run.returncode == 1, f"the pins did not object to '{name}':\n{run.stdout[-2000:]}"
