@@ -17,7 +17,7 @@
 //     variance of the row combined from the two half-rows, gamma / beta, bf16, staged in shared memory and
 //     written with a TMA store (the last tile is clipped by the tensor map).
 //   The X tile of the next tile is prefetched by TMA while the current one is processed.
-// No cluster multicast anywhere.  Every wait is bounded; after a timeout the kernel records DG4_ERR_TIMEOUT and
+// Every CTA loads its own tiles (no load is shared across CTAs).  Every wait is bounded; after a timeout the kernel records DG4_ERR_TIMEOUT and
 // the CTA leaves its tile loop.
 #include "dg4_internal.h"
 #include "dg4_sm100.cuh"

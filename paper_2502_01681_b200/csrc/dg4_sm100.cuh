@@ -1,5 +1,5 @@
 // Thin wrappers over the Blackwell (sm_100a) instructions the projection kernels use: mbarrier, TMA tensor
-// loads (no multicast), tcgen05 MMA / TMEM allocation / TMEM loads, and the shared-memory matrix descriptor.
+// loads (each into the issuing CTA's own shared memory), tcgen05 MMA / TMEM allocation / TMEM loads, and the shared-memory matrix descriptor.
 // Every wait is bounded: it gives up after a fixed number of polls and reports failure to the caller.
 #pragma once
 
