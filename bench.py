@@ -543,6 +543,21 @@ def run_per_config(args):
                     for _ in range(3):
                         par()
                     r["layer"] = timed(par, 20)
+                    # the workload's whole stack of parallel layers: eager launches, then captured once in a CUDA graph
+                    def stack():
+                        h.copy_(x)
+                        for l in range(w.layers):
+                            dg4.dg4_layer_fwd_parallel(gr, dsc, h, wq[l], wo[l], h, ws)
+                    r["stack"] = timed(stack, 20)
+                    side = torch.cuda.Stream()
+                    side.wait_stream(stream)
+                    cg = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(cg, stream=side):
+                        stack()
+                    stream.wait_stream(side)
+                    cg.replay()
+                    r["stack_graph"] = timed(cg.replay, 20)
+                    del cg
                 if "levelised" in w.modes:
                     lev = lambda: dg4.dg4_layers_fwd_levelised(gr, dsc, h, wq, wo, ws, status)
                     h.copy_(x)
@@ -581,13 +596,15 @@ def run_per_config(args):
             print(f"| {r['cfg']} {r['name']} ({r['dtype']}) | {r['n']} | {r['n_nbr']} | {r['levels']} | {r['create_ms']:.2f} "
                   f"| {r['prep_ms']:.3f} | {r['warm'][0]:.4f} / {r['warm'][1]:.4f} | {r['cold'][0]:.4f} / {r['cold'][1]:.4f} "
                   f"| {r['n'] / t:.3e} | {gbs:.0f} | {100 * gbs / peak:.0f} % | {100 * gbs / 8000:.0f} % |")
-        print("\n| cfg | parallel layer (QKV + attention + output) | levelised, all layers in one launch | per layer "
+        print("\n| cfg | parallel layer (QKV + attention + output) | all parallel layers, eager launches | the same as one "
+              "CUDA graph | levelised, all layers in one launch | per layer "
               "| us per wavefront step (levels + layers - 1 steps) | levelised, one layer as per-level launches |")
-        print("|---|---:|---:|---:|---:|---:|")
+        print("|---|---:|---:|---:|---:|---:|---:|---:|")
         for r in rows:
             if "layer" in r or "lev" in r:
                 L = synth.workload(r["cfg"]).layers
-                lay = f"{r['layer'][0]:.3f} / {r['layer'][1]:.3f}" if "layer" in r else "-"
+                lay = (f"{r['layer'][0]:.3f} / {r['layer'][1]:.3f} | {r['stack'][0]:.3f} / {r['stack'][1]:.3f} "
+                       f"| {r['stack_graph'][0]:.3f} / {r['stack_graph'][1]:.3f}") if "layer" in r else "- | - | -"
                 if "lev" in r:
                     lev = (f"{r['lev'][0]:.2f} / {r['lev'][1]:.2f} | {r['lev'][0] / L:.2f} "
                            f"| {1e3 * r['lev'][0] / (r['levels'] + L - 1):.2f} | {r['lev_launches'][0]:.1f}")

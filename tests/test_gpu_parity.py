@@ -561,3 +561,46 @@ def test_stream_ordered_destroy_and_pooled_create():
     gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
     assert (dg4.dg4_graph_export(gr, dg4.DG4_ARR_NBR_PTR) == orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)[0]).all()
     dg4.dg4_graph_destroy(gr)
+
+
+@pytest.mark.parametrize("mode", ["parallel", "levelised"])
+def test_forward_calls_can_be_captured_in_a_cuda_graph(mode):
+    """The forward calls only enqueue work on the caller's stream (no allocation, no synchronisation), so a stack
+    of layers can be captured once and replayed: the launch-bound small circuits need that."""
+    w = synth.workload(2, 10)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+    weights = _weights(w, 3)
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True)
+    ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, 3)),
+                     dtype=torch.uint8, device="cuda")
+    x = dev_bf16(w.x_bf16_bits())
+    wq = [dev_bf16(t[0]) for t in weights]
+    wo = [dev_bf16(t[2]) for t in weights]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    h = torch.empty_like(x)
+
+    def run():
+        h.copy_(x)
+        if mode == "parallel":
+            for l in range(3):
+                dg4.dg4_layer_fwd_parallel(gr, dsc, h, wq[l], wo[l], h, ws)
+        else:
+            dg4.dg4_layers_fwd_levelised(gr, dsc, h, wq, wo, ws, status)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run()                                              # first calls outside the capture (one-off function attributes)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager = h.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        run()
+    for _ in range(2):
+        h.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(h, eager)
+    assert int(status.item()) == 0
