@@ -182,3 +182,44 @@ def test_block_dense_parts_at_full_size_sampled_rows():
     assert rel_row_err(host_f64_of_bf16(z[idx]), want_ln).max() <= BF16_ROW_TOL
     # every row was written: a LayerNorm output row is never all zero with these beta
     assert bool((z.abs().amax(dim=1) > 0).all()) and bool((y.abs().amax(dim=1) > 0).all())
+
+
+def test_eight_hop_cones_at_full_size_sampled_rows():
+    """The paper's cone depth (k = 8) on the 10M-node circuit: 1.6e9 list entries.  The checker recomputes sampled
+    nodes from the circuit itself: their cone by plain set expansion (size against the exported row pointers) and
+    their attention row over that cone."""
+    w = synth.workload(5)
+    g = w.graph()
+    n = g.n
+    hops, heads, scale = 8, 8, 0.25
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, hops, 0)
+    info = dg4.dg4_graph_info(gr)
+    ptr = dg4.dg4_graph_export(gr, dg4.DG4_ARR_NBR_PTR)
+    assert ptr[0] == 0 and int(ptr[-1]) == info.n_nbr and info.n_nbr > 1_000_000_000
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    q, k, v = ((torch.randn(n, 128, device="cuda", generator=gen) * s).to(torch.bfloat16) for s in (0.5, 0.5, 1.0))
+    o = torch.empty_like(q)
+    dg4.dg4_sparse_attn_fwd(gr, dg4.desc(heads, dg4.DG4_BF16, scale), q, k, v, o)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(23)
+    samples = np.unique(np.concatenate([[0, w.n_pi, n - 1], rng.integers(0, n, 150)]))
+    lists = [cone_list(g, int(s), hops) for s in samples]
+    for s, lst in zip(samples, lists):
+        assert int(ptr[s + 1] - ptr[s]) == len(lst), int(s)
+    members = sorted(set(u for lst in lists for u in lst))
+    pos = {u: i for i, u in enumerate(members)}
+    midx = torch.from_numpy(np.array(members, np.int64)).cuda()
+    kk, vv = host_f64_of_bf16(k[midx]), host_f64_of_bf16(v[midx])
+    qq = np.zeros_like(kk)
+    sel = np.array([pos[int(s)] for s in samples])
+    qq[sel] = host_f64_of_bf16(q[torch.from_numpy(samples).cuda()])
+    cptr, cidx = [0], []                  # compact problem: sampled nodes keep their cones, the others only themselves
+    lst_of = {int(s): lst for s, lst in zip(samples, lists)}
+    for u in members:
+        for m in lst_of.get(u, [u]):
+            cidx.append(pos[m])
+        cptr.append(len(cidx))
+    want = orc.round_bf16(orc.attention(qq, kk, vv, np.array(cptr, np.int32), np.array(cidx, np.int32), heads, scale))
+    got = host_f64_of_bf16(o[torch.from_numpy(samples).cuda()])
+    assert rel_row_err(got, want[sel]).max() <= BF16_ROW_TOL
+    dg4.dg4_graph_destroy(gr)
