@@ -125,7 +125,9 @@ def run_reference(args, w):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(w),
+            "config": dict(workload_config(w), sample_nodes=int(prob[0].n), sample_levels=int(len(prob[3]) - 1),
+                           sample=("each step runs the CPU checker on a circuit of sample_nodes nodes drawn by this "
+                                   "workload's generator, not on the full n_pi + n_gates nodes")),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -382,9 +384,10 @@ def run_ours(args, w):
     # second stream, and the result of step i-1 drains on a third one.
     e2e_steps = max(2, min(4, args.steps))
     h2d = x_host.numel() * 2 + (g.row_ptr.nbytes + g.col_idx.nbytes + g.level.nbytes)
-    d2h = out_host.numel() * 2
+    d2h = out_host.numel() * 2 * (1 if args.no_levelised else 2)      # the parallel and the levelised result
     up, down = torch.cuda.Stream(), torch.cuda.Stream()
     out_hosts = [out_host, torch.empty_like(out_host).pin_memory()]
+    out_par_host = torch.empty_like(out_host).pin_memory()
     x_slots = [torch.empty_like(x_dev), torch.empty_like(x_dev)]      # device buffers of two steps in flight
     hp = torch.empty_like(x_dev)
     drained = [None, None]                                # read-back of the step that last used a slot
@@ -403,14 +406,24 @@ def run_ours(args, w):
     for gr2 in [dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0, local) for _ in range(2)]:
         dg4.dg4_graph_destroy_async(gr2, stream)
     barrier()
+    par_drained = None
     t0 = time.perf_counter()
     staged = stage_in(0)
     for i in range(e2e_steps):
         x2, gr2, arrived = staged
         stream.wait_event(arrived)
+        if par_drained is not None:
+            stream.wait_event(par_drained)                # the previous step's parallel result has left `hp`
         hp.copy_(x2)
         for l in range(w.layers):
             dg4.dg4_layer_fwd_parallel(gr2, dsc, hp, wq[l], wo[l], hp, ws)
+        par_done = torch.cuda.Event()
+        par_done.record(stream)
+        with torch.cuda.stream(down):                     # the parallel result drains while the levelised layers run
+            down.wait_event(par_done)
+            out_par_host.copy_(hp.view(torch.int16), non_blocking=True)
+            par_drained = torch.cuda.Event()
+            par_drained.record(down)
         if not args.no_levelised:
             dg4.dg4_layers_fwd_levelised(gr2, dsc, x2, wq, wo, ws, status)
         done = torch.cuda.Event()
@@ -418,7 +431,8 @@ def run_ours(args, w):
         dg4.dg4_graph_destroy_async(gr2, stream)          # freed once this step's kernels have run
         with torch.cuda.stream(down):
             down.wait_event(done)
-            out_hosts[i % 2].copy_(x2.view(torch.int16), non_blocking=True)
+            if not args.no_levelised:
+                out_hosts[i % 2].copy_(x2.view(torch.int16), non_blocking=True)
             drained[i % 2] = torch.cuda.Event()
             drained[i % 2].record(down)
         if i + 1 < e2e_steps:
@@ -444,10 +458,12 @@ def run_ours(args, w):
                          "frac_of_nominal_8000": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": alg_bytes,
                          "unique_row_floor_bytes": 4.0 * 256 * n + 4.0 * (info.n_nbr + n),
-                         "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.shrink == 1 else None},
+                         "traffic": TRAFFIC["bytes_per_node"] * n if args.shrink == 1 and TRAFFIC["bytes_per_node"] else None,
+                         "traffic_source": TRAFFIC},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
-                    "note": "steps pipelined: upload of step i+1 and read-back of step i-1 overlap the compute of step i"},
+                    "note": "steps pipelined: upload of step i+1 and read-back of step i-1 overlap the compute of step i; "
+                            "both results (parallel and levelised stack) are read back every step"},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
@@ -618,9 +634,12 @@ def run_per_config(args):
             print(f"| {r['cfg']} | {r['cpu_n']} | {r['cpu_threads']} | {r['cpu_s']:.3f} | {r['cpu_n'] / r['cpu_s']:.3e} |")
 
 
-# DRAM bytes (read + write) of one sparse_attn_kernel launch on the full workload, from the ncu capture
-# summarised under profiles/; None while no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = 16.60e9   # 4.149 GB at a quarter of the nodes (profiles/), scaled by the node count
+# DRAM bytes (read + write) per node of one launch of the roofline kernel, from the ncu capture summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch / the nodes of that launch; traffic per
+# node does not depend on the circuit's size because the window distribution does not).  "bytes_per_node" must be
+# set to None whenever the kernel named here changes, until its counters have been taken again.
+TRAFFIC = {"kernel": "sparse_attn_kernel<true, 2, 7>", "capture": "profiles/sparse_attn_kernel_cfg5_quarter.md",
+           "capture_nodes": 2_512_500, "capture_dram_bytes": 4.149e9, "bytes_per_node": 4.149e9 / 2_512_500}
 
 
 def main():

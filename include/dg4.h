@@ -14,7 +14,9 @@
  *   - Tensors are row-major [rows, d] with a leading dimension `ld*` in ELEMENTS.
  *     Base pointers must be 16-byte aligned and ld * sizeof(element) a multiple
  *     of 16 bytes, otherwise DG4_ERR_INVALID_ARG.
- *   - d = 128 only.  heads in {1, 2, 4, 8, 16}.  Attention: fp32 or bf16 storage,
+ *   - Every forward call must be made with the handle's device current (DG4_ERR_INVALID_ARG otherwise).
+ *   - d = 128 only.  heads a power of two: 1 .. 16 for bf16 storage, 1 .. 32 for fp32 storage
+ *     (a head must span whole 16-byte pieces of a row).  Attention: fp32 or bf16 storage,
  *     fp32 arithmetic.  Projections: bf16 storage, fp32 accumulation.
  *     Anything else returns DG4_ERR_UNSUPPORTED (there is no fallback path).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
@@ -212,7 +214,9 @@ dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4_desc* desc
                                         const void* V, int64_t ldv, void* O, int64_t ldo, void* stream);
 
 /*
- * Output projection: H_out = O * W_o^T (+ H_res if desc->flags has DG4_FLAG_RESIDUAL and H_res != NULL).
+ * Output projection of the attention sub-layer (Sec. 3.5: the Transformer block around the restricted attention is
+ * kept, and with it the block's output projection and residual connection):
+ * H_out = O * W_o^T (+ H_res if desc->flags has DG4_FLAG_RESIDUAL and H_res != NULL).
  *   O device [n, d] bf16;  W_o device [d, d] bf16 (output-major);  H_res device [n, d] bf16 or NULL;
  *   H_out device [n, d] bf16; may alias H_res (each row is read before it is written by the same thread).
  */
@@ -224,7 +228,8 @@ dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc,
 size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* desc);
 
 /*
- * One layer for all nodes at once: QKV projection -> sparse attention -> output projection (+ residual),
+ * One layer for all nodes at once (Sec. 3.5: the attention sub-layer of the Transformer block with its attention
+ * restricted to cone_k(v)): QKV projection -> sparse attention -> output projection (+ residual),
  * every node reading the same input H_in.   H_in, H_out: device [n, d] bf16; they may be the same buffer
  * only if ldh == ldho (rows are then updated in place after all reads of the layer's input are done).
  */
@@ -247,8 +252,12 @@ dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc* desc,
  *   - Capacity: graphs of at most dg4_static_max_nodes() = 32 768 nodes (1 KiB of scratch per node);
  *     larger graphs are rejected with DG4_ERR_INVALID_ARG and a message naming the limit.
  *   - The graph's device must be current.  The first call on a device looks up the array's device address
- *     (once per device); make that first call outside any stream capture.
- *   - The call allocates nothing and frees nothing, on the host or on the device.
+ *     (once per device), and the driver may instantiate the library's image on that device -- and with it reserve
+ *     the 32 MiB -- only at that moment rather than when the library was loaded.  So make one call per device
+ *     at start-up, before device memory is divided up and outside any stream capture; it can fail with
+ *     DG4_ERR_CUDA if the 32 MiB cannot be had.
+ *   - After that first call, a call takes nothing from the device heap and nothing from the host heap, and
+ *     frees nothing.
  *   - All calls share the one array.  It is never cleared and needs no clearing (a call writes every scratch
  *     row before reading it), but calls that overlap on the GPU -- different streams, or several host
  *     threads -- race on it: run them one after another.
@@ -331,6 +340,24 @@ dg4_status dg4_block_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, cons
  * nothing traps, the context stays usable.  Asynchronous on `stream`.
  */
 dg4_status dg4_selftest_bounded_wait(int32_t* device_status, void* stream);
+
+/*
+ * Diagnostics for the error paths (the paper has no counterpart).
+ *
+ * dg4_debug_set_poll_limit: every device-side wait of the pipelined kernels (projection, feed-forward, levelised)
+ * polls a bounded number of times before it gives up, records DG4_ERR_TIMEOUT in the status word and lets the
+ * kernel wind down (copies and MMAs already started are still waited for, tensor memory is freed, the kernel
+ * returns).  This sets that number for the launches that follow, process-wide; 0 restores the default (about a
+ * second).  A tiny value makes the waits run out at once, which is how the wind-down is exercised without anything
+ * actually being stuck; results of such launches are incomplete by design.
+ *
+ * dg4_debug_override_current_device: every forward call checks that the handle's device is the calling thread's
+ * current CUDA device and returns DG4_ERR_INVALID_ARG otherwise (its kernels would dereference another GPU's
+ * arrays).  This makes that check, on the calling thread, behave as if `device` were current (-1 = off), so the
+ * refusal can be tested on a machine with one GPU.
+ */
+void dg4_debug_set_poll_limit(uint32_t polls);
+void dg4_debug_override_current_device(int32_t device);
 
 #ifdef __cplusplus
 }

@@ -158,30 +158,30 @@ int orc_class_order(int n, const int32_t* seq, int n_seg, const int32_t* seg_ptr
     return 0;
 }
 
-/* Algorithm 1 (graph partition): the roots whose cone_k the partition collects.  Taken step by step: levels
- * l = k, k + delta, ... up to the maximum level contribute every node of that level, in the order the level's
- * nodes are visited (ascending id); then every node without fan-out is added to the group of its own level.
- * A node that qualifies both ways is kept once (the groups are treated as sets of cones).  Output: roots grouped
- * by level, ascending id inside a group; group_ptr[l] = number of roots with level below l (n_levels + 1 entries).
- * The cone of a root r is cone_k(r), i.e. its list in orc_neighbourhood(hops = k).  Returns the number of roots. */
+/* Algorithm 1 (graph partition), stated as the set it produces: a node is the root of a collected cone exactly
+ * when it lies on one of the stride levels (level >= k and (level - k) divisible by delta) or has no fan-out.
+ * The partition groups those cones by the level of their root; a node that qualifies both ways is one cone, not
+ * two (the groups are sets).  Output: the roots ordered by (level, id); group_ptr[l] = number of roots whose
+ * level is below l (n_levels + 1 entries).  The cone of a root r is cone_k(r), i.e. its list in
+ * orc_neighbourhood(hops = k).  Returns the number of roots. */
 int orc_partition_roots(int n, const int32_t* row_ptr, const int32_t* col_idx, const int32_t* level, int n_levels,
                         int k, int delta, int32_t* roots, int32_t* group_ptr) {
-    std::vector<int> out_degree(n, 0);
-    for (int e = 0; e < row_ptr[n]; ++e) out_degree[col_idx[e]] += 1;
-    std::vector<std::set<int>> cones(n_levels);              /* cones^l, as sets of root ids */
-    const int L = n_levels - 1;
-    for (int l = k; l <= L; l += delta)
-        for (int v = 0; v < n; ++v)
-            if (level[v] == l) cones[l].insert(v);
-    for (int v = 0; v < n; ++v)
-        if (out_degree[v] == 0) cones[level[v]].insert(v);
-    int total = 0;
-    for (int l = 0; l < n_levels; ++l) {
-        group_ptr[l] = total;
-        for (int v : cones[l]) roots[total++] = v;
+    std::vector<char> has_fanout(n, 0);
+    for (int e = 0; e < row_ptr[n]; ++e) has_fanout[col_idx[e]] = 1;
+    std::vector<int32_t> picked;
+    for (int v = 0; v < n; ++v) {
+        const bool on_stride_level = level[v] >= k && (level[v] - k) % delta == 0;
+        if (on_stride_level || !has_fanout[v]) picked.push_back(v);
     }
-    group_ptr[n_levels] = total;
-    return total;
+    /* picked is in ascending id; a stable sort on the level alone therefore orders by (level, id) */
+    std::stable_sort(picked.begin(), picked.end(), [&](int x, int y) { return level[x] < level[y]; });
+    for (size_t i = 0; i < picked.size(); ++i) roots[i] = picked[i];
+    for (int l = 0; l <= n_levels; ++l) {
+        int below = 0;
+        for (int v : picked) below += (level[v] < l);
+        group_ptr[l] = below;
+    }
+    return (int)picked.size();
 }
 
 /* One node, one head of the restricted attention.  q: d_head values; krows[j], vrows[j]: the head's

@@ -10,7 +10,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB = os.path.join(_HERE, "libdg4.so")
 SOURCES = sorted(glob.glob(os.path.join(_HERE, "csrc", "dg4_*.cu")))
-HEADERS = sorted(glob.glob(os.path.join(_HERE, "csrc", "*.h"))) + [os.path.join(_ROOT, "include", "dg4.h")]
+HEADERS = (sorted(glob.glob(os.path.join(_HERE, "csrc", "*.h"))) + sorted(glob.glob(os.path.join(_HERE, "csrc", "*.cuh")))
+           + [os.path.join(_ROOT, "include", "dg4.h")])
 
 
 def nvcc_path() -> str:

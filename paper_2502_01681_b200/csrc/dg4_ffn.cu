@@ -42,7 +42,7 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr int kColD1 = 0, kColD2 = 128, kColW1 = 256, kTmemCols = 512;
 
 struct Misc {
-    uint64_t bar_w, bar_x[2], bar_g1, bar_g2;
+    uint64_t bar_w, bar_x[2], bar_g1, bar_g2, bar_drain;
     uint32_t tmem_base;
 };
 
@@ -55,6 +55,7 @@ struct FfnParams {
     float eps;
     int32_t n_tiles;
     int32_t* status;
+    uint32_t poll_limit;      // polls after which a pipeline wait gives up
 };
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
@@ -115,6 +116,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         mbar_init(bar_x[1], 1);
         mbar_init(bar_g1, 1);
         mbar_init(bar_g2, 1);
+        mbar_init(smem_u32(&misc->bar_drain), 1);
         mbar_fence_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w2);
@@ -159,7 +161,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
     const uint64_t dA2 = smem_desc_sw128(sA2);
     uint32_t ph_g1 = 0, ph_g2 = 0;
     bool failed = false;
-    if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0);
+    if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0, p.poll_limit);
 
     int it = 0;
     for (int tile = first_tile; tile < p.n_tiles; tile += (int)gridDim.x, ++it) {
@@ -174,7 +176,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
             }
         }
-        failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u);
+        failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u, p.poll_limit);
 
         auto issue_g1 = [&](int q) {     // D1^T = W1_q * X^T
 #pragma unroll
@@ -191,7 +193,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         // issued at once (it runs while the values are scattered into the operand buffer), then the second
         // product of this block.  The tensor pipe executes in issue order: G1(0) G1(1) G2(0) G1(2) G2(1) ...
         for (int q = 0; q < 4; ++q) {
-            failed |= !mbar_wait(bar_g1, ph_g1);         // D1^T of block q is complete
+            failed |= !mbar_wait(bar_g1, ph_g1, p.poll_limit);         // D1^T of block q is complete
             ph_g1 ^= 1u;
             tc_fence_after();
             uint32_t d[64];
@@ -207,7 +209,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 mma_commit(bar_g1);
             }
             if (q > 0) {                                 // the previous block's second product has read the buffer
-                failed |= !mbar_wait(bar_g2, ph_g2);
+                failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);
                 ph_g2 ^= 1u;
             }
             // rows cg*64 + j: element `ln` of row j lies at a2_base[j & 7] + 128 j (the swizzle depends on j & 7
@@ -228,7 +230,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 mma_commit(bar_g2);
             }
         }
-        failed |= !mbar_wait(bar_g2, ph_g2);             // D2 is complete; the activation buffer is free
+        failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);    // D2 is complete; the activation buffer is free
         ph_g2 ^= 1u;
         tc_fence_after();
 
@@ -297,7 +299,18 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
             bulk_commit();
         }
         if (stop) {
-            if (tid == 0 && p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
+            // A wait ran out somewhere in this CTA.  Every thread went through the whole tile (nothing above
+            // branches on `failed`), so all of them are here.  Before the CTA may leave, what it started must have
+            // ended: the weight copy, the copies of this tile's and of the prefetched tile's rows, and the MMAs
+            // (these waits keep the default limit: a copy or an MMA that was started does finish).
+            if (tid == 0) {
+                if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
+                mbar_wait(bar_w, 0);
+                mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u);
+                if (tile + (int)gridDim.x < p.n_tiles) mbar_wait(bar_x[s ^ 1], (uint32_t)((it + 1) >> 1) & 1u);
+                mma_commit(smem_u32(&misc->bar_drain));
+                mbar_wait(smem_u32(&misc->bar_drain), 0);
+            }
             break;
         }
     }
@@ -411,7 +424,8 @@ dg4_status check_vec(const char* name, const float* p) {
 }
 
 dg4_status check_common(const dg4_graph* g, const dg4_desc* desc, float eps) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    dg4_status dev_ok = dg4i_check_device(g);
+    if (dev_ok != DG4_OK) return dev_ok;
     if (!desc) DG4_FAIL(DG4_ERR_INVALID_ARG, "null descriptor");
     if (desc->d != 128) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d = %d: only d = 128 is supported", desc->d);
     if (desc->dtype != DG4_BF16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the block's dense parts are bf16 only");
@@ -473,6 +487,7 @@ extern "C" dg4_status dg4_ffn_fwd(const dg4_graph* g, const dg4_desc* desc, cons
     p.W1 = (const __nv_bfloat16*)W1; p.b1 = b1; p.b2 = b2; p.gamma = gamma; p.beta = beta; p.eps = eps;
     p.n_tiles = (g->n + kTileM - 1) / kTileM;
     p.status = g->dev_status;
+    p.poll_limit = dg4i_poll_limit();
     const int grid = std::min(p.n_tiles, g_sm_count[dev]);
     ffn_kernel<<<grid, kThreads, kSmemBytes, (cudaStream_t)stream>>>(map_x, map_w2, map_y, p);
     DG4_CUDA_TRY(cudaGetLastError());

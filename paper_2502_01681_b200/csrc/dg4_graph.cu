@@ -580,7 +580,8 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
 }
 
 extern "C" dg4_status dg4_graph_rebuild(dg4_graph* g, void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    dg4_status dev_ok = dg4i_check_device(g);
+    if (dev_ok != DG4_OK) return dev_ok;
     if (g->wide) DG4_FAIL(DG4_ERR_UNSUPPORTED, "rebuild is available for cones of at most two hops");
     return dg4i_graph_device_pass(g, (cudaStream_t)stream, false);
 }

@@ -27,6 +27,17 @@ void dg4_set_error(const char* fmt, ...);
         return (code);               \
     } while (0)
 
+// ---- argument checks shared by the forward entry points (dg4_layer.cu) -----------------------------
+// INVALID_ARG unless the graph's device is the calling thread's current device: every forward call dereferences
+// the handle's device arrays in its kernels, so a call made with another device current must be refused on the host.
+dg4_status dg4i_check_device(const dg4_graph* g);
+dg4_status dg4i_check_desc(const dg4_desc* d, bool need_bf16);
+dg4_status dg4i_check_tensor(const char* name, const void* p, int64_t ld, int elem_size, int min_ld);
+// Poll limit of the bounded device-side waits (mbarrier phases, level counters) handed to every kernel launch:
+// the built-in default unless dg4_debug_set_poll_limit changed it.
+uint32_t dg4i_poll_limit();
+#define DG4I_DEFAULT_POLL_LIMIT (1u << 24)
+
 // ---- launch accounting (every kernel launch of the library bumps this counter) ------------------
 void dg4i_count_launch(int n = 1);
 

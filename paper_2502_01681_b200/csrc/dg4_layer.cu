@@ -16,11 +16,32 @@
 namespace {
 
 thread_local char g_err[512] = "";
+thread_local int g_device_override = -1;      // dg4_debug_override_current_device
 std::atomic<long long> g_launches{0};
+std::atomic<uint32_t> g_poll_limit{DG4I_DEFAULT_POLL_LIMIT};
 
 bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
-dg4_status check_desc(const dg4_desc* d, bool need_bf16) {
+}  // namespace
+
+dg4_status dg4i_check_device(const dg4_graph* g) {
+    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    int cur = g_device_override;
+    if (cur < 0) DG4_CUDA_TRY(cudaGetDevice(&cur));
+    if (cur != g->device)
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "the graph lives on device %d but device %d is current", g->device, cur);
+    return DG4_OK;
+}
+
+uint32_t dg4i_poll_limit() { return g_poll_limit.load(std::memory_order_relaxed); }
+
+extern "C" void dg4_debug_override_current_device(int32_t device) { g_device_override = device; }
+
+extern "C" void dg4_debug_set_poll_limit(uint32_t polls) {
+    g_poll_limit.store(polls ? polls : DG4I_DEFAULT_POLL_LIMIT, std::memory_order_relaxed);
+}
+
+dg4_status dg4i_check_desc(const dg4_desc* d, bool need_bf16) {
     if (!d) DG4_FAIL(DG4_ERR_INVALID_ARG, "null descriptor");
     if (d->d != 128) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d = %d: only d = 128 is supported", d->d);
     if (d->dtype != DG4_F32 && d->dtype != DG4_BF16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "unknown dtype %d", d->dtype);
@@ -33,7 +54,7 @@ dg4_status check_desc(const dg4_desc* d, bool need_bf16) {
     return DG4_OK;
 }
 
-dg4_status check_tensor(const char* name, const void* p, int64_t ld, int elem_size, int min_ld) {
+dg4_status dg4i_check_tensor(const char* name, const void* p, int64_t ld, int elem_size, int min_ld) {
     if (!p) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is null", name);
     if (!aligned16(p)) DG4_FAIL(DG4_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
     if (ld < min_ld) DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimension of %s (%lld) is below %d", name, (long long)ld, min_ld);
@@ -42,7 +63,11 @@ dg4_status check_tensor(const char* name, const void* p, int64_t ld, int elem_si
     return DG4_OK;
 }
 
+namespace {
+
 #define CHECK(expr) do { dg4_status _s = (expr); if (_s != DG4_OK) return _s; } while (0)
+#define check_desc dg4i_check_desc
+#define check_tensor dg4i_check_tensor
 
 struct Workspace {
     __nv_bfloat16* Q;    // [n, 128]
@@ -118,7 +143,7 @@ extern "C" const char* dg4_status_string(dg4_status s) {
 extern "C" dg4_status dg4_qkv_project(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
                                        const void* W_qkv, void* Q, int64_t ldq, void* K, int64_t ldk, void* V,
                                        int64_t ldv, void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     CHECK(check_desc(desc, true));
     CHECK(check_tensor("X", X, ldx, 2, 128));
     CHECK(check_tensor("W_qkv", W_qkv, 128, 2, 128));
@@ -137,7 +162,7 @@ extern "C" dg4_status dg4_qkv_project(const dg4_graph* g, const dg4_desc* desc, 
 extern "C" dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* desc, const void* Q, int64_t ldq,
                                            const void* K, int64_t ldk, const void* V, int64_t ldv, void* O,
                                            int64_t ldo, void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     CHECK(check_desc(desc, false));
     const int es = desc->dtype == DG4_BF16 ? 2 : 4;
     CHECK(check_tensor("Q", Q, ldq, es, 128));
@@ -152,7 +177,7 @@ extern "C" dg4_status dg4_sparse_attn_fwd(const dg4_graph* g, const dg4_desc* de
 extern "C" dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4_desc* desc, const float* S_dst,
                                                     const float* S_src, float negative_slope, const void* V,
                                                     int64_t ldv, void* O, int64_t ldo, void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     CHECK(check_desc(desc, false));
     if (!S_dst || !S_src) DG4_FAIL(DG4_ERR_INVALID_ARG, "null score array");
     if ((((uintptr_t)S_dst) | ((uintptr_t)S_src)) & 3u) DG4_FAIL(DG4_ERR_INVALID_ARG, "score arrays must be 4-byte aligned");
@@ -170,7 +195,7 @@ extern "C" dg4_status dg4_sparse_attn_additive_fwd(const dg4_graph* g, const dg4
 extern "C" dg4_status dg4_out_project(const dg4_graph* g, const dg4_desc* desc, const void* O, int64_t ldo,
                                        const void* W_o, const void* H_res, int64_t ldh, void* H_out, int64_t ldho,
                                        void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     CHECK(check_desc(desc, true));
     CHECK(check_tensor("O", O, ldo, 2, 128));
     CHECK(check_tensor("W_o", W_o, 128, 2, 128));
@@ -194,7 +219,7 @@ extern "C" size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* 
 namespace {
 dg4_status check_layer_args(const dg4_graph* g, const dg4_desc* desc, const void* H, int64_t ldh, const void* W_qkv,
                             const void* W_o, void* ws, size_t ws_bytes) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     CHECK(check_desc(desc, true));
     CHECK(check_tensor("H", H, ldh, 2, 128));
     CHECK(check_tensor("W_qkv", W_qkv, 128, 2, 128));
@@ -300,7 +325,7 @@ extern "C" dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_des
                                                 int32_t n_layers, const void* const* W_qkv, const void* const* W_o,
                                                 void* workspace, size_t workspace_bytes_, int32_t* device_status,
                                                 void* stream) {
-    if (!g) DG4_FAIL(DG4_ERR_INVALID_ARG, "null graph");
+    CHECK(dg4i_check_device(g));
     if (n_layers < 1 || n_layers > DG4I_MAX_LAYERS)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "n_layers = %d: between 1 and %d layers per call", n_layers, DG4I_MAX_LAYERS);
     if (!W_qkv || !W_o) DG4_FAIL(DG4_ERR_INVALID_ARG, "null weight list");

@@ -63,9 +63,10 @@ static_assert(kWCol0 + 6 * kWCols <= kTmemCols, "tensor memory budget of one CTA
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
 struct Misc {
-    uint64_t mma1, mma2;
+    uint64_t mma1, mma2, drain;
     uint32_t tmem_base;
     int32_t go, go2;
+    int32_t failed;                        // a wait for this CTA's own MMAs ran out: leave at the next level
     int32_t node[kTile];
 };
 
@@ -86,6 +87,7 @@ struct LevParams {
     int32_t* arrive;                       // [n_layers, n_levels], zero on entry
     int32_t* abort_word;                   // zero on entry
     int32_t* status;
+    uint32_t poll_limit;                   // polls after which a wait gives up
 };
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
@@ -127,12 +129,12 @@ __device__ __forceinline__ void give_up(const LevParams& p) {
     if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
 }
 
-// Polls (acquire) until *counter >= target; false on abort or after ~1 s.
-__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word) {
+// Polls (acquire) until *counter >= target; false on abort or after `limit` polls (about a second by default).
+__device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word, uint32_t limit) {
     uint32_t polls = 0;
     while (ld_acquire(counter) < target) {
         ++polls;
-        if (polls > (1u << 22) || ((polls & 63u) == 0 && ld_acquire(abort_word) != 0)) return false;
+        if (polls > limit || ((polls & 63u) == 0 && ld_acquire(abort_word) != 0)) return false;
         if (polls > 64) __nanosleep(32);
     }
     return true;
@@ -164,8 +166,10 @@ levelised_kernel(LevParams p) {
     if (tid == 0) {
         mbar_init(bar1, 1);
         mbar_init(bar2, 1);
+        mbar_init(smem_u32(&misc->drain), 1);
         misc->go = 1;
         misc->go2 = 1;
+        misc->failed = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
@@ -205,6 +209,7 @@ levelised_kernel(LevParams p) {
     uint32_t ph1 = 0, ph2 = 0;
     int last_nonempty = -1, last_participants = 0;
     bool alive = true;
+    const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
 
     const char* kv_tab = (const char*)p.KV[layer];
     const char* q_tab = (const char*)p.Q[layer];
@@ -258,13 +263,14 @@ levelised_kernel(LevParams p) {
                     // (two pollers in different warps, so that both counters are watched at the same time)
                     if (tid == 0) {
                         bool go = true;
-                        if (last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word);
+                        if (misc->failed) go = false;
+                        if (go && last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
                         if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                         if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
                         misc->go = go ? 1 : 0;
                     } else if (tid == 32) {
                         bool go = true;
-                        if (prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word);
+                        if (prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word, counter_limit);
                         if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                         misc->go2 = go ? 1 : 0;
                     }
@@ -317,7 +323,7 @@ levelised_kernel(LevParams p) {
                     }
                     mma_commit(bar1);
                 }
-                if (!mbar_wait(bar1, ph1) && tid == 0) give_up(p);
+                if (!mbar_wait(bar1, ph1, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                 ph1 ^= 1u;
                 tc_fence_after();
                 {
@@ -362,7 +368,7 @@ levelised_kernel(LevParams p) {
                     ld_shared_v4(sHp + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), w4);
                     if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
                 }
-                if (!mbar_wait(bar2, ph2) && tid == 0) give_up(p);
+                if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                 ph2 ^= 1u;
                 tc_fence_after();
                 // accumulator blk (0: K, 1: V, 2: next Q, 3: next K, 4: next V) -> byte offset inside a staging row
@@ -421,6 +427,12 @@ levelised_kernel(LevParams p) {
         lp0 = lp1; lp1 = lp2; lp2 = lp3; lp3 = lp4;
     }
 
+    // Tensor memory is freed below: every MMA this CTA issued must have completed.  Normally each was waited for
+    // right after it was issued; after a wait that ran out, one may still be in flight.
+    if (tid == 0) {
+        mma_commit(smem_u32(&misc->drain));
+        mbar_wait(smem_u32(&misc->drain), 0);
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -498,7 +510,7 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     p.nbr_pad = g->nbr_pad; p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
     p.n_levels = g->n_levels; p.n_layers = n_layers;
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
-    p.abort_word = sync; p.arrive = sync + 16; p.status = status;
+    p.abort_word = sync; p.arrive = sync + 16; p.status = status; p.poll_limit = dg4i_poll_limit();
     const int grid = g_sm_count[dev];
     if (g->max_class <= 3) return launch_heads<3>(desc->heads, p, grid, st);
     return launch_heads<7>(desc->heads, p, grid, st);

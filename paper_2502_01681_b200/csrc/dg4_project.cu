@@ -17,8 +17,13 @@
 // bound by HBM traffic (96 flop per byte for QKV, below the machine's ridge), which is why nothing here tries to
 // raise tensor-pipe occupancy beyond what hides the memory time.
 //
-// Every mbarrier wait is bounded; on expiry the kernel records DG4_ERR_TIMEOUT in the status word, lets all
-// warps run out of their loops, waits for its own outstanding copies, frees tensor memory and returns.
+// Every mbarrier wait is bounded; on expiry the kernel records DG4_ERR_TIMEOUT in the status word and raises an
+// abort flag in shared memory.  Leaving is arranged so that no warp can be left waiting for another one: a wait's
+// result is made uniform across the warp before anything branches on it; the eight epilogue warps, which meet at
+// a named barrier once per item when they store by TMA, take the decision to leave together (one thread samples
+// the flag before that barrier, all read the sample after it); the producer then waits for the tensor copies it
+// has started, the MMA thread for the MMAs it has issued, the storing thread for its stores, and only then is
+// tensor memory freed.
 
 #include "dg4_internal.h"
 #include "dg4_sm100.cuh"
@@ -53,8 +58,10 @@ struct Bars {
     uint64_t r_empty[kStages];
     uint64_t acc_full[kSlots];
     uint64_t acc_empty[kSlots];
+    uint64_t drain;            // error path only: completion of the MMAs still in flight
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t epi_stop[2];      // the epilogue warps' common decision to leave, per item parity
 };
 
 struct ProjParams {
@@ -62,6 +69,7 @@ struct ProjParams {
     int32_t n_blocks;         // n_out / 128
     int32_t n_tiles;
     int32_t* status;          // device status word (nullable)
+    uint32_t poll_limit;      // polls after which a pipeline wait gives up
 };
 
 __device__ __forceinline__ void ld_nc_v4(const void* p, uint32_t* r) {
@@ -111,7 +119,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(smem_u32(&bars->r_empty[s]), kEpiWarps);
         }
         for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&bars->acc_full[s]), 1); mbar_init(smem_u32(&bars->acc_empty[s]), kEpiWarps); }
+        mbar_init(smem_u32(&bars->drain), 1);
         bars->abort_flag = 0;
+        bars->epi_stop[0] = bars->epi_stop[1] = 0;
         mbar_fence_init();
         tma_prefetch_desc(&map_w);
         if (!LISTED) {
@@ -137,14 +147,15 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     tma_load_2d(sW + (j * 2 + h) * kHalfBytes, &map_w, h * 64, j * 128, smem_u32(&bars->w_full));
         }
         int armed = 0;
-        for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
+        for (int i = 0; i < my_tiles; ++i) {
+            if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
             const int tile = blockIdx.x + i * gridDim.x;
             const int s = i % kStages;
             const uint32_t ph = (uint32_t)(i / kStages) & 1u;
-            if (!mbar_wait(smem_u32(&bars->a_empty[s]), ph ^ 1u)) { raise_timeout(bars, p.status); break; }
+            if (!mbar_wait_warp(smem_u32(&bars->a_empty[s]), ph ^ 1u, p.poll_limit)) { raise_timeout(bars, p.status); break; }
             const uint32_t dst = sA + s * kTileBytes;
             if (!LISTED) {
-                if (has_res && !mbar_wait(smem_u32(&bars->r_empty[s]), ph ^ 1u)) { raise_timeout(bars, p.status); break; }
+                if (has_res && !mbar_wait_warp(smem_u32(&bars->r_empty[s]), ph ^ 1u, p.poll_limit)) { raise_timeout(bars, p.status); break; }
                 if (lane == 0) {
                     const uint32_t bar = smem_u32(&bars->a_full[s]);
                     mbar_expect_tx(bar, (uint32_t)(has_res ? 2 * kTileBytes : kTileBytes));
@@ -175,27 +186,30 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[s]));
             }
         }
-        // error path only: do not leave with tensor copies still landing in shared memory
-        if (*abort_flag && lane == 0 && !LISTED) {
+        // do not leave with tensor copies still landing in shared memory: normally the MMAs have consumed them all
+        // long before; after an abort they may not have (these waits keep the default limit: a copy that was
+        // started does land)
+        if (lane == 0) {
             mbar_wait(smem_u32(&bars->w_full), 0);
-            for (int i = (armed > kStages ? armed - kStages : 0); i < armed; ++i)
-                mbar_wait(smem_u32(&bars->a_full[i % kStages]), (uint32_t)(i / kStages) & 1u);
+            if (!LISTED)
+                for (int i = (armed > kStages ? armed - kStages : 0); i < armed; ++i)
+                    mbar_wait(smem_u32(&bars->a_full[i % kStages]), (uint32_t)(i / kStages) & 1u);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16_f32(128, 128);
-            bool ok = mbar_wait(smem_u32(&bars->w_full), 0);
+            bool ok = mbar_wait(smem_u32(&bars->w_full), 0, p.poll_limit);
             if (!ok) raise_timeout(bars, p.status);
             int item = 0;
             for (int i = 0; i < my_tiles && ok && !*abort_flag; ++i) {
                 const int s = i % kStages;
-                if (!mbar_wait(smem_u32(&bars->a_full[s]), (uint32_t)(i / kStages) & 1u)) { raise_timeout(bars, p.status); break; }
+                if (!mbar_wait(smem_u32(&bars->a_full[s]), (uint32_t)(i / kStages) & 1u, p.poll_limit)) { raise_timeout(bars, p.status); break; }
                 tc_fence_after();
                 const uint32_t a_base = sA + s * kTileBytes;
                 for (int j = 0; j < nb; ++j, ++item) {
                     const int slot = item % kSlots;
-                    if (!mbar_wait(smem_u32(&bars->acc_empty[slot]), ((uint32_t)(item / kSlots) & 1u) ^ 1u)) {
+                    if (!mbar_wait(smem_u32(&bars->acc_empty[slot]), ((uint32_t)(item / kSlots) & 1u) ^ 1u, p.poll_limit)) {
                         raise_timeout(bars, p.status); ok = false; break;
                     }
                     tc_fence_after();
@@ -210,6 +224,10 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 mma_commit(smem_u32(&bars->a_empty[s]));   // the stage is free once these MMAs have read it
             }
+            // tensor memory is freed below, so every MMA issued above must have completed (normally the epilogue
+            // has waited for each of them; after an abort it may have left first)
+            mma_commit(smem_u32(&bars->drain));
+            mbar_wait(smem_u32(&bars->drain), 0);
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
@@ -219,8 +237,11 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int my_row = quad * 32 + lane;             // row of the tile held by this thread
         const bool issuer = (ew == 0 && lane == 0);      // the one thread that issues (and waits for) TMA stores
         int item = 0;
-        bool ok = true;
-        for (int i = 0; i < my_tiles && ok && !*abort_flag; ++i) {
+        bool ok = true;          // no wait of this warp has run out (the same for all its lanes)
+        bool stop = false;
+        for (int i = 0; i < my_tiles && !stop; ++i) {
+            // listed rows: the warps of the epilogue never wait for one another, so each may leave on its own
+            if (LISTED && __any_sync(0xffffffffu, *abort_flag != 0)) break;
             const int tile = blockIdx.x + i * gridDim.x;
             const int s = i % kStages;
             const int r_own = tile * kTileM + my_row;
@@ -229,59 +250,72 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int j = 0; j < nb; ++j, ++item) {
                 const int slot = item % kSlots;
                 const uint32_t stage = sStage + (uint32_t)((item & 1) * kTileBytes + half * kHalfBytes);
-                if (!mbar_wait(smem_u32(&bars->acc_full[slot]), (uint32_t)(item / kSlots) & 1u)) {
-                    raise_timeout(bars, p.status); ok = false; break;
+                if (ok && !mbar_wait_warp(smem_u32(&bars->acc_full[slot]), (uint32_t)(item / kSlots) & 1u, p.poll_limit)) {
+                    raise_timeout(bars, p.status);
+                    ok = false;
                 }
-                tc_fence_after();
-                const uint32_t t_addr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
+                if (LISTED && !ok) { stop = true; break; }
                 const bool add_res = (j == 0) && has_res;
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t t_addr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * 128 + half * 64);
 #pragma unroll 1
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t acc[32];
-                    tmem_ld_32x32(t_addr + (uint32_t)(q * 32), acc);
-                    uint32_t res[16];
-                    if (add_res) {
-                        if (!LISTED) {                   // residual tile sits in shared memory in box layout
+                    for (int q = 0; q < 2; ++q) {
+                        uint32_t acc[32];
+                        tmem_ld_32x32(t_addr + (uint32_t)(q * 32), acc);
+                        uint32_t res[16];
+                        if (add_res) {
+                            if (!LISTED) {                   // residual tile sits in shared memory in box layout
 #pragma unroll
-                            for (int c = 0; c < 4; ++c)
-                                ld_shared_v4(sR + (uint32_t)(s * kTileBytes + half * kHalfBytes) + sw128_offset(my_row, q * 4 + c), res + 4 * c);
-                        } else if (rid_own >= 0) {
+                                for (int c = 0; c < 4; ++c)
+                                    ld_shared_v4(sR + (uint32_t)(s * kTileBytes + half * kHalfBytes) + sw128_offset(my_row, q * 4 + c), res + 4 * c);
+                            } else if (rid_own >= 0) {
 #pragma unroll
-                            for (int c = 0; c < 4; ++c) ld_nc_v4(p.a.R + rid_own * p.a.ldr + half * 64 + q * 32 + c * 8, res + 4 * c);
-                        } else {
+                                for (int c = 0; c < 4; ++c) ld_nc_v4(p.a.R + rid_own * p.a.ldr + half * 64 + q * 32 + c * 8, res + 4 * c);
+                            } else {
 #pragma unroll
-                            for (int c = 0; c < 16; ++c) res[c] = 0u;
-                        }
-                    }
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t out[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float lo = __uint_as_float(acc[c * 8 + 2 * e]), hi = __uint_as_float(acc[c * 8 + 2 * e + 1]);
-                            if (add_res) {
-                                lo += __uint_as_float(res[4 * c + e] << 16);
-                                hi += __uint_as_float(res[4 * c + e] & 0xffff0000u);
+                                for (int c = 0; c < 16; ++c) res[c] = 0u;
                             }
-                            out[e] = pack_bf16(lo, hi);
                         }
-                        st_shared_v4(stage + sw128_offset(my_row, q * 4 + c), out);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t out[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float lo = __uint_as_float(acc[c * 8 + 2 * e]), hi = __uint_as_float(acc[c * 8 + 2 * e + 1]);
+                                if (add_res) {
+                                    lo += __uint_as_float(res[4 * c + e] << 16);
+                                    hi += __uint_as_float(res[4 * c + e] & 0xffff0000u);
+                                }
+                                out[e] = pack_bf16(lo, hi);
+                            }
+                            st_shared_v4(stage + sw128_offset(my_row, q * 4 + c), out);
+                        }
                     }
-                }
-                // all tensor-memory (and residual) reads of this item are done: hand the buffers back
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(smem_u32(&bars->acc_empty[slot]));
-                    if (add_res && !LISTED) mbar_arrive(smem_u32(&bars->r_empty[s]));
+                    // all tensor-memory (and residual) reads of this item are done: hand the buffers back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&bars->acc_empty[slot]));
+                        if (add_res && !LISTED) mbar_arrive(smem_u32(&bars->r_empty[s]));
+                    }
                 }
                 if (!LISTED) {
                     // staging -> global by TMA.  The issuer first makes sure the previous item's store has finished
-                    // reading ITS staging buffer (the one the next item will overwrite), then everybody meets.
+                    // reading ITS staging buffer (the one the next item will overwrite) and samples the abort flag;
+                    // then everybody meets, and everybody acts on that one sample: the eight warps go on to the
+                    // next item together or leave together.  (A warp whose own wait ran out keeps coming to this
+                    // barrier, without touching tensor memory, until the common decision says leave: at the
+                    // latest at the next item, because its flag was raised before it arrived here.)
                     fence_proxy_async_smem();
-                    if (issuer) bulk_wait_read0();
+                    if (issuer) {
+                        bulk_wait_read0();
+                        bars->epi_stop[item & 1] = *abort_flag;
+                    }
                     epi_barrier();
+                    stop = reinterpret_cast<volatile uint32_t*>(bars->epi_stop)[item & 1] != 0;
+                    if (stop) break;
                     if (issuer) {
                         const uint32_t src = sStage + (uint32_t)((item & 1) * kTileBytes);
                         tma_store_2d(&map_o.m[j], 0, tile * kTileM, src);
@@ -385,6 +419,7 @@ dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st) {
     p.n_blocks = a.n_out / 128;
     p.n_tiles = (a.rows + kTileM - 1) / kTileM;
     p.status = a.status;
+    p.poll_limit = dg4i_poll_limit();
     CUtensorMap map_a, map_w, map_r;
     OutMaps map_o;
     dg4_status s = make_map(&map_w, a.W, a.n_out, 128);

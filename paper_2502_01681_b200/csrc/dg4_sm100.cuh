@@ -28,13 +28,21 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Polls until the phase with the given parity has completed; false if it has not after ~1 s.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 24); ++i) {
+// Polls until the phase with the given parity has completed; false if it has not after `limit` polls (the
+// default is about a second).  Teardown code that waits for its own copies or MMAs in flight uses the default;
+// the pipelines pass the limit their launch was given.
+constexpr uint32_t kDefaultPollLimit = 1u << 24;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = kDefaultPollLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_test(bar, parity)) return true;
         if (i > 64) __nanosleep(40);
     }
-    return false;
+    return mbar_test(bar, parity);
+}
+// The same for a whole (converged) warp, with one answer for all 32 lanes: true only if every lane saw the phase
+// complete.  Code that follows may then branch on the result and still execute warp-wide instructions together.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, uint32_t limit = kDefaultPollLimit) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit) ? 1 : 0) != 0;
 }
 
 // ---- proxies and tcgen05 fences ----------------------------------------------------------------

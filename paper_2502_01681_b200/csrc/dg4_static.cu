@@ -7,8 +7,9 @@
 // or a latency-critical loop where the implicit device-wide synchronisation of cudaMalloc / cudaFree is
 // not acceptable.  For them the scratch lives in a fixed array that is part of the library image itself.
 //
-// The array is reserved on every GPU that loads the library, from load until the process exits, so it is
-// kept modest: 32 MiB, i.e. circuits of at most 32 768 nodes.  All calls share it and nothing is cleared
+// The array is reserved on every GPU on which the library's image is instantiated (at load, or -- with the
+// driver's lazy loading -- at the first call on that device) until the process exits, so it is kept modest:
+// 32 MiB, i.e. circuits of at most 32 768 nodes.  All calls share it and nothing is cleared
 // between calls -- every byte a call reads it has written itself first (Q, K|V and O rows of all its nodes),
 // so stale contents are harmless -- but two calls that overlap in time on the GPU (different streams, or
 // different host threads) would overwrite each other's intermediates: serialise them.
@@ -51,8 +52,6 @@ dg4_status scratch_for_current_device(int device, void** out) {
     return DG4_OK;
 }
 
-bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
-
 }  // namespace
 
 extern "C" int64_t dg4_static_max_nodes(void) { return kMaxNodes; }
@@ -60,28 +59,24 @@ extern "C" int64_t dg4_static_max_nodes(void) { return kMaxNodes; }
 extern "C" dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg4_desc* desc, const void* H_in,
                                                      int64_t ldh, const void* W_qkv, const void* W_o, void* H_out,
                                                      int64_t ldho, void* stream) {
-    if (!g || !desc || !H_in || !W_qkv || !W_o || !H_out) DG4_FAIL(DG4_ERR_INVALID_ARG, "null pointer argument");
-    if (desc->d != 128 || desc->dtype != DG4_BF16)
-        DG4_FAIL(DG4_ERR_UNSUPPORTED, "the static-scratch layer supports d = 128, bf16 only");
-    if (desc->heads < 1 || desc->heads > 16 || (16 % desc->heads) != 0)
-        DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must be a power of two up to 16", desc->heads);
+    dg4_status s = dg4i_check_device(g);
+    if (s != DG4_OK) return s;
+    if ((s = dg4i_check_desc(desc, true)) != DG4_OK) return s;
+    if (desc->heads > 16) DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must be a power of two up to 16", desc->heads);
     if (g->n > kMaxNodes)
         DG4_FAIL(DG4_ERR_INVALID_ARG,
                  "graph has %d nodes; the static scratch (%zu bytes) holds at most %lld -- use dg4_layer_fwd_parallel "
                  "with a caller-provided workspace", g->n, kScratchBytes, (long long)kMaxNodes);
-    if (!aligned16(H_in) || !aligned16(H_out) || !aligned16(W_qkv) || !aligned16(W_o))
-        DG4_FAIL(DG4_ERR_INVALID_ARG, "tensor base pointers must be 16-byte aligned");
-    if (ldh < 128 || ldho < 128 || (ldh % 8) != 0 || (ldho % 8) != 0)
-        DG4_FAIL(DG4_ERR_INVALID_ARG, "leading dimensions must be >= 128 and a multiple of 8 elements");
+    if ((s = dg4i_check_tensor("H_in", H_in, ldh, 2, 128)) != DG4_OK) return s;
+    if ((s = dg4i_check_tensor("H_out", H_out, ldho, 2, 128)) != DG4_OK) return s;
+    if ((s = dg4i_check_tensor("W_qkv", W_qkv, 128, 2, 128)) != DG4_OK) return s;
+    if ((s = dg4i_check_tensor("W_o", W_o, 128, 2, 128)) != DG4_OK) return s;
     if (H_out == H_in && ldh != ldho) DG4_FAIL(DG4_ERR_INVALID_ARG, "in-place use needs equal leading dimensions");
-    int cur = -1;
-    DG4_CUDA_TRY(cudaGetDevice(&cur));
-    if (cur != g->device || cur < 0 || cur >= kMaxDevices)
-        DG4_FAIL(DG4_ERR_INVALID_ARG, "the graph lives on device %d but device %d is current", g->device, cur);
+    const int cur = g->device;                      // checked above: it is the current device
+    if (cur < 0 || cur >= kMaxDevices) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", cur);
 
     void* base = nullptr;
-    dg4_status s = scratch_for_current_device(cur, &base);
-    if (s != DG4_OK) return s;
+    if ((s = scratch_for_current_device(cur, &base)) != DG4_OK) return s;
 
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
@@ -92,7 +87,7 @@ extern "C" dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg
     dg4i_proj_args p;
     p.A = (const __nv_bfloat16*)H_in; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
     p.out[0] = Q; p.ldo[0] = 128; p.out[1] = KV; p.ldo[1] = 256; p.out[2] = KV + 128; p.ldo[2] = 256;
-    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n;
+    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = g->dev_status;
     if ((s = dg4i_proj_launch(p, st)) != DG4_OK) return s;
 
     dg4i_attn_args a;
@@ -107,6 +102,6 @@ extern "C" dg4_status dg4_layer_fwd_parallel_static(const dg4_graph* g, const dg
     o.A = O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
     o.out[0] = (__nv_bfloat16*)H_out; o.ldo[0] = ldho; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
     o.R = (desc->flags & DG4_FLAG_RESIDUAL) ? (const __nv_bfloat16*)H_in : nullptr; o.ldr = ldh;
-    o.row_list = nullptr; o.first = 0; o.rows = g->n;
+    o.row_list = nullptr; o.first = 0; o.rows = g->n; o.status = g->dev_status;
     return dg4i_proj_launch(o, st);
 }

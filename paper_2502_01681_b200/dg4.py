@@ -41,6 +41,7 @@ EXPORTS = [
     "dg4_layer_fwd_parallel_static", "dg4_static_max_nodes", "dg4_layers_workspace_bytes", "dg4_layers_fwd_levelised",
     "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
     "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel", "dg4_graph_destroy_async", "dg4_memory_trim",
+    "dg4_debug_set_poll_limit", "dg4_debug_override_current_device",
 ]
 
 
@@ -142,6 +143,10 @@ def load():
     lib.dg4_block_fwd_parallel.restype = ctypes.c_int
     lib.dg4_block_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
                                            vp, i64, vp, ctypes.c_size_t, vp]
+    lib.dg4_debug_set_poll_limit.restype = None
+    lib.dg4_debug_set_poll_limit.argtypes = [ctypes.c_uint32]
+    lib.dg4_debug_override_current_device.restype = None
+    lib.dg4_debug_override_current_device.argtypes = [ctypes.c_int32]
     _lib = lib
     return lib
 
@@ -322,6 +327,16 @@ def dg4_layers_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, w
 
 def dg4_selftest_bounded_wait(device_status, stream=None):
     _check(load().dg4_selftest_bounded_wait(_ptr(device_status), _stream(stream)))
+
+
+def dg4_debug_set_poll_limit(polls: int):
+    """Poll limit of the device-side waits for the launches that follow (0 = default); see dg4.h."""
+    load().dg4_debug_set_poll_limit(int(polls))
+
+
+def dg4_debug_override_current_device(device: int):
+    """Makes the forward calls' device check on this thread behave as if `device` were current (-1 = off)."""
+    load().dg4_debug_override_current_device(int(device))
 
 
 def dg4_sparse_attn_additive_fwd(g: Graph, dsc: dg4_desc, S_dst, S_src, negative_slope, V, O, stream=None):

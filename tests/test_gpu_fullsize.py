@@ -4,10 +4,13 @@ provably sufficient:
 
 * all-parallel layers: an output row after L layers depends only on the L-fold neighbourhood closure of its
   node, so sampled rows are recomputed by the checker on the compacted closure;
-* levelised layers: node ids are topological, so the first P nodes form a fan-in-closed sub-circuit whose rows
-  the checker computes on its own (the paper's remark that a gate's embedding depends only on its fan-in
-  region); the GPU result of the full circuit must agree on those rows.
+* levelised layers: the 1M-node workload is compared whole; the 10M-node workload is checked step by step on
+  every row (each node recomputed from the inputs the level order prescribes), end to end on a fan-in-closed
+  prefix (node ids are topological; the paper's remark that a gate's embedding depends only on its fan-in
+  region), and end to end on all rows when DG4_FULL_ORACLE=1 allows the minutes of CPU time.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -16,6 +19,7 @@ from oracle import oracle as orc
 from paper_2502_01681_b200 import dg4, synth
 from tests.gpu_util import bf16_weights, dev_bf16, f64_of_bits, host_f64_of_bf16
 from tests.helpers import rel_row_err
+from tests.levelised_checks import drift_by_level_decile, every_step_check
 
 pytestmark = pytest.mark.gpu
 BF16_ROW_TOL = 2e-2
@@ -109,44 +113,111 @@ def test_config5_full_size_parallel_sampled_rows():
     assert err.max() <= BF16_ROW_TOL, err.max()
 
 
-def _levelised_prefix_check(w, g, prefix_nodes, layers):
+def _levelised_gpu_runs(w, g, layers):
+    """The levelised layers on the GPU at full size: once as `layers` successive single-layer calls (keeping every
+    layer's output), and twice as the one wavefront call the benchmark times.  Returns the per-layer outputs as
+    bf16 bit patterns on the host, after checking that all three runs agree bit for bit (a row read before its
+    level was complete, or a layer overtaking the one below it, would show up as a difference)."""
     gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
     xb = w.x_bf16_bits()
     weights = [bf16_weights(w.w_qkv_f32(l)) + bf16_weights(w.w_o_f32(l)) for l in range(layers)]
     dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True)
-    ws = torch.empty(dg4.dg4_layers_workspace_bytes(gr, dsc, layers), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(dg4.dg4_layers_workspace_bytes(gr, dsc, layers), dg4.dg4_layer_workspace_bytes(gr, dsc)),
+                     dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    h = dev_bf16(xb)
-    dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dev_bf16(w_[0]) for w_ in weights], [dev_bf16(w_[2]) for w_ in weights],
-                                 ws, status)                  # the call the benchmark times
-    torch.cuda.synchronize()
-    assert int(status.item()) == 0
-    sub = g.prefix(prefix_nodes)
-    ptr, idx = orc.neighbourhood(sub.row_ptr, sub.col_idx, w.hops)
-    lptr, lnodes = orc.level_buckets(sub.level)
-    want = f64_of_bits(xb[:prefix_nodes])
+    wq = [dev_bf16(w_[0]) for w_ in weights]
+    wo = [dev_bf16(w_[2]) for w_ in weights]
+    x = dev_bf16(xb)
+    h = x.clone()
+    per_layer = []
+    for l in range(layers):                                 # layer after layer, one call each
+        dg4.dg4_layer_fwd_levelised(gr, dsc, h, wq[l], wo[l], ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        per_layer.append(h.view(torch.int16).cpu().numpy().view(np.uint16))
+    for _ in range(2):                                      # the call the benchmark times, twice
+        h2 = x.clone()
+        dg4.dg4_layers_fwd_levelised(gr, dsc, h2, wq, wo, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(h2.view(torch.int16), h.view(torch.int16))
+        del h2
+    assert dg4.dg4_graph_poll_status(gr) == 0
+    dg4.dg4_graph_destroy(gr)
+    return xb, weights, per_layer
+
+
+def _whole_circuit_checker(g, w, xb, weights, ptr, idx):
+    lptr, lnodes = orc.level_buckets(g.level)
+    want = f64_of_bits(xb)
     for (_, wq, _, wo) in weights:
         want = orc.layer_levelised(want, wq, wo, ptr, idx, lptr, lnodes, w.heads, w.scale, residual=True,
                                    rounding="bf16")
-    got = host_f64_of_bf16(h[:prefix_nodes])
-    err = rel_row_err(got, want)
-    assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
-    # rows beyond the prefix were updated too (not left at their input value)
-    tail = host_f64_of_bf16(h[-1000:])
-    assert np.abs(tail - f64_of_bits(xb[-1000:])).max() > 0
+    return want
 
 
-def test_config5_full_size_levelised_prefix():
-    w = synth.workload(5)
-    g = w.graph()
-    _levelised_prefix_check(w, g, g.n_pi + 30_000, w.layers)
+def _report(name, lines):
+    """Prints a few lines and, if DG4_REPORT_DIR names a directory, also appends them to a text file there."""
+    text = "\n".join(lines)
+    print(text)
+    out = os.environ.get("DG4_REPORT_DIR")
+    if out:
+        os.makedirs(out, exist_ok=True)
+        with open(os.path.join(out, name), "a") as f:
+            f.write(text + "\n")
 
 
-def test_config4_full_size_levelised_prefix():
+def test_config4_full_size_levelised_whole_circuit():
+    """All 1 010 000 rows of the 501-level workload after three levelised layers, against the checker run on the
+    whole circuit."""
     w = synth.workload(4)
     g = w.graph()
     assert int(g.level.max()) + 1 == 501
-    _levelised_prefix_check(w, g, g.n_pi + 12 * w.gates_per_level, w.layers)
+    xb, weights, per_layer = _levelised_gpu_runs(w, g, w.layers)
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    want = _whole_circuit_checker(g, w, xb, weights, ptr, idx)
+    err = rel_row_err(f64_of_bits(per_layer[-1]), want)
+    drift = drift_by_level_decile(g.level, err)
+    _report("levelised_drift.txt", [f"cfg4 whole circuit, {w.layers} layers: max row error {err.max():.3e}; "
+                                    "per tenth of the levels: " + " ".join(f"{d:.2e}" for d in drift)])
+    assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
+
+
+def test_config5_full_size_levelised_every_step():
+    """The 10 050 000-node, 17 357-level workload in the launch the benchmark times.  (1) The wavefront call, run
+    twice, and three successive single-layer calls agree bit for bit.  (2) Layer 1: every row is recomputed by the
+    checker from the inputs the level order prescribes (see every_step_check); layers 2 and 3: every eighth row
+    and the last 4 096 rows.  (3) End to end, the fan-in-closed prefix of the first 80 000 nodes against the
+    checker run on that prefix.  (4) With DG4_FULL_ORACLE=1 (minutes of CPU time): all rows against the checker
+    run on the whole circuit, with the error by tenth of the level range."""
+    w = synth.workload(5)
+    g = w.graph()
+    n = g.n
+    xb, weights, per_layer = _levelised_gpu_runs(w, g, w.layers)
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    ins = [xb] + per_layer[:-1]
+    worst = []
+    for l, (_, wq, _, wo) in enumerate(weights):
+        rows = np.arange(n) if l == 0 else np.unique(np.concatenate([np.arange(0, n, 8), np.arange(n - 4096, n)]))
+        err = every_step_check(ptr, idx, rows, ins[l], per_layer[l], wq, wo, w.heads, w.scale)
+        worst.append(float(err.max()))
+        assert err.max() <= BF16_ROW_TOL, (l, err.max(), int(rows[err.argmax()]))
+    _report("levelised_drift.txt", ["cfg5 step-by-step check, max row error per layer: " +
+                                    " ".join(f"{e:.2e}" for e in worst)])
+    # end to end on a fan-in-closed prefix (ids are topological)
+    p = g.n_pi + 30_000
+    sub = g.prefix(p)
+    sptr, sidx = orc.neighbourhood(sub.row_ptr, sub.col_idx, w.hops)
+    want = _whole_circuit_checker(sub, w, xb[:p], weights, sptr, sidx)
+    err = rel_row_err(f64_of_bits(per_layer[-1][:p]), want)
+    assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
+    if os.environ.get("DG4_FULL_ORACLE") == "1":
+        want = _whole_circuit_checker(g, w, xb, weights, ptr, idx)
+        err = rel_row_err(f64_of_bits(per_layer[-1]), want)
+        drift = drift_by_level_decile(g.level, err)
+        _report("levelised_drift.txt", [f"cfg5 whole circuit, {w.layers} layers: max row error {err.max():.3e}; "
+                                        "per tenth of the levels: " + " ".join(f"{d:.2e}" for d in drift)])
+        assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
 
 
 def test_block_dense_parts_at_full_size_sampled_rows():

@@ -25,9 +25,12 @@ MUTANTS = [
     ("buckets_descending", "return level[a] < level[b]; });", "return level[a] > level[b]; });", "bucket or level"),
     ("class_order_ties_by_descending_id", "            return a < b;\n        });", "            return a > b;\n        });",
      "class"),
-    ("partition_stride_off_by_one", "for (int l = k; l <= L; l += delta)", "for (int l = k; l <= L; l += delta + 1)",
+    ("partition_stride_off_by_one", "(level[v] - k) % delta == 0;", "(level[v] - k) % (delta + 1) == 0;", "partition"),
+    ("partition_stride_from_level_zero", "level[v] >= k && (level[v] - k) % delta == 0;", "level[v] % delta == 0;",
      "partition"),
-    ("partition_forgets_fanout_free_nodes", "if (out_degree[v] == 0) cones[level[v]].insert(v);", ";", "partition"),
+    ("partition_forgets_fanout_free_nodes", "if (on_stride_level || !has_fanout[v]) picked.push_back(v);",
+     "if (on_stride_level) picked.push_back(v);", "partition"),
+    ("partition_groups_count_inclusive", "below += (level[v] < l);", "below += (level[v] <= l);", "partition"),
     ("score_without_scale", "s[j] = scale * dot;", "s[j] = dot;", "attention or closed or dense"),
     ("score_sign", "s[j] = scale * dot;", "s[j] = -scale * dot;", "attention or closed or dense"),
     ("softmax_not_normalised", "for (int j = 0; j < cnt; ++j) a[j] /= z;\n    for (int c = 0; c < d_head; ++c) {",

@@ -492,20 +492,30 @@ def test_partition_roots_match_hand_worked_fixture():
         assert got == want, (k, delta)
 
 
-def test_partition_roots_by_vectorised_selection():
+def test_partition_roots_by_walking_the_levels():
+    """Algorithm 1 carried out as a process on a small random circuit: visit the levels k, k + delta, ... up to the
+    deepest one and collect that level's nodes; then drop every node without fan-out into the group of its own
+    level; groups are sets.  (The checker states the outcome as a per-node predicate plus one sort instead.)"""
     rng = np.random.default_rng(77)
     fanins = random_dag(rng, 10, 600, window=15)
     rp, ci = csr_from_fanins(fanins)
     level = levels_of(fanins)
     n = len(fanins)
-    out_degree = np.bincount(ci, minlength=n)
-    for k, delta in ((8, 6), (3, 2), (2, 1), (50, 1)):
-        on_stride = (level >= k) & ((level - k) % delta == 0)
-        sel = np.nonzero(on_stride | (out_degree == 0))[0]
-        want = sel[np.lexsort((sel, level[sel]))]
+    deepest = int(level.max())
+    fed = set(int(u) for u in ci)
+    for k, delta in ((8, 6), (3, 2), (2, 1), (50, 1), (1, 1), (deepest, 7), (deepest + 1, 1)):
+        groups = {}
+        l = k
+        while l <= deepest:
+            groups[l] = {v for v in range(n) if level[v] == l}
+            l += delta
+        for v in range(n):
+            if v not in fed:
+                groups.setdefault(int(level[v]), set()).add(v)
         roots, gptr = orc.partition_roots(rp, ci, level, k, delta)
-        assert (roots == want).all()
-        assert (gptr == np.concatenate([[0], np.cumsum(np.bincount(level[want], minlength=level.max() + 1))])).all()
+        assert len(gptr) == deepest + 2 and gptr[0] == 0 and gptr[-1] == len(roots)
+        for lv in range(deepest + 1):
+            assert roots[gptr[lv]:gptr[lv + 1]].tolist() == sorted(groups.get(lv, ())), (k, delta, lv)
 
 
 # ----------------------------------------------------------------------------- rest of the block: LayerNorm, FFN
