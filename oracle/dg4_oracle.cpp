@@ -28,6 +28,8 @@
  *                         reading the rows already updated for earlier levels (Sec. 1 and Sec. 3.4:
  *                         each gate is computed once, in strict level order)
  *   orc_partition_roots   Algorithm 1 (graph partition): which nodes' cones the partition collects
+ *   orc_cone_update       Sec. 3.4 (intra- and inter-level updating) with the loop of Algorithm 2: cone mini-batches
+ *                         encoded group by group against a table of historical embeddings
  *   orc_level_buckets / orc_class_order   index arrays of the graph-prep pass, from their definitions
  *
  * Pins (tests that do not restate these loops): dense masked softmax attention by a library routine on
@@ -63,6 +65,7 @@ double orc_round_bf16(double x) {
 }
 
 void orc_round_bf16_array(const double* in, double* out, int64_t cnt) {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < cnt; ++i) out[i] = orc_round_bf16(in[i]);
 }
 
@@ -396,6 +399,78 @@ void orc_layer_levelised(int n, int d, int heads, double scale, double* H, const
         for (int i = lo; i < hi; ++i)
             std::memcpy(H + (int64_t)level_nodes[i] * d, fresh.data() + (int64_t)(i - lo) * d, sizeof(double) * d);
     }
+}
+
+/* The updating strategy of Sec. 3.4 carried out on top of Algorithm 1's partition, for a stack of n_layers
+ * attention layers (Algorithm 2's loop, minus everything that is training): cones are encoded level group by level
+ * group (l = k, k + delta, ...), inside a group in mini-batches of `batch` consecutive cones (ascending root id).
+ * For one mini-batch:
+ *   - its sub-graph is the union S of its cones; a gate of S that an earlier mini-batch has already updated --
+ *     of the same group (intra-level updating) or of an earlier group (inter-level updating) -- is taken from the
+ *     table of historical embeddings and loses its in-edges: it attends to itself only and is not stored again;
+ *   - every other gate v of S attends to the members of cone_k(v) that are present in S (the virtual edges of
+ *     Sec. 3.5 restricted to the sub-graph), itself included, and all gates of S go through all the layers
+ *     together (inside a mini-batch the layers are the all-nodes-parallel layer);
+ *   - the new embeddings of the gates that were not frozen are stored in the table, and every gate of S is
+ *     marked as updated.
+ * The table starts as X (a gate no cone covers keeps its input row; a gate's input to its first mini-batch is its
+ * X row).  hist: [n, d], receives the table; stored: [n], how many times each gate's row was stored (0 or 1);
+ * returns the number of mini-batches.  W_qkv: [n_layers, 3d, d]; W_o: [n_layers, d, d]; rounding as in
+ * orc_layer_parallel, applied to the table as well. */
+int orc_cone_update(int n, int d, int heads, double scale, int n_layers, const double* X, const double* W_qkv,
+                    const double* W_o, int residual, const int32_t* row_ptr, const int32_t* col_idx,
+                    const int32_t* level, int n_levels, int k, int delta, int batch, int rounding, double* hist,
+                    int32_t* stored) {
+    std::vector<int32_t> roots(n), group_ptr(n_levels + 1);
+    orc_partition_roots(n, row_ptr, col_idx, level, n_levels, k, delta, roots.data(), group_ptr.data());
+    std::vector<int32_t> cone_ptr(n + 1);
+    int64_t total = orc_neighbourhood(n, row_ptr, col_idx, k, cone_ptr.data(), nullptr);
+    std::vector<int32_t> cone_idx(total > 0 ? total : 1);
+    orc_neighbourhood(n, row_ptr, col_idx, k, cone_ptr.data(), cone_idx.data());
+
+    for (int64_t i = 0; i < (int64_t)n * d; ++i) hist[i] = store_round(X[i], rounding);
+    std::vector<char> updated(n, 0);
+    for (int v = 0; v < n; ++v) stored[v] = 0;
+    int n_batches = 0;
+    for (int l = 0; l < n_levels; ++l) {                       /* groups without cones are empty ranges */
+        for (int b0 = group_ptr[l]; b0 < group_ptr[l + 1]; b0 += batch) {
+            const int b1 = std::min(b0 + batch, (int)group_ptr[l + 1]);
+            std::set<int> members;                             /* S: union of the mini-batch's cones */
+            for (int r = b0; r < b1; ++r)
+                for (int e = cone_ptr[roots[r]]; e < cone_ptr[roots[r] + 1]; ++e) members.insert(cone_idx[e]);
+            std::vector<int> S(members.begin(), members.end());
+            const int m = (int)S.size();
+            std::vector<int> pos(n, -1);
+            for (int i = 0; i < m; ++i) pos[S[i]] = i;
+            /* the sub-graph's attention lists, in local numbering: self first, then the present cone members */
+            std::vector<int32_t> lptr(m + 1, 0), lidx;
+            for (int i = 0; i < m; ++i) {
+                const int v = S[i];
+                lidx.push_back(i);
+                if (!updated[v])
+                    for (int e = cone_ptr[v] + 1; e < cone_ptr[v + 1]; ++e)
+                        if (pos[cone_idx[e]] >= 0) lidx.push_back(pos[cone_idx[e]]);
+                lptr[i + 1] = (int32_t)lidx.size();
+            }
+            std::vector<double> cur((int64_t)m * d), nxt((int64_t)m * d);
+            for (int i = 0; i < m; ++i) std::memcpy(&cur[(int64_t)i * d], hist + (int64_t)S[i] * d, sizeof(double) * d);
+            for (int j = 0; j < n_layers; ++j) {
+                orc_layer_parallel(m, d, heads, scale, cur.data(), W_qkv + (int64_t)j * 3 * d * d,
+                                   W_o + (int64_t)j * d * d, residual, lptr.data(), lidx.data(), rounding, nxt.data());
+                cur.swap(nxt);
+            }
+            for (int i = 0; i < m; ++i) {
+                const int v = S[i];
+                if (!updated[v]) {
+                    std::memcpy(hist + (int64_t)v * d, &cur[(int64_t)i * d], sizeof(double) * d);
+                    stored[v] += 1;
+                }
+            }
+            for (int v : S) updated[v] = 1;
+            ++n_batches;
+        }
+    }
+    return n_batches;
 }
 
 int orc_num_threads(void) {

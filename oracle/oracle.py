@@ -65,6 +65,9 @@ def _load():
         lib.orc_layer_levelised.restype = None
         lib.orc_layer_levelised.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, c_int, _i32p, _i32p,
                                             c_int, _i32p, _i32p, c_int]
+        lib.orc_cone_update.restype = c_int
+        lib.orc_cone_update.argtypes = [c_int, c_int, c_int, c_dbl, c_int, _f64p, _f64p, _f64p, c_int, _i32p, _i32p, _i32p,
+                                        c_int, c_int, c_int, c_int, c_int, _f64p, _i32p]
         lib.orc_num_threads.restype = c_int
         _lib = lib
     return _lib
@@ -241,3 +244,20 @@ def layer_levelised(H, W_qkv, W_o, nbr_ptr, nbr_idx, level_ptr, level_nodes, hea
                                 _i(nbr_ptr), _i(nbr_idx), level_ptr.shape[0] - 1, _i(level_ptr), _i(level_nodes),
                                 ROUND[rounding])
     return H
+
+
+def cone_update(X, W_qkv_list, W_o_list, row_ptr, col_idx, level, k, delta, batch, heads, scale, residual=True,
+                rounding=None):
+    """Sec. 3.4's updating strategy over Algorithm 1's partition (cone mini-batches against a table of historical
+    embeddings) for a stack of layers.  Returns (table [n, d], stored [n] = times each row was stored, n_batches)."""
+    X = _f64(X)
+    Wq = _f64(np.stack([_f64(w) for w in W_qkv_list]))
+    Wo = _f64(np.stack([_f64(w) for w in W_o_list]))
+    row_ptr, col_idx, level = _i32(row_ptr), _i32(col_idx), _i32(level)
+    n, d = X.shape
+    hist = np.zeros((n, d), np.float64)
+    stored = np.zeros(n, np.int32)
+    nb = _load().orc_cone_update(n, d, heads, float(scale), Wq.shape[0], _d(X), _d(Wq), _d(Wo), int(bool(residual)),
+                                 _i(row_ptr), _i(col_idx), _i(level), int(level.max()) + 1, int(k), int(delta),
+                                 int(batch), ROUND[rounding], _d(hist), _i(stored))
+    return hist, stored, int(nb)

@@ -129,7 +129,7 @@ def test_attention_fp32_heads_and_hops(hops, heads):
     fanins = random_dag(np.random.default_rng(heads), 9, 1500, window=30)
     rp, ci = csr_from_fanins(fanins)
     got, want = _attention_case(rp, ci, levels_of(fanins), hops, heads, "f32", 1.0 / np.sqrt(128 // heads), 1.0)
-    assert np.abs(got - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+    assert np.abs(got - want).max() <= F32_ABS_TOL
 
 
 @pytest.mark.parametrize("hops", [1, 2])
@@ -148,7 +148,10 @@ def test_attention_peaked_softmax(dtype):
     rp, ci = csr_from_fanins(fanins)
     got, want = _attention_case(rp, ci, levels_of(fanins), 2, 8, dtype, 1.0, 2.0)
     if dtype == "f32":
-        assert np.abs(got - want).max() <= 5e-5      # values up to ~8; same relative accuracy
+        # Scores here reach |s| ~ 70 and outputs ~ 9: fp32 holds such a score (in the log2 units the exponential is
+        # taken in) only to 2^-17, i.e. a weight to about 1e-5 of itself, so the 1e-5 bound is taken relative to the
+        # largest output magnitude in this one test (every other fp32 test meets 1e-5 absolute).
+        assert np.abs(got - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
     else:
         assert rel_row_err(got, want).max() <= BF16_ROW_TOL
 
@@ -410,7 +413,7 @@ def test_additive_score_attention_matches_checker(dtype, hops, heads):
         dg4.dg4_sparse_attn_additive_fwd(g, dg4.desc(heads, dg4.DG4_F32, 1.0), dsd, dss, 0.2, dv, o)
         torch.cuda.synchronize()
         want = orc.attention_additive(sd, ss, v32, ptr, idx, 0.2)
-        assert np.abs(o.cpu().numpy().astype(np.float64) - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+        assert np.abs(o.cpu().numpy().astype(np.float64) - want).max() <= F32_ABS_TOL
     else:
         vb = synth.f32_to_bf16_bits(v32)
         dv = dev_bf16(vb)
@@ -457,7 +460,7 @@ def test_wide_cone_attention_matches_checker(dtype, hops, heads):
     scale = 1.0 / np.sqrt(128 // heads)
     got, want = _attention_case(rp, ci, levels_of(fanins), hops, heads, dtype, scale, 1.5)
     if dtype == "f32":
-        assert np.abs(got - want).max() <= F32_ABS_TOL * max(1.0, np.abs(want).max())
+        assert np.abs(got - want).max() <= F32_ABS_TOL
     else:
         assert rel_row_err(got, want).max() <= BF16_ROW_TOL
 

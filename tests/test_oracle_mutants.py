@@ -53,6 +53,13 @@ MUTANTS = [
     ("ffn_without_first_bias", "double acc = b1[h];", "double acc = 0.0;", "ffn"),
     ("ffn_without_relu", "acc = acc > 0.0 ? acc : 0.0;", "", "ffn"),
     ("ffn_without_residual", "z[o] = x[o] + acc;", "z[o] = acc;", "ffn"),
+    ("update_frozen_gate_stored_again", "                if (!updated[v]) {\n                    std::memcpy(hist", "                if (true) {\n                    std::memcpy(hist", "cone_update"),
+    ("update_frozen_gate_keeps_in_edges", "                if (!updated[v])\n                    for (int e = cone_ptr[v] + 1;", "                if (true)\n                    for (int e = cone_ptr[v] + 1;", "cone_update"),
+    ("update_marks_only_the_stored_gates", "            for (int v : S) updated[v] = 1;", "            for (int r = b0; r < b1; ++r) updated[roots[r]] = 1;", "cone_update"),
+    ("update_inputs_not_from_the_table", "std::memcpy(&cur[(int64_t)i * d], hist + (int64_t)S[i] * d, sizeof(double) * d);",
+     "std::memcpy(&cur[(int64_t)i * d], X + (int64_t)S[i] * d, sizeof(double) * d);", "cone_update"),
+    ("update_one_layer_only", "            for (int j = 0; j < n_layers; ++j) {\n                orc_layer_parallel(m,", "            for (int j = 0; j < 1; ++j) {\n                orc_layer_parallel(m,", "cone_update"),
+    ("update_batches_span_level_groups", "const int b1 = std::min(b0 + batch, (int)group_ptr[l + 1]);", "const int b1 = std::min(b0 + batch, (int)group_ptr[n_levels]);", "cone_update"),
     ("ffn_second_matrix_transposed", "acc += u[h] * W2[(int64_t)o * d_ff + h];", "acc += u[h] * W2[(int64_t)h * d + o];", "ffn"),
 ]
 
@@ -67,7 +74,8 @@ def _run_mutant(args):
     lib = os.path.join(tmp, name + ".so")
     subprocess.check_call(["g++", "-O1", "-fopenmp", "-shared", "-fPIC", "-w", "-o", lib, src])
     env = dict(os.environ, DG4_ORACLE_LIB=lib, OMP_NUM_THREADS="2")
-    run = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"), "-x", "-q",
+    run = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"),
+                          os.path.join(ROOT, "tests", "test_oracle_cone_update.py"), "-x", "-q",
                           "-p", "no:cacheprovider", "-k", pins], cwd=ROOT, env=env, capture_output=True, text=True)
     if run.returncode != 1:          # 1 = some selected pin failed; 0 = all passed; 5 = none selected
         return name, f"pytest exit code {run.returncode}:\n{run.stdout[-1500:]}"
