@@ -170,6 +170,40 @@ dg4_status dg4_graph_export(const dg4_graph* g, dg4_array_id which, int32_t* hos
 dg4_status dg4_graph_partition(const dg4_graph* g, int32_t delta, int32_t* roots, int32_t* group_ptr,
                                int64_t* n_roots);
 
+/*
+ * The updating strategy of Sec. 3.4 (intra- and inter-level updating) over the partition of Algorithm 1, for a
+ * stack of attention layers, with the table of historical embeddings on the device.  Cone depth k = the hops the
+ * handle was created with; stride delta; mini-batches of `batch` consecutive cones (ascending root id) inside a
+ * level group.  For each mini-batch, in the order of Algorithm 2's loop (groups l = k, k + delta, ... and the
+ * groups that only hold cones of fan-out-free gates, ascending):
+ *   - the sub-graph is the union S of the mini-batch's cones;
+ *   - a gate of S that an earlier mini-batch has updated (same group: intra-level; earlier group: inter-level)
+ *     enters with its row of the table, attends to itself only (its in-edges are removed) and is not stored again;
+ *   - every other gate v of S enters with its row of the table (its input row: it was never stored), and attends
+ *     to itself and to the members of cone_k(v) present in S;
+ *   - all gates of S go through the n_layers layers together (QKV projection, attention over those lists, output
+ *     projection (+ residual if desc->flags has DG4_FLAG_RESIDUAL)); then the rows of the gates that were not
+ *     frozen are stored in the table and every gate of S is marked as updated.
+ * A gate no cone covers keeps its input row.
+ *   H           device, [n, d] bf16: on entry the input rows, on return the table of historical embeddings
+ *   W_qkv, W_o  host arrays of n_layers device pointers ([3d, d] and [d, d] bf16 each); n_layers 1 .. 64
+ *   delta       >= 1 (the paper uses delta < k so that consecutive groups overlap; not enforced)
+ *   batch       1 .. 65536 cones per mini-batch (the paper uses 128)
+ *   workspace   device, dg4_cone_update_workspace_bytes() bytes, 256-byte aligned: three int32 per gate plus
+ *               buffers sized by the mini-batch (at most batch * (2^(k+1)-1) gates), not by the circuit
+ *   stored      device, [n] int32 or NULL: receives how many times each gate's row was stored (0 or 1)
+ *   n_batches   host or NULL: receives the number of mini-batches
+ * Unlike the other forward calls this one is a host-driven loop: it runs Algorithm 1 (dg4_graph_partition, which
+ * allocates its scratch and synchronises the device) and then reads the size of each mini-batch's sub-graph back
+ * from the device, so it waits on `stream` between mini-batches and must not be captured.  On return all work has
+ * been enqueued on `stream`.  Errors: INVALID_ARG, UNSUPPORTED (dtype other than bf16, heads > 16), ALLOC, CUDA.
+ */
+size_t dg4_cone_update_workspace_bytes(const dg4_graph* g, const dg4_desc* desc, int32_t batch);
+dg4_status dg4_cone_update_fwd(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh, int32_t n_layers,
+                               const void* const* W_qkv, const void* const* W_o, int32_t delta, int32_t batch,
+                               void* workspace, size_t workspace_bytes, int32_t* stored, int64_t* n_batches,
+                               void* stream);
+
 /* Waits for the device to go idle and reads the handle's status word: DG4_OK, or DG4_ERR_TIMEOUT if a bounded
  * device-side wait of an earlier forward call ran out (that call's output is then incomplete). */
 dg4_status dg4_graph_poll_status(const dg4_graph* g, int32_t* out);

@@ -42,6 +42,7 @@ EXPORTS = [
     "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
     "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel", "dg4_graph_destroy_async", "dg4_memory_trim",
     "dg4_debug_set_poll_limit", "dg4_debug_override_current_device",
+    "dg4_cone_update_workspace_bytes", "dg4_cone_update_fwd",
 ]
 
 
@@ -143,6 +144,11 @@ def load():
     lib.dg4_block_fwd_parallel.restype = ctypes.c_int
     lib.dg4_block_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
                                            vp, i64, vp, ctypes.c_size_t, vp]
+    lib.dg4_cone_update_workspace_bytes.restype = ctypes.c_size_t
+    lib.dg4_cone_update_workspace_bytes.argtypes = [vp, dp, ctypes.c_int32]
+    lib.dg4_cone_update_fwd.restype = ctypes.c_int
+    lib.dg4_cone_update_fwd.argtypes = [vp, dp, vp, i64, ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                        ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_size_t, vp, ctypes.POINTER(i64), vp]
     lib.dg4_debug_set_poll_limit.restype = None
     lib.dg4_debug_set_poll_limit.argtypes = [ctypes.c_uint32]
     lib.dg4_debug_override_current_device.restype = None
@@ -327,6 +333,26 @@ def dg4_layers_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, w
 
 def dg4_selftest_bounded_wait(device_status, stream=None):
     _check(load().dg4_selftest_bounded_wait(_ptr(device_status), _stream(stream)))
+
+
+def dg4_cone_update_workspace_bytes(g: Graph, dsc: dg4_desc, batch: int) -> int:
+    return int(load().dg4_cone_update_workspace_bytes(g.handle, ctypes.byref(dsc), int(batch)))
+
+
+def dg4_cone_update_fwd(g: Graph, dsc: dg4_desc, H, W_qkv_list, W_o_list, delta: int, batch: int, workspace,
+                        stored=None, stream=None) -> int:
+    """Sec. 3.4's updating strategy over Algorithm 1's partition (cone mini-batches against the table H, updated in
+    place).  Returns the number of mini-batches."""
+    n = len(W_qkv_list)
+    assert n == len(W_o_list)
+    arr = ctypes.c_void_p * n
+    wq = arr(*[t.data_ptr() for t in W_qkv_list])
+    wo = arr(*[t.data_ptr() for t in W_o_list])
+    nb = ctypes.c_int64(0)
+    _check(load().dg4_cone_update_fwd(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), n, wq, wo, int(delta), int(batch),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(stored),
+                                      ctypes.byref(nb), _stream(stream)))
+    return int(nb.value)
 
 
 def dg4_debug_set_poll_limit(polls: int):
