@@ -21,6 +21,18 @@
 #ifndef DG4_ATTN_MIN_BLOCKS
 #define DG4_ATTN_MIN_BLOCKS 3
 #endif
+// L2 eviction priority of the gathered K | V rows: 1 = ask L2 to keep them (they are gathered again by later nodes)
+#ifndef DG4_ATTN_KV_EVICT_LAST
+#define DG4_ATTN_KV_EVICT_LAST 0
+#endif
+// neighbour-table entries are read once: 1 = ask L2 to drop them first
+#ifndef DG4_ATTN_PAD_EVICT_FIRST
+#define DG4_ATTN_PAD_EVICT_FIRST 0
+#endif
+// 1 = the value rows of table slots beyond |N(v)| are not loaded (the key rows still are, unpredicated)
+#ifndef DG4_ATTN_V_PREDICATED
+#define DG4_ATTN_V_PREDICATED 0
+#endif
 
 namespace {
 
@@ -45,10 +57,22 @@ __global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_
     int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) / G);
     const size_t col = (size_t)sub * EPP * ES;     // byte offset of this lane's piece inside a row
 
+#if DG4_ATTN_KV_EVICT_LAST
+    const uint64_t keep = l2_policy_evict_last();
+#define DG4_LD_KV(ptr) ld_piece_nc_hint(ptr, keep)
+#else
+#define DG4_LD_KV(ptr) ld_piece_nc(ptr)
+#endif
+#if DG4_ATTN_PAD_EVICT_FIRST
+    const uint64_t drop = l2_policy_evict_first();
+#define DG4_LD_PAD(ptr) ld_int_nc_hint(ptr, drop)
+#else
+#define DG4_LD_PAD(ptr) (*(ptr))
+#endif
     int v_next = -1, pad_next = 0;
     if (slot < a.count) {
         v_next = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
-        if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+        if (sub < W) pad_next = DG4_LD_PAD(a.nbr_pad + (size_t)v_next * W + sub);
     }
     for (; slot < a.count; slot += stride) {
         const int v = v_next;
@@ -57,7 +81,7 @@ __global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_
             const int s2 = slot + stride;
             if (s2 < a.count) {
                 v_next = a.node_list ? a.node_list[a.first + s2] : a.first + s2;
-                if (sub < W) pad_next = a.nbr_pad[(size_t)v_next * W + sub];
+                if (sub < W) pad_next = DG4_LD_PAD(a.nbr_pad + (size_t)v_next * W + sub);
             }
         }
         const int cnt = __shfl_sync(mask, pad, grp_base);
@@ -71,13 +95,20 @@ __global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_
         // branches and lets the kernel fit three blocks per SM; the arithmetic below still stops at cnt.
         qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
 #pragma unroll
-        for (int j = 0; j < MAXN; ++j) kq[j] = ld_piece_nc((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
+        for (int j = 0; j < MAXN; ++j) kq[j] = DG4_LD_KV((const char*)a.K + (size_t)u[j] * a.ldk * ES + col);
 #pragma unroll
-        for (int j = 0; j < MAXN; ++j) vq[j] = ld_piece_nc((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
+        for (int j = 0; j < MAXN; ++j) {
+#if DG4_ATTN_V_PREDICATED
+            if (j < cnt)
+#endif
+            vq[j] = DG4_LD_KV((const char*)a.V + (size_t)u[j] * a.ldv * ES + col);
+        }
         float acc[EPP];
         attend<BF16, LPH, MAXN>(qp, kq, vq, cnt, a.scale, mask, acc);
         st_piece_stream((char*)a.O + (size_t)v * a.ldo * ES + col, Elem<BF16>::pack(acc));
     }
+#undef DG4_LD_KV
+#undef DG4_LD_PAD
 }
 
 // Additive (GAT-style) scores: e = LeakyReLU(S_src[u, head] + S_dst[v, head]) from node-level scalars, so a

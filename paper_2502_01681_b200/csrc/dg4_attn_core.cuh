@@ -15,6 +15,29 @@ __device__ __forceinline__ Piece ld_piece_nc(const void* p) {        // read-onl
                  : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
     return r;
 }
+// L2 eviction priorities (a 64-bit policy word made once per thread): rows that are gathered again by later nodes
+// are asked to stay, data that passes through once is asked to leave first.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ Piece ld_piece_nc_hint(const void* p, uint64_t pol) {   // read-only, with an L2 policy
+    Piece r;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p), "l"(pol));
+    return r;
+}
+__device__ __forceinline__ int ld_int_nc_hint(const int* p, uint64_t pol) {
+    int r;
+    asm volatile("ld.global.nc.L2::cache_hint.s32 %0, [%1], %2;" : "=r"(r) : "l"(p), "l"(pol));
+    return r;
+}
 __device__ __forceinline__ Piece ld_piece_cg(const void* p) {        // coherent at L2: data written by other CTAs
     Piece r;
     asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"

@@ -132,12 +132,12 @@ struct dg4i_proj_args {
 };
 dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st);
 
-// Persistent levelised kernel over n_layers layers run as a wavefront.  Q[0], KV[0] hold the projections of the
-// input rows for all nodes (layer 0's weights); Q[k], KV[k] for k >= 1 are filled by the kernel.  H is updated in
-// place.  `sync` is zeroed by the call and must hold dg4i_levelised_sync_bytes() bytes.
+// Persistent levelised kernel over n_layers layers run as a wavefront.  KV[k] ([n, 256] bf16, contents irrelevant on
+// entry) receives layer k's K | V rows of the nodes as they are updated.  H is updated in place.  `sync` is zeroed
+// by the call and must hold dg4i_levelised_sync_bytes() bytes.
 #define DG4I_MAX_LAYERS 8
 size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers);
-dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers, __nv_bfloat16* const* Q,
+dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers,
                                  __nv_bfloat16* const* KV, __nv_bfloat16* H, int64_t ldh,
                                  const __nv_bfloat16* const* W_qkv, const __nv_bfloat16* const* W_o, int32_t* sync,
                                  int32_t* status, cudaStream_t st);

@@ -78,8 +78,8 @@ struct Workspace {
 size_t tensors_bytes(int64_t n) { return ((size_t)n * 128 * 2 * 4 + 255) & ~(size_t)255; }
 size_t sync_bytes(const dg4_graph* g, int n_layers) { return (dg4i_levelised_sync_bytes(g, n_layers) + 255) & ~(size_t)255; }
 size_t workspace_bytes(const dg4_graph* g) { return tensors_bytes(g->n) + sync_bytes(g, 1); }
-// several levelised layers in one call: per layer a Q table [n,128] and a K|V table [n,256], then the counters
-size_t layer_tables_bytes(int64_t n) { return ((size_t)n * 768 + 255) & ~(size_t)255; }
+// several levelised layers in one call: per layer a K|V table [n,256], then the counters
+size_t layer_tables_bytes(int64_t n) { return ((size_t)n * 512 + 255) & ~(size_t)255; }
 size_t layers_workspace_bytes(const dg4_graph* g, int n_layers) {
     size_t multi = layer_tables_bytes(g->n) * (size_t)n_layers + sync_bytes(g, n_layers);
     size_t single = workspace_bytes(g);          // the per-level-launch driver reuses one layer's workspace
@@ -268,24 +268,24 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
     int32_t* status_word = device_status ? device_status : g->dev_status;
 
+    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layer needs DG4_FLAG_LEVEL_LAUNCHES");
+    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
+        // one persistent kernel walks the levels; it projects each tile's own Q | K | V on the fly and fills the
+        // K | V table as nodes are updated
+        int32_t* sync = (int32_t*)((char*)workspace + tensors_bytes(g->n));
+        __nv_bfloat16* kv1[1] = {w.KV};
+        const __nv_bfloat16* wq1[1] = {(const __nv_bfloat16*)W_qkv};
+        const __nv_bfloat16* wo1[1] = {(const __nv_bfloat16*)W_o};
+        return dg4i_levelised_launch(g, desc, 1, kv1, (__nv_bfloat16*)H, ldh, wq1, wo1, sync, status_word, st);
+    }
+
     // Q | K | V of every node from the layer's input
     dg4i_proj_args p;
     p.A = (const __nv_bfloat16*)H; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
     p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;
     p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
     CHECK(dg4i_proj_launch(p, st));
-
-    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
-        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layer needs DG4_FLAG_LEVEL_LAUNCHES");
-    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
-        // one persistent kernel walks the levels
-        int32_t* sync = (int32_t*)((char*)workspace + tensors_bytes(g->n));
-        __nv_bfloat16* q1[1] = {w.Q};
-        __nv_bfloat16* kv1[1] = {w.KV};
-        const __nv_bfloat16* wq1[1] = {(const __nv_bfloat16*)W_qkv};
-        const __nv_bfloat16* wo1[1] = {(const __nv_bfloat16*)W_o};
-        return dg4i_levelised_launch(g, desc, 1, q1, kv1, (__nv_bfloat16*)H, ldh, wq1, wo1, sync, status_word, st);
-    }
 
     // alternative driver: one group of launches per level (attention, output projection, K|V refresh)
     const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;
@@ -352,25 +352,16 @@ extern "C" dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_des
 
     if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
     int32_t* status_word = device_status ? device_status : g->dev_status;
-    __nv_bfloat16* q[DG4I_MAX_LAYERS];
     __nv_bfloat16* kv[DG4I_MAX_LAYERS];
     const __nv_bfloat16* wq[DG4I_MAX_LAYERS];
     const __nv_bfloat16* wo[DG4I_MAX_LAYERS];
     const size_t per_layer = layer_tables_bytes(g->n);
     for (int k = 0; k < n_layers; ++k) {
-        char* basep = (char*)workspace + per_layer * (size_t)k;
-        q[k] = (__nv_bfloat16*)basep;
-        kv[k] = (__nv_bfloat16*)(basep + (size_t)g->n * 256);
+        kv[k] = (__nv_bfloat16*)((char*)workspace + per_layer * (size_t)k);
         wq[k] = (const __nv_bfloat16*)W_qkv[k];
         wo[k] = (const __nv_bfloat16*)W_o[k];
     }
     int32_t* sync = (int32_t*)((char*)workspace + per_layer * (size_t)n_layers);
-
-    // the first layer's Q | K | V of every node from the input rows; later layers' tables are filled on the fly
-    dg4i_proj_args p;
-    p.A = (const __nv_bfloat16*)H; p.lda = ldh; p.W = wq[0]; p.n_out = 384;
-    p.out[0] = q[0]; p.ldo[0] = 128; p.out[1] = kv[0]; p.ldo[1] = 256; p.out[2] = kv[0] + 128; p.ldo[2] = 256;
-    p.R = nullptr; p.ldr = 0; p.row_list = nullptr; p.first = 0; p.rows = g->n; p.status = status_word;
-    CHECK(dg4i_proj_launch(p, st));
-    return dg4i_levelised_launch(g, desc, n_layers, q, kv, (__nv_bfloat16*)H, ldh, wq, wo, sync, status_word, st);
+    // every layer projects its tiles' own Q | K | V on the fly and fills its K | V table as nodes are updated
+    return dg4i_levelised_launch(g, desc, n_layers, kv, (__nv_bfloat16*)H, ldh, wq, wo, sync, status_word, st);
 }

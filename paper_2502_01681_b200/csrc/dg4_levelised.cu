@@ -1,34 +1,51 @@
 // Levelised layers as ONE persistent kernel (Sec. 1 / Sec. 3.4: gates are encoded level by level in
 // topological order, each gate once, reading the rows already updated for lower levels).
 //
-// Work of one tile (16 nodes of one level, for one layer k):
-//   1. gather the K | V rows of every neighbour from layer k's K|V table (16 lanes per node, 16 bytes per
+// Work of one tile (16 nodes of one level, for one layer k), in two parts:
+//   PROLOGUE (depends only on the layer below): the tile's input rows -- H as layer k-1 left it, or the caller's
+//      rows for the first layer -- are brought into shared memory in the tensor core's K-major, 128-byte-swizzled
+//      operand layout, and Q | K | V of the tile's own nodes are computed from them TRANSPOSED on the tensor
+//      cores: D[feature, node] = W * X^T (tcgen05.mma, M = 128 features, N = 16 nodes, K = 128).  A node's own
+//      query, key and value always come from its row as the previous layer left it, and nobody else ever reads
+//      them (other nodes gather its K | V only after its update), so they stay on chip: no Q table, no up-front
+//      projection of all nodes.
+//   MAIN (depends on the level below in the same layer):
+//   1. gather the K | V rows of every OTHER neighbour from layer k's K|V table (16 lanes per node, 16 bytes per
 //      lane), compute scores, softmax and the weighted value sum in registers, and write the 16 x 128
-//      attention tile into shared memory in the tensor core's K-major, 128-byte-swizzled operand layout;
-//   2. output projection TRANSPOSED on the tensor cores: D[feature, node] = W_o * O^T (tcgen05.mma, M = 128
-//      features, N = 16 nodes, K = 128), so a small tile costs a fraction of a 128-row tile and all warps take
-//      part in the epilogue (128 TMEM lanes x 16 columns);
-//   3. add the residual, round to bf16, write the new rows to H and -- in operand layout again -- to shared
-//      memory;
-//   4. from the new rows, again transposed: refresh the tile's K | V rows of layer k (so that higher levels
-//      gather updated rows) and, if there is a layer k+1, project that layer's Q | K | V rows of these nodes
-//      (a node's own query, key and value always come from its row as the previous layer left it).
+//      attention tile into shared memory in operand layout;
+//   2. output projection, transposed again: D[feature, node] = W_o * O^T, so a small tile costs a fraction of a
+//      128-row tile and all warps take part in the epilogue (128 TMEM lanes x 16 columns);
+//   3. add the residual (the input rows still in shared memory), round to bf16, write the new rows to H and --
+//      in operand layout again -- to shared memory;
+//   4. from the new rows, transposed: the tile's K | V rows of layer k, stored to the table so that higher levels
+//      gather updated rows.
+// The prologue of a CTA's NEXT tile is folded into the main part of the current one: the next tile's rows are
+// requested once the layer below is known to have finished them, they are written to the second input buffer
+// before the barrier that precedes step 4, and their Q | K | V product is issued right behind step 4's MMAs, so
+// it runs while the CTA stores its rows, arrives and waits for the level to complete.  The level-to-level chain
+// is then wait -> gather -> W_o -> K|V refresh -> arrive; the projections of the next tile hide in the hand-off.
+// A CTA that has no tile in a level but has one in the next does that prologue while it is idle.
+// The MMAs are issued by a thread of a ninth warp that does nothing else: issuing an M128 x N16 x K16 instruction
+// occupies the issuing thread for about as long as the tensor pipe needs to execute it, so a worker thread that
+// issued the next tile's 24 instructions would hold up its own warp's epilogue (and with it the level) for their
+// whole duration.  The workers hand the issuing thread one order at a time (a word in shared memory and an
+// mbarrier arrival) and wait only for the completion barrier of the product they need next.
 //
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
-// to layers round-robin; each keeps its layer's W_o, W_k, W_v and the next layer's W_q, W_k, W_v resident in
-// TENSOR memory (six blocks of 128 lanes x 64 columns beside the accumulators) and issues its MMAs with the A
-// operand read from there, so the weights are never re-read from shared memory and shared memory holds only the
-// node-side tiles.  With n layers the dependent chain is n_levels + n - 1 tile steps long
-// instead of n * n_levels, while computing exactly what n successive level-by-level sweeps compute.
+// to layers round-robin; each keeps its layer's W_o, W_k, W_v and W_q resident in TENSOR memory (four blocks
+// of 128 lanes x 64 columns beside the accumulators) and issues its MMAs with the A operand read from there, so
+// the weights are never re-read from shared memory and shared memory holds only the node-side tiles.  With n
+// layers the dependent chain is n_levels + n - 1 tile steps long instead of n * n_levels, while computing exactly
+// what n successive level-by-level sweeps compute.
 //
 // Levels are separated by counters in global memory instead of kernel launches: every (layer, level) has an
 // arrival counter that only the CTAs owning a tile of it bump (release); before a level in which it has work a
 // CTA waits (acquire) until the counter of its layer's previous non-empty level and the counter of the previous
 // layer's same level are full.  Completion is transitive, because every CTA that arrived had itself waited the
 // same way.  Launched cooperatively (all CTAs co-resident).  Every wait is bounded; on expiry the kernel records
-// DG4_ERR_TIMEOUT, raises an abort word that every other wait polls, and all CTAs leave their loops, free
-// tensor memory and return.
+// DG4_ERR_TIMEOUT, raises an abort word that every other wait polls, and all CTAs leave their loops, wait for the
+// MMAs they have issued, free tensor memory and return.
 
 #include "dg4_internal.h"
 #include "dg4_attn_core.cuh"
@@ -42,37 +59,47 @@ using namespace sm100;
 using namespace attn;
 
 constexpr int kTile = 16;                    // nodes per tile
-constexpr int kThreads = kTile * 16;         // 16 lanes per node
+constexpr int kWorkers = kTile * 16;         // 16 lanes per node: eight warps that gather, attend and run the epilogues
+constexpr int kThreads = kWorkers + 32;      // and a ninth warp whose first lane issues every tcgen05.mma
 constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
-constexpr int kTmemCols = 512;               // six accumulators of kTile columns, then six weight blocks of 64 columns
-constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks W_o | W_k | W_v | next W_q | W_k | W_v
+constexpr int kTileOp = 2 * kBHalf;          // a kTile x 128 bf16 tile in operand layout (4 KiB)
+constexpr int kTmemCols = 512;
+constexpr int kAccO = 0, kAccK2 = 1, kAccV2 = 2, kAccQ = 3, kAccK = 4, kAccV = 5;   // accumulators of kTile columns
+constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks W_o | W_k | W_v | W_q
 constexpr int kWCols = 64;                   // a 128 x 128 bf16 block: 128 lanes x 64 columns of two elements
-constexpr int kStageRow = 1280;              // staging per node: K|V of this layer 512, Q of the next 256, its K|V 512
+constexpr int kBlkO = 0, kBlkK = 1, kBlkV = 2, kBlkQ = 3;
+constexpr int kStageRow = 768 + 16;          // staging per node: Q 256 | K 256 | V 256 (+ padding against bank conflicts)
 
-constexpr int kOffO = 0;                          // attention tile (operand layout)
-constexpr int kOffHp = kOffO + 2 * kBHalf;        // new rows (operand layout)
-constexpr int kOffHres = kOffHp + 2 * kBHalf;     // residual rows, plain [kTile][256 B]
-constexpr int kOffStage = kOffHres + kTile * 256; // output staging, plain [kTile][kStageRow]
+constexpr int kOffO = 0;                               // attention tile (operand layout)
+constexpr int kOffHp = kOffO + kTileOp;                // new rows (operand layout)
+constexpr int kOffX = kOffHp + kTileOp;                // input rows of the current and of the next tile (operand layout)
+constexpr int kOffHres = kOffX + 2 * kTileOp;          // the same rows, plain [kTile][256 B], twice
+constexpr int kOffStage = kOffHres + 2 * kTile * 256;  // staging, plain [kTile][kStageRow]
 constexpr int kOffMisc = kOffStage + kTile * kStageRow;
 constexpr int kSmemBytes = kOffMisc + 256 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-static_assert(kWCol0 + 6 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
+static_assert(kWCol0 + 4 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
+static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) == 0, "operand tiles are 1024-byte aligned");
 // Every CTA allocates all of its SM's tensor memory, so two CTAs must never share an SM (the second one's
 // allocation would wait for the first, which waits for the second's levels): the launch asks for more than half
 // of an SM's shared memory, which rules that out.
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
+enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdWo = 2, kCmdKv = 3, kCmdKvThenQkv = 4 };
+
 struct Misc {
-    uint64_t mma1, mma2, drain;
+    uint64_t mma0, mma1, mma2, drain;
+    uint64_t cmd_bar;                      // the workers' next order for the issuing thread is in `cmd`
+    int32_t cmd, cmd_buf;
     uint32_t tmem_base;
     int32_t go, go2;
     int32_t failed;                        // a wait for this CTA's own MMAs ran out: leave at the next level
+    int32_t pre_ok;                        // the layer below has finished the rows of this CTA's next tile
     int32_t node[kTile];
 };
 
 struct LevParams {
-    __nv_bfloat16* Q[DG4I_MAX_LAYERS];     // [n, 128] per layer
-    __nv_bfloat16* KV[DG4I_MAX_LAYERS];    // [n, 256] per layer
+    __nv_bfloat16* KV[DG4I_MAX_LAYERS];    // [n, 256] per layer: K | V of the nodes the layer has updated so far
     const __nv_bfloat16* Wo[DG4I_MAX_LAYERS];    // [128, 128] per layer, out x in
     const __nv_bfloat16* Wqkv[DG4I_MAX_LAYERS];  // [384, 128] per layer
     __nv_bfloat16* H;                      // [n, ldh], updated in place by every layer in turn
@@ -123,11 +150,18 @@ __device__ __forceinline__ uint16_t bf16_bits(float x) {
 __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
     return (uint32_t)((k >> 6) * kBHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
 }
+// byte offset of the 16-byte piece `sub` (0..15) of row `row` in the same layout
+__device__ __forceinline__ uint32_t operand_piece(int row, int sub) {
+    return (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(row, sub & 7);
+}
 
 __device__ __forceinline__ void give_up(const LevParams& p) {
     atomicExch(p.abort_word, 1);
     if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
 }
+
+// barrier among the eight worker warps only (the issuing warp never joins it)
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 
 // Polls (acquire) until *counter >= target; false on abort or after `limit` polls (about a second by default).
 __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target, const int32_t* abort_word, uint32_t limit) {
@@ -148,28 +182,31 @@ levelised_kernel(LevParams p) {
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
-    const uint32_t sO = base + kOffO, sHp = base + kOffHp, sHres = base + kOffHres, sSt = base + kOffStage;
+    const uint32_t sO = base + kOffO, sHp = base + kOffHp, sX = base + kOffX, sHres = base + kOffHres, sSt = base + kOffStage;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid >> 4, sub = tid & 15;          // node slot of the tile and lane within the node
     const int grp_base = lane - sub;
     const unsigned gmask = 0xffffu << grp_base;
-    const uint32_t bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
+    const uint32_t bar0 = smem_u32(&misc->mma0), bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
 
     // this CTA's layer, its rank among the CTAs of that layer, and how many CTAs each layer has
     const int layer = (int)blockIdx.x % p.n_layers;
     const int bid = (int)blockIdx.x / p.n_layers;
     auto ctas_of = [&](int k) { return ((int)gridDim.x - k + p.n_layers - 1) / p.n_layers; };
     const int nctas = ctas_of(layer);
-    const bool has_next = layer + 1 < p.n_layers;
-    const int n_acc = has_next ? 5 : 2;                  // accumulators of the second MMA group
 
     if (tid == 0) {
+        mbar_init(bar0, 1);
         mbar_init(bar1, 1);
         mbar_init(bar2, 1);
         mbar_init(smem_u32(&misc->drain), 1);
+        mbar_init(smem_u32(&misc->cmd_bar), 1);
+        misc->cmd = kCmdExit;
+        misc->cmd_buf = 0;
         misc->go = 1;
         misc->go2 = 1;
         misc->failed = 0;
+        misc->pre_ok = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
@@ -177,24 +214,24 @@ levelised_kernel(LevParams p) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc->tmem_base;
-    static_assert(kThreads / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
+    static_assert(kWorkers / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
     const int q4 = warp & 3, cg = warp >> 2;             // TMEM lane quadrant of the warp; which half of the columns it takes
     const int feat = q4 * 32 + lane;                     // output feature (TMEM lane) this thread holds
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
-    {
-        const int n_blocks = has_next ? 6 : 3;
-        for (int blk = 0; blk < n_blocks; ++blk) {
-            const __nv_bfloat16* wb = blk == 0 ? p.Wo[layer]
-                                     : blk < 3 ? p.Wqkv[layer] + (size_t)blk * 128 * 128
-                                               : p.Wqkv[layer + 1] + (size_t)(blk - 3) * 128 * 128;
+    if (warp < 8) {
+        for (int blk = 0; blk < 4; ++blk) {
+            const __nv_bfloat16* wb = blk == kBlkO ? p.Wo[layer]
+                                     : blk == kBlkQ ? p.Wqkv[layer]
+                                                    : p.Wqkv[layer] + (size_t)blk * 128 * 128;     // kBlkK = 1, kBlkV = 2
             const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint4 lo = src[2 * c], hi = src[2 * c + 1];
                 const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-                tmem_st_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kWCol0 + blk * kWCols + cg * 32 + c * 8), r);
+                tmem_st_32x8(tmem + lane_base + (uint32_t)(kWCol0 + blk * kWCols + cg * 32 + c * 8), r);
             }
         }
         tmem_st_wait();
@@ -206,233 +243,345 @@ levelised_kernel(LevParams p) {
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
     // matrix descriptors of the node-side operands; stepping along K only adds to the address field
     const uint64_t dO = smem_desc_sw128(sO), dHp = smem_desc_sw128(sHp);
-    uint32_t ph1 = 0, ph2 = 0;
-    int last_nonempty = -1, last_participants = 0;
-    bool alive = true;
-    const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
-
-    const char* kv_tab = (const char*)p.KV[layer];
-    const char* q_tab = (const char*)p.Q[layer];
-    int32_t* my_arrive = p.arrive + (size_t)layer * p.n_levels;
-    const int32_t* prev_arrive = layer > 0 ? p.arrive + (size_t)(layer - 1) * p.n_levels : nullptr;
-    const int prev_ctas = layer > 0 ? ctas_of(layer - 1) : 0;
-
-    // The index chain of a tile (node id -> neighbour-table entry) is two dependent loads that do not depend on
-    // any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
-    // level-to-level critical path: while level l is processed, the node id of this CTA's first tile of level
-    // l+2 and the table entry for level l+1 are in flight.
-    // The level offsets run four levels ahead in registers: every acquire of a counter drops the L1 contents,
-    // so a plain load at the top of a level would cost a trip to L2 on the level-to-level chain.
-    auto lp_at = [&](int lv) { return p.level_ptr[lv < p.n_levels ? lv : p.n_levels]; };
-    auto stage_node = [&](int lv_first, int lv_end) -> int {   // node of (first tile of this CTA, this slot) of a level
-        const int r = bid * kTile + slot;
-        return (r < lv_end - lv_first) ? p.level_nodes[lv_first + r] : -1;
+    const uint64_t dX[2] = {smem_desc_sw128(sX), smem_desc_sw128(sX + kTileOp)};
+    // issues Q | K | V = W * X^T for the rows in input buffer b (one thread)
+    auto issue_qkv = [&](int b) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
+            mma_bf16_ta(tmem + (uint32_t)(kTile * kAccQ), tmem + (uint32_t)(kWCol0 + kBlkQ * kWCols + ks * 8), dX[b] + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+            mma_bf16_ta(tmem + (uint32_t)(kTile * kAccK), tmem + (uint32_t)(kWCol0 + kBlkK * kWCols + ks * 8), dX[b] + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+            mma_bf16_ta(tmem + (uint32_t)(kTile * kAccV), tmem + (uint32_t)(kWCol0 + kBlkV * kWCols + ks * 8), dX[b] + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+        }
+        mma_commit(bar0);
     };
-    int lp0 = lp_at(0), lp1 = lp_at(1), lp2 = lp_at(2), lp3 = lp_at(3);
-    auto pad_of = [&](int v) -> int { return (v >= 0 && sub < W) ? p.nbr_pad[(size_t)v * W + sub] : 0; };
-    int v0 = stage_node(lp0, lp1);                     // level l  : node id and this lane's table word
-    int pad0 = pad_of(v0);
-    int vC = stage_node(lp1, lp2);                     // level l+1: node id
-
-    for (int l = 0; l < p.n_levels && alive; ++l) {
-        const int first = lp0;
-        const int n_l = lp1 - lp0;
-        // issue the next load of every pipelined chain; the results are first used one level later
-        const int lp4 = lp_at(l + 4);
-        const int vB = stage_node(lp2, lp3);
-        const int padC = pad_of(vC);
-        const int tiles = (n_l + kTile - 1) / kTile;
-        if (n_l > 0 && bid < tiles) {
-            bool waited = false;
-            int v_nx = -1, pad_nx = 0;           // index chain of this CTA's next tile in a wide level
-            for (int tile = bid; tile < tiles; tile += nctas) {
-                int v, pad;
-                if (tile == bid) {
-                    v = v0; pad = pad0;
-                } else {                         // further tiles of a wide level: fetched during the tile before
-                    v = v_nx; pad = pad_nx;
+    if (warp == 8) {
+        // ---------------------------------------------------------------- the issuing thread
+        if (lane == 0) {
+            const uint32_t cmd_bar = smem_u32(&misc->cmd_bar);
+            uint32_t phc = 0;
+            int strikes = 0;
+            for (;;) {
+                if (!mbar_wait(cmd_bar, phc, p.poll_limit)) {
+                    // no order for a long time: normal while the CTA idles through levels in which it has no tile,
+                    // unless the run was aborted meanwhile; a bound on the total keeps even that wait finite
+                    if (ld_acquire(p.abort_word) != 0) break;
+                    if (++strikes >= 64) { give_up(p); break; }
+                    continue;
                 }
-                {
-                    const int r = (tile + nctas) * kTile + slot;
-                    v_nx = (tile + nctas < tiles && r < n_l) ? p.level_nodes[first + r] : -1;
-                }
-                const bool valid = v >= 0;
-
-                if (!waited) {
-                    // ---- this layer's previous level and the previous layer's same level must be complete
-                    // (two pollers in different warps, so that both counters are watched at the same time)
-                    if (tid == 0) {
-                        bool go = true;
-                        if (misc->failed) go = false;
-                        if (go && last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
-                        if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
-                        if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
-                        misc->go = go ? 1 : 0;
-                    } else if (tid == 32) {
-                        bool go = true;
-                        if (prev_arrive) go = wait_counter(prev_arrive + l, tiles < prev_ctas ? tiles : prev_ctas, p.abort_word, counter_limit);
-                        if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
-                        misc->go2 = go ? 1 : 0;
-                    }
-                    __syncthreads();
-                    waited = true;
-                    if (!misc->go || !misc->go2) { alive = false; break; }
-                }
-
-                // ---- gather and attend
-                Piece kq[MAXN], vq[MAXN], qp, hres;
-                int u[MAXN];
-                const int cnt = valid ? __shfl_sync(gmask, pad, grp_base) : 1;
-                u[0] = v;
-#pragma unroll
-                for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(gmask, pad, grp_base + j);
-                float acc[8];
-                if (valid) {
-#pragma unroll
-                    for (int j = 0; j < MAXN; ++j)
-                        if (j < cnt) vq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + 256 + sub * 16);
-                    if (cnt > 1) {
-                        qp = ld_piece_cg(q_tab + (size_t)v * 256 + sub * 16);
-#pragma unroll
-                        for (int j = 0; j < MAXN; ++j)
-                            if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
-                    }
-                    if (p.residual) hres = ld_piece_cg((const char*)p.H + (size_t)v * p.ldh * 2 + sub * 16);
-                } else {
-                    vq[0].w[0] = vq[0].w[1] = vq[0].w[2] = vq[0].w[3] = 0u;
-                }
-                if (!valid || !p.residual) hres.w[0] = hres.w[1] = hres.w[2] = hres.w[3] = 0u;
-                attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, gmask, acc);
-                pad_nx = pad_of(v_nx);           // its node id has arrived by now; the entry is used by the next tile
-                {
-                    Piece o = Elem<true>::pack(acc);
-                    st_shared_v4(sO + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), o.w);
-                    st_shared_v4(sHres + (uint32_t)(slot * 256 + sub * 16), hres.w);
-                    if (sub == 0) misc->node[slot] = v;
-                }
-                fence_proxy_async_smem();
-                __syncthreads();
-
-                // ---- output projection, transposed: D[feature, node] = W_o * O^T
-                if (tid == 0) {
+                phc ^= 1u;
+                strikes = 0;
+                const int cmd = *reinterpret_cast<volatile int32_t*>(&misc->cmd);
+                const int b = *reinterpret_cast<volatile int32_t*>(&misc->cmd_buf);
+                if (cmd == kCmdExit) break;
+                if (cmd == kCmdQkv) {
+                    issue_qkv(b);
+                } else if (cmd == kCmdWo) {
+                    // output projection, transposed: D[feature, node] = W_o * O^T
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                        mma_bf16_ta(tmem, tmem + (uint32_t)(kWCol0 + ks * 8), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccO), tmem + (uint32_t)(kWCol0 + kBlkO * kWCols + ks * 8), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
                     }
                     mma_commit(bar1);
-                }
-                if (!mbar_wait(bar1, ph1, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
-                ph1 ^= 1u;
-                tc_fence_after();
-                {
-                    uint32_t d[8];
-                    tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(cg * 8), d);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int nn = 0; nn < 8; ++nn) {
-                        const int node = cg * 8 + nn;
-                        const uint16_t rb = ld_shared_b16(sHres + (uint32_t)(node * 256 + feat * 2));
-                        const float val = __uint_as_float(d[nn]) + __uint_as_float((uint32_t)rb << 16);
-                        st_shared_b16(sHp + operand_offset(node, feat), bf16_bits(val));
-                    }
-                }
-                tc_fence_before();
-                fence_proxy_async_smem();
-                __syncthreads();
-
-                // ---- from the new rows, transposed: this layer's K | V refresh and the next layer's Q | K | V
-                if (tid == 0) {
+                } else {
+                    // from the new rows, transposed: this layer's K | V refresh; right behind it, if ordered, the next
+                    // tile's Q | K | V (it runs while this tile's rows are stored and the level completes)
                     tc_fence_after();
-                    // K-step outermost: consecutive instructions accumulate into different accumulators, so none
-                    // has to wait for the one before it
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-#pragma unroll
-                        for (int blk = 0; blk < 5; ++blk) {
-                            if (blk < n_acc) {
-                                mma_bf16_ta(tmem + (uint32_t)(kTile * (1 + blk)),
-                                            tmem + (uint32_t)(kWCol0 + (1 + blk) * kWCols + ks * 8), dHp + (b_off >> 4), idesc,
-                                            ks > 0 ? 1u : 0u);
-                            }
-                        }
+                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccK2), tmem + (uint32_t)(kWCol0 + kBlkK * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccV2), tmem + (uint32_t)(kWCol0 + kBlkV * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
                     }
                     mma_commit(bar2);
+                    if (cmd == kCmdKvThenQkv) issue_qkv(b);
                 }
-                // meanwhile: the new rows go to H (16 lanes cover one 256-byte row)
-                const int node_v = misc->node[slot];
-                {
-                    uint32_t w4[4];
-                    ld_shared_v4(sHp + (uint32_t)((sub >> 3) * kBHalf) + sw128_offset(slot, sub & 7), w4);
-                    if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
-                }
-                if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
-                ph2 ^= 1u;
-                tc_fence_after();
-                // accumulator blk (0: K, 1: V, 2: next Q, 3: next K, 4: next V) -> byte offset inside a staging row
-                {
-                    uint32_t d[5][8];
+            }
+            // Tensor memory is freed below: every MMA issued must have completed.  Normally each was waited for by
+            // the workers; after a wait that ran out, one may still be in flight.
+            mma_commit(smem_u32(&misc->drain));
+            mbar_wait(smem_u32(&misc->drain), 0);
+        }
+    } else {
+        // ---------------------------------------------------------------- the eight worker warps
+        // hands the issuing thread its next order (one worker thread, after the barrier that made the operands
+        // of that order visible)
+        auto post = [&](int cmd, int b) {
+            misc->cmd = cmd;
+            misc->cmd_buf = b;
+            mbar_arrive(smem_u32(&misc->cmd_bar));
+        };
+        uint32_t ph0 = 0, ph1 = 0, ph2 = 0;
+        int last_nonempty = -1, last_participants = 0;
+        bool alive = true;
+        const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
+
+        const char* kv_tab = (const char*)p.KV[layer];
+        int32_t* my_arrive = p.arrive + (size_t)layer * p.n_levels;
+        const int32_t* prev_arrive = layer > 0 ? p.arrive + (size_t)(layer - 1) * p.n_levels : nullptr;
+        const int prev_ctas = layer > 0 ? ctas_of(layer - 1) : 0;
+        auto prev_target = [&](int tiles_of_level) { return tiles_of_level < prev_ctas ? tiles_of_level : prev_ctas; };
+
+        // this lane's piece of node v's input row (zero for an empty slot) into input buffer b, both layouts
+        auto stage_input = [&](int b, const Piece& x) {
+            st_shared_v4(sX + (uint32_t)(b * kTileOp) + operand_piece(slot, sub), x.w);
+            st_shared_v4(sHres + (uint32_t)(b * kTile * 256 + slot * 256 + sub * 16), x.w);
+        };
+        auto load_input = [&](int v) {
+            Piece x;
+            if (v >= 0) x = ld_piece_cg((const char*)p.H + (size_t)v * p.ldh * 2 + sub * 16);
+            else x.w[0] = x.w[1] = x.w[2] = x.w[3] = 0u;
+            return x;
+        };
+
+        // The index chain of a tile (node id -> neighbour-table entry) is two dependent loads that do not depend on
+        // any other CTA's results.  It is software-pipelined across levels so that none of it sits on the
+        // level-to-level critical path: while level l is processed, the node id of this CTA's first tile of level
+        // l+2 and the table entry for level l+1 are in flight.
+        // The level offsets run four levels ahead in registers: every acquire of a counter drops the L1 contents,
+        // so a plain load at the top of a level would cost a trip to L2 on the level-to-level chain.
+        auto lp_at = [&](int lv) { return p.level_ptr[lv < p.n_levels ? lv : p.n_levels]; };
+        auto stage_node = [&](int lv_first, int lv_end) -> int {   // node of (first tile of this CTA, this slot) of a level
+            const int r = bid * kTile + slot;
+            return (r < lv_end - lv_first) ? p.level_nodes[lv_first + r] : -1;
+        };
+        int lp0 = lp_at(0), lp1 = lp_at(1), lp2 = lp_at(2), lp3 = lp_at(3);
+        auto pad_of = [&](int v) -> int { return (v >= 0 && sub < W) ? p.nbr_pad[(size_t)v * W + sub] : 0; };
+        int v0 = stage_node(lp0, lp1);                     // level l  : node id and this lane's table word
+        int pad0 = pad_of(v0);
+        int vC = stage_node(lp1, lp2);                     // level l+1: node id
+
+        bool pro_ready = false;      // the Q | K | V product of this CTA's next tile has been issued (rows in buffer `buf`)
+        int buf = 0;
+
+        for (int l = 0; l < p.n_levels && alive; ++l) {
+            const int first = lp0;
+            const int n_l = lp1 - lp0;
+            // issue the next load of every pipelined chain; the results are first used one level later
+            const int lp4 = lp_at(l + 4);
+            const int vB = stage_node(lp2, lp3);
+            const int padC = pad_of(vC);
+            const int tiles = (n_l + kTile - 1) / kTile;
+            const int tiles_next = (lp2 - lp1 + kTile - 1) / kTile;      // tiles of level l + 1
+            if (n_l > 0 && bid < tiles) {
+                bool waited = false;
+                int v_nx = -1, pad_nx = 0;           // index chain of this CTA's next tile in a wide level
+                for (int tile = bid; tile < tiles; tile += nctas) {
+                    int v, pad;
+                    if (tile == bid) {
+                        v = v0; pad = pad0;
+                    } else {                         // further tiles of a wide level: fetched during the tile before
+                        v = v_nx; pad = pad_nx;
+                    }
+                    const bool more_here = tile + nctas < tiles;
+                    {
+                        const int r = (tile + nctas) * kTile + slot;
+                        v_nx = (more_here && r < n_l) ? p.level_nodes[first + r] : -1;
+                    }
+                    const bool valid = v >= 0;
+
+                    // ---- this tile's own Q | K | V: read from tensor memory if the product was issued during the
+                    // tile before, else brought up from scratch below (after the counters)
+                    auto epilogue_qkv = [&]() {
+                        if (!mbar_wait(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                        ph0 ^= 1u;
+                        tc_fence_after();
+                        uint32_t d[3][8];
 #pragma unroll
-                    for (int blk = 0; blk < 5; ++blk)
-                        if (blk < n_acc)
-                            tmem_ld_32x8(tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(kTile * (1 + blk) + cg * 8), d[blk]);
-                    tmem_ld_wait();
+                        for (int blk = 0; blk < 3; ++blk)
+                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccQ + blk) + cg * 8), d[blk]);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int blk = 0; blk < 5; ++blk) {
-                        if (blk < n_acc) {
+                        for (int blk = 0; blk < 3; ++blk) {
+                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
+#pragma unroll
+                            for (int nn = 0; nn < 8; ++nn)
+                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
+                        }
+                        tc_fence_before();
+                    };
+                    if (pro_ready) epilogue_qkv();
+
+                    if (!waited) {
+                        // ---- this layer's previous level must be complete, and (unless the prologue already saw it)
+                        // the previous layer's same level: two pollers in different warps, so that both counters are
+                        // watched at the same time
+                        if (tid == 0) {
+                            bool go = true;
+                            if (misc->failed) go = false;
+                            if (go && last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
+                            if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                            if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
+                            misc->go = go ? 1 : 0;
+                        } else if (tid == 32) {
+                            bool go = true;
+                            if (prev_arrive && !pro_ready) go = wait_counter(prev_arrive + l, prev_target(tiles), p.abort_word, counter_limit);
+                            if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                            misc->go2 = go ? 1 : 0;
+                        }
+                        worker_sync();
+                        waited = true;
+                        if (!misc->go || !misc->go2) { alive = false; break; }
+                    } else if (pro_ready) {
+                        worker_sync();             // the staged Q | K | V are visible to every lane
+                    }
+                    if (!pro_ready) {
+                        // from scratch (a CTA's first tile, or the layer below was not ready in time): rows -> shared
+                        // memory -> product -> staging
+                        stage_input(buf, load_input(v));
+                        fence_proxy_async_smem();
+                        worker_sync();
+                        if (tid == 0) post(kCmdQkv, buf);
+                        epilogue_qkv();
+                        worker_sync();
+                    }
+                    const uint32_t sHres_cur = sHres + (uint32_t)(buf * kTile * 256);
+
+                    // ---- gather and attend
+                    Piece kq[MAXN], vq[MAXN], qp;
+                    int u[MAXN];
+                    const int cnt = valid ? __shfl_sync(gmask, pad, grp_base) : 1;
+                    u[0] = v;
+#pragma unroll
+                    for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(gmask, pad, grp_base + j);
+                    float acc[8];
+                    if (valid) {
+#pragma unroll
+                        for (int j = 1; j < MAXN; ++j)
+                            if (j < cnt) vq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + 256 + sub * 16);
+#pragma unroll
+                        for (int j = 1; j < MAXN; ++j)
+                            if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
+                    }
+                    // which tile comes next for this CTA, and may its rows be requested already?
+                    const bool next_level_tile = !more_here && l + 1 < p.n_levels && bid < tiles_next;
+                    const bool want_pre = more_here || next_level_tile;
+                    const int v_pre = more_here ? v_nx : vC;
+                    if (tid == 32) {
+                        int ok = want_pre ? 1 : 0;
+                        if (next_level_tile && prev_arrive) ok = ld_acquire(prev_arrive + l + 1) >= prev_target(tiles_next) ? 1 : 0;
+                        misc->pre_ok = ok;
+                    }
+                    {   // the node's own query, key and value: from the staging rows
+                        const uint32_t row = sSt + (uint32_t)(slot * kStageRow + sub * 16);
+                        ld_shared_v4(row, qp.w);
+                        ld_shared_v4(row + 256, kq[0].w);
+                        ld_shared_v4(row + 512, vq[0].w);
+                    }
+                    attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, gmask, acc);
+                    pad_nx = pad_of(v_nx);           // its node id has arrived by now; the entry is used by the next tile
+                    {
+                        Piece o = Elem<true>::pack(acc);
+                        st_shared_v4(sO + operand_piece(slot, sub), o.w);
+                        if (sub == 0) misc->node[slot] = v;
+                    }
+                    fence_proxy_async_smem();
+                    worker_sync();
+
+                    // ---- output projection, transposed: D[feature, node] = W_o * O^T
+                    if (tid == 0) post(kCmdWo, 0);
+                    // meanwhile: request the next tile's input rows (the layer below has finished them)
+                    const bool pre_ok = want_pre && misc->pre_ok != 0;
+                    Piece xpre;
+                    if (pre_ok) xpre = load_input(v_pre);
+                    if (!mbar_wait(bar1, ph1, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph1 ^= 1u;
+                    tc_fence_after();
+                    {
+                        uint32_t d[8];
+                        tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * kAccO + cg * 8), d);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int nn = 0; nn < 8; ++nn) {
+                            const int node = cg * 8 + nn;
+                            const uint16_t rb = p.residual ? ld_shared_b16(sHres_cur + (uint32_t)(node * 256 + feat * 2)) : (uint16_t)0;
+                            const float val = __uint_as_float(d[nn]) + __uint_as_float((uint32_t)rb << 16);
+                            st_shared_b16(sHp + operand_offset(node, feat), bf16_bits(val));
+                        }
+                    }
+                    if (pre_ok) stage_input(buf ^ 1, xpre);
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    worker_sync();
+
+                    // ---- from the new rows, transposed: this layer's K | V refresh; right behind it, the next tile's
+                    // Q | K | V (it runs while this tile's rows are stored and the level completes)
+                    if (tid == 0) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
+                    // meanwhile: the new rows go to H (16 lanes cover one 256-byte row)
+                    const int node_v = misc->node[slot];
+                    {
+                        uint32_t w4[4];
+                        ld_shared_v4(sHp + operand_piece(slot, sub), w4);
+                        if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
+                    }
+                    if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph2 ^= 1u;
+                    tc_fence_after();
+                    {
+                        uint32_t d[2][8];
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk)
+                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk) {
                             const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
 #pragma unroll
                             for (int nn = 0; nn < 8; ++nn)
                                 st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
                         }
                     }
-                }
-                tc_fence_before();
-                __syncthreads();
-                if (node_v >= 0) {
-                    const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
-                    uint32_t w4[4];
+                    tc_fence_before();
+                    worker_sync();
+                    if (node_v >= 0) {
+                        const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
+                        uint32_t w4[4];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {        // this layer's K | V row
-                        ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
-                        st_global_v4((char*)p.KV[layer] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
-                    }
-                    if (has_next) {                      // the next layer's Q row and (not yet updated) K | V row
-                        ld_shared_v4(row + (uint32_t)(512 + sub * 16), w4);
-                        st_global_v4((char*)p.Q[layer + 1] + (size_t)node_v * 256 + sub * 16, w4);
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            ld_shared_v4(row + (uint32_t)(768 + (sub + 16 * h) * 16), w4);
-                            st_global_v4((char*)p.KV[layer + 1] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
+                        for (int h = 0; h < 2; ++h) {        // this layer's K | V row
+                            ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
+                            st_global_v4((char*)p.KV[layer] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
                         }
                     }
+                    worker_sync();    // the tile's shared buffers may be overwritten from here on
+                    pro_ready = pre_ok;
+                    if (pre_ok) buf ^= 1;
                 }
-                __syncthreads();    // the tile's shared buffers may be overwritten from here on
+                if (!alive) break;
+                // ---- this CTA's part of (layer, level l) is in global memory: arrive on its counter (release)
+                // (by a thread that does not poll: the release waits for the CTA's outstanding stores, and the pollers
+                // should already be watching the next level's counters meanwhile)
+                if (tid == 64) red_release_add(my_arrive + l, 1);
+            } else if (!pro_ready && l + 1 < p.n_levels && bid < tiles_next) {
+                // ---- no tile in this level but one in the next: bring that tile up while there is nothing else to do
+                if (tid == 32) {
+                    bool go = true;
+                    if (prev_arrive) go = wait_counter(prev_arrive + l + 1, prev_target(tiles_next), p.abort_word, counter_limit);
+                    if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                    misc->go2 = go ? 1 : 0;
+                }
+                worker_sync();
+                if (!misc->go2) { alive = false; break; }
+                stage_input(buf, load_input(vC));
+                fence_proxy_async_smem();
+                worker_sync();
+                if (tid == 0) post(kCmdQkv, buf);
+                pro_ready = true;
             }
-            if (!alive) break;
-            // ---- this CTA's part of (layer, level l) is in global memory: arrive on its counter (release)
-            // (by a thread that does not poll: the release waits for the CTA's outstanding stores, and the pollers
-            // should already be watching the next level's counters meanwhile)
-            if (tid == 64) red_release_add(my_arrive + l, 1);
+            if (n_l > 0) {
+                last_nonempty = l;
+                last_participants = tiles < nctas ? tiles : nctas;
+            }
+            // rotate the pipeline by one level
+            v0 = vC; pad0 = padC;
+            vC = vB;
+            lp0 = lp1; lp1 = lp2; lp2 = lp3; lp3 = lp4;
         }
-        if (n_l > 0) {
-            last_nonempty = l;
-            last_participants = tiles < nctas ? tiles : nctas;
-        }
-        // rotate the pipeline by one level
-        v0 = vC; pad0 = padC;
-        vC = vB;
-        lp0 = lp1; lp1 = lp2; lp2 = lp3; lp3 = lp4;
+        if (tid == 0) post(kCmdExit, 0);
     }
 
-    // Tensor memory is freed below: every MMA this CTA issued must have completed.  Normally each was waited for
-    // right after it was issued; after a wait that ran out, one may still be in flight.
-    if (tid == 0) {
-        mma_commit(smem_u32(&misc->drain));
-        mbar_wait(smem_u32(&misc->drain), 0);
-    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -478,7 +627,7 @@ size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers) {
     return ((size_t)g->n_levels * (size_t)n_layers + 64) * sizeof(int32_t);
 }
 
-dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers, __nv_bfloat16* const* Q,
+dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers,
                                  __nv_bfloat16* const* KV, __nv_bfloat16* H, int64_t ldh,
                                  const __nv_bfloat16* const* W_qkv, const __nv_bfloat16* const* W_o, int32_t* sync,
                                  int32_t* status, cudaStream_t st) {
@@ -502,7 +651,6 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         const int kk = k < n_layers ? k : 0;           // unused slots repeat layer 0 (never read)
         p.Wo[k] = W_o[kk];
         p.Wqkv[k] = W_qkv[kk];
-        p.Q[k] = Q[kk];
         p.KV[k] = KV[kk];
     }
     DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, n_layers), st));
