@@ -355,6 +355,12 @@ dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, vo
  * Attention being dg4_qkv_project + dg4_sparse_attn_fwd on the handle's neighbourhoods (desc gives heads and
  * scale; the residual connections are always on).  workspace: dg4_layer_workspace_bytes() bytes, 256-byte aligned,
  * owned by the caller; the library allocates nothing.  H_out may be H_in.
+ *
+ * dg4_block_fwd_levelised: the same block in the paper's level-by-level order (Sec. 1 and Sec. 3.4 for the order,
+ * Sec. 3.5 for the block), in place on H: levels 0, 1, ... in turn; a node takes its query and its own key / value
+ * from its row as it was when the call started, and the key / value of every other member of N(v) from that node's
+ * row as already replaced by this call, i.e. from its BLOCK output.  One group of kernel launches per level (the
+ * level's rows are taken through the handle's level buckets); cones of any supported width.
  */
 dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
                              const float* gamma, const float* beta, float eps, void* Y, int64_t ldy, void* stream);
@@ -366,6 +372,11 @@ dg4_status dg4_block_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, cons
                                   const void* W1, const float* b1, const void* W2, const float* b2,
                                   const float* ln2_gamma, const float* ln2_beta, float eps, int32_t d_ff,
                                   void* H_out, int64_t ldho, void* workspace, size_t workspace_bytes, void* stream);
+dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                   const void* W_qkv, const void* W_o, const float* ln1_gamma, const float* ln1_beta,
+                                   const void* W1, const float* b1, const void* W2, const float* b2,
+                                   const float* ln2_gamma, const float* ln2_beta, float eps, int32_t d_ff,
+                                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Diagnostic (the paper has no counterpart): launches one small CTA that waits, with the same bounded wait the

@@ -27,6 +27,8 @@
  *   orc_layer_levelised   the same layer applied level by level in topological order, each level
  *                         reading the rows already updated for earlier levels (Sec. 1 and Sec. 3.4:
  *                         each gate is computed once, in strict level order)
+ *   orc_block_levelised   the whole block (attention sub-layer, LayerNorm, feed-forward sub-layer, LayerNorm) in the same
+ *                         level-by-level order
  *   orc_partition_roots   Algorithm 1 (graph partition): which nodes' cones the partition collects
  *   orc_cone_update       Sec. 3.4 (intra- and inter-level updating) with the loop of Algorithm 2: cone mini-batches
  *                         encoded group by group against a table of historical embeddings
@@ -395,6 +397,62 @@ void orc_layer_levelised(int n, int d, int heads, double scale, double* H, const
             double* dst = fresh.data() + (int64_t)(i - lo) * d;
             project_row(d, d, o.data(), W_o, residual ? H + (int64_t)v * d : nullptr, dst);
             for (int c = 0; c < d; ++c) dst[c] = store_round(dst[c], rounding);
+        }
+        for (int i = lo; i < hi; ++i)
+            std::memcpy(H + (int64_t)level_nodes[i] * d, fresh.data() + (int64_t)(i - lo) * d, sizeof(double) * d);
+    }
+}
+
+/* The whole Transformer block (Sec. 3.5: the attention module is replaced, the rest of the post-norm block is kept)
+ * applied level by level, in place on H: a node v of bucket l takes its query and its own key / value from its
+ * current (not yet updated) row, the key / value of every other neighbour from that neighbour's row as already
+ * updated in this sweep -- i.e. from the neighbour's BLOCK output -- and its new row is
+ *     H1 = LayerNorm_1(H[v] + Attention * W_o^T),   H[v] <- LayerNorm_2(H1 + FFN(H1)).
+ * rounding 1: Q, K, V, O, the sum before LayerNorm_1, H1, the hidden activations and the new row are rounded to
+ * bfloat16 (the places where an implementation with 16-bit storage has to round). */
+void orc_block_levelised(int n, int d, int heads, double scale, double* H, const double* W_qkv, const double* W_o,
+                         const double* g1, const double* be1, int d_ff, const double* W1, const double* b1,
+                         const double* W2, const double* b2, const double* g2, const double* be2, double eps,
+                         const int32_t* nbr_ptr, const int32_t* nbr_idx, int n_levels, const int32_t* level_ptr,
+                         const int32_t* level_nodes, int rounding) {
+    (void)n;
+    int dh = d / heads;
+    const double* Wq = W_qkv;
+    const double* Wk = W_qkv + (int64_t)d * d;
+    const double* Wv = W_qkv + (int64_t)2 * d * d;
+    for (int lev = 0; lev < n_levels; ++lev) {
+        const int lo = level_ptr[lev], hi = level_ptr[lev + 1];
+        std::vector<double> fresh((int64_t)(hi - lo) * d);
+#pragma omp parallel for schedule(static)
+        for (int i = lo; i < hi; ++i) {
+            int v = level_nodes[i];
+            int b = nbr_ptr[v], cnt = nbr_ptr[v + 1] - b;
+            std::vector<double> q(d), kk((int64_t)cnt * d), vv((int64_t)cnt * d), o(d), pre(d), h1(d);
+            project_row(d, d, H + (int64_t)v * d, Wq, nullptr, q.data());
+            for (int j = 0; j < cnt; ++j) {
+                int64_t u = nbr_idx[b + j];
+                project_row(d, d, H + u * d, Wk, nullptr, kk.data() + (int64_t)j * d);
+                project_row(d, d, H + u * d, Wv, nullptr, vv.data() + (int64_t)j * d);
+            }
+            for (int c = 0; c < d; ++c) q[c] = store_round(q[c], rounding);
+            for (int64_t c = 0; c < (int64_t)cnt * d; ++c) {
+                kk[c] = store_round(kk[c], rounding);
+                vv[c] = store_round(vv[c], rounding);
+            }
+            std::vector<const double*> kr(cnt), vr(cnt);
+            for (int h = 0; h < heads; ++h) {
+                for (int j = 0; j < cnt; ++j) {
+                    kr[j] = kk.data() + (int64_t)j * d + h * dh;
+                    vr[j] = vv.data() + (int64_t)j * d + h * dh;
+                }
+                attend_one(dh, scale, q.data() + h * dh, cnt, kr.data(), vr.data(), o.data() + h * dh, nullptr);
+            }
+            for (int c = 0; c < d; ++c) o[c] = store_round(o[c], rounding);
+            project_row(d, d, o.data(), W_o, H + (int64_t)v * d, pre.data());
+            for (int c = 0; c < d; ++c) pre[c] = store_round(pre[c], rounding);
+            orc_layernorm(1, d, pre.data(), g1, be1, eps, h1.data());
+            for (int c = 0; c < d; ++c) h1[c] = store_round(h1[c], rounding);
+            orc_ffn(1, d, d_ff, h1.data(), W1, b1, W2, b2, g2, be2, eps, rounding, fresh.data() + (int64_t)(i - lo) * d);
         }
         for (int i = lo; i < hi; ++i)
             std::memcpy(H + (int64_t)level_nodes[i] * d, fresh.data() + (int64_t)(i - lo) * d, sizeof(double) * d);

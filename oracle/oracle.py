@@ -65,6 +65,9 @@ def _load():
         lib.orc_layer_levelised.restype = None
         lib.orc_layer_levelised.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, c_int, _i32p, _i32p,
                                             c_int, _i32p, _i32p, c_int]
+        lib.orc_block_levelised.restype = None
+        lib.orc_block_levelised.argtypes = [c_int, c_int, c_int, c_dbl, _f64p, _f64p, _f64p, _f64p, _f64p, c_int, _f64p, _f64p,
+                                            _f64p, _f64p, _f64p, _f64p, c_dbl, _i32p, _i32p, c_int, _i32p, _i32p, c_int]
         lib.orc_cone_update.restype = c_int
         lib.orc_cone_update.argtypes = [c_int, c_int, c_int, c_dbl, c_int, _f64p, _f64p, _f64p, c_int, _i32p, _i32p, _i32p,
                                         c_int, c_int, c_int, c_int, c_int, _f64p, _i32p]
@@ -243,6 +246,20 @@ def layer_levelised(H, W_qkv, W_o, nbr_ptr, nbr_idx, level_ptr, level_nodes, hea
     _load().orc_layer_levelised(n, d, heads, float(scale), _d(H), _d(W_qkv), _d(W_o), int(bool(residual)),
                                 _i(nbr_ptr), _i(nbr_idx), level_ptr.shape[0] - 1, _i(level_ptr), _i(level_nodes),
                                 ROUND[rounding])
+    return H
+
+
+def block_levelised(H, W_qkv, W_o, ln1_gamma, ln1_beta, W1, b1, W2, b2, ln2_gamma, ln2_beta, nbr_ptr, nbr_idx, level_ptr,
+                    level_nodes, heads, scale, eps=1e-5, rounding=None):
+    """The whole block (attention sub-layer + LayerNorm, feed-forward sub-layer + LayerNorm) level by level."""
+    H = _f64(H).copy()
+    W_qkv, W_o, W1, W2 = _f64(W_qkv), _f64(W_o), _f64(W1), _f64(W2)
+    g1, be1, b1, b2, g2, be2 = (_f64(a) for a in (ln1_gamma, ln1_beta, b1, b2, ln2_gamma, ln2_beta))
+    nbr_ptr, nbr_idx, level_ptr, level_nodes = _i32(nbr_ptr), _i32(nbr_idx), _i32(level_ptr), _i32(level_nodes)
+    n, d = H.shape
+    _load().orc_block_levelised(n, d, heads, float(scale), _d(H), _d(W_qkv), _d(W_o), _d(g1), _d(be1), W1.shape[0],
+                                _d(W1), _d(b1), _d(W2), _d(b2), _d(g2), _d(be2), float(eps), _i(nbr_ptr), _i(nbr_idx),
+                                level_ptr.shape[0] - 1, _i(level_ptr), _i(level_nodes), ROUND[rounding])
     return H
 
 

@@ -30,7 +30,8 @@ namespace {
 using namespace sm100;
 
 constexpr int kTileM = 128;                 // rows per tile
-constexpr int kThreads = 256;
+constexpr int kWorkers = 256;               // eight warps: epilogues of both products
+constexpr int kThreads = kWorkers + 32;     // and a ninth warp whose first lane issues every tcgen05.mma
 constexpr int kHalf = 128 * 128;            // bytes of one K-half (64 bf16 columns) of a 128-row operand tile
 constexpr int kTileBytes = 2 * kHalf;       // 32 KiB: a 128 x 128 bf16 operand tile
 constexpr int kOffW2 = 0;                   // 4 chunks of W2
@@ -44,6 +45,8 @@ constexpr int kColD1 = 0, kColD2 = 128, kColW1 = 256, kTmemCols = 512;
 struct Misc {
     uint64_t bar_w, bar_x[2], bar_g1, bar_g2, bar_drain;
     uint32_t tmem_base;
+    int32_t posted;            // products the workers have released to the issuing thread so far (monotone)
+    int32_t stop;              // the workers are leaving: no further products
 };
 
 struct FfnParams {
@@ -56,7 +59,19 @@ struct FfnParams {
     int32_t n_tiles;
     int32_t* status;
     uint32_t poll_limit;      // polls after which a pipeline wait gives up
+    // rows taken from a list (the level-by-level block): X and Y are then addressed directly, not through tensor maps
+    const int32_t* row_list;
+    int32_t first, rows;
+    const __nv_bfloat16* X; int64_t ldx;
+    __nv_bfloat16* Y; int64_t ldy;
 };
+
+__device__ __forceinline__ void ld_nc_v4(const void* p, uint32_t* r) {
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p));
+}
+__device__ __forceinline__ void st_global_v4(void* p, const uint32_t* r) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
@@ -87,6 +102,14 @@ __device__ __forceinline__ void relu_pack_store2(uint32_t addr_lo, uint32_t addr
         "st.shared.b16 [%1], h;\n\t}"
         ::"r"(addr_lo), "r"(addr_hi), "f"(lo), "f"(hi) : "memory");
 }
+// barrier (and barrier with an OR reduction) among the eight worker warps only
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
+__device__ __forceinline__ bool worker_sync_or(bool flag) {
+    uint32_t out;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.or.pred q, 1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(out) : "r"(flag ? 1u : 0u), "n"(kWorkers) : "memory");
+    return out != 0;
+}
 // byte offset of element k (0..127) of row `row` in a 128-row operand tile (two K-halves, 128-byte swizzle)
 __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
     return (uint32_t)((k >> 6) * kHalf) + sw128_offset(row, (k & 63) >> 3) + (uint32_t)((k & 7) * 2);
@@ -94,6 +117,7 @@ __device__ __forceinline__ uint32_t operand_offset(int row, int k) {
 // descriptor address increment of K-step ks (16 elements) inside an operand tile
 __device__ __forceinline__ uint64_t kstep(int ks) { return (uint64_t)(((ks >> 2) * kHalf + (ks & 3) * 32) >> 4); }
 
+template <bool LISTED>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w2,
            const __grid_constant__ CUtensorMap map_y, FfnParams p) {
@@ -117,6 +141,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         mbar_init(bar_g1, 1);
         mbar_init(bar_g2, 1);
         mbar_init(smem_u32(&misc->bar_drain), 1);
+        misc->posted = 0;
+        misc->stop = 0;
         mbar_fence_init();
         tma_prefetch_desc(&map_x);
         tma_prefetch_desc(&map_w2);
@@ -126,8 +152,10 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
             for (int q = 0; q < 4; ++q)
                 for (int h = 0; h < 2; ++h)
                     tma_load_2d(sW2 + q * kTileBytes + h * kHalf, &map_w2, q * 128 + h * 64, 0, bar_w);
-            mbar_expect_tx(bar_x[0], kTileBytes);
-            for (int h = 0; h < 2; ++h) tma_load_2d(sX + h * kHalf, &map_x, h * 64, first_tile * kTileM, bar_x[0]);
+            if (!LISTED) {
+                mbar_expect_tx(bar_x[0], kTileBytes);
+                for (int h = 0; h < 2; ++h) tma_load_2d(sX + h * kHalf, &map_x, h * 64, first_tile * kTileM, bar_x[0]);
+            }
         }
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
@@ -137,184 +165,247 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
     const uint32_t tmem = misc->tmem_base;
 
     // W1 into tensor memory: hidden unit `ln` of block q in lane `ln`, two consecutive inputs per 32-bit column
-    // (the bytes as they lie in global memory); each thread copies half a row (128 bytes) of every block.
-    float b1v[4];
-    for (int q = 0; q < 4; ++q) {
-        const uint4* src = reinterpret_cast<const uint4*>(p.W1 + (size_t)(q * 128 + ln) * 128 + cg * 64);
+    // (the bytes as they lie in global memory); each worker thread copies half a row (128 bytes) of every block.
+    float b1v[4] = {0.f, 0.f, 0.f, 0.f};
+    if (warp < 8) {
+        for (int q = 0; q < 4; ++q) {
+            const uint4* src = reinterpret_cast<const uint4*>(p.W1 + (size_t)(q * 128 + ln) * 128 + cg * 64);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint4 lo = src[2 * c], hi = src[2 * c + 1];
-            const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-            tmem_st_32x8(tmem + lane_base + (uint32_t)(kColW1 + q * 64 + cg * 32 + c * 8), r);
+            for (int c = 0; c < 4; ++c) {
+                const uint4 lo = src[2 * c], hi = src[2 * c + 1];
+                const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                tmem_st_32x8(tmem + lane_base + (uint32_t)(kColW1 + q * 64 + cg * 32 + c * 8), r);
+            }
+            b1v[q] = p.b1[q * 128 + ln];
         }
-        b1v[q] = p.b1[q * 128 + ln];
+        tmem_st_wait();
     }
-    tmem_st_wait();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 
     const uint32_t idesc = idesc_bf16_f32(128, 128);
-    uint32_t a2_base[8];                                 // where this thread's hidden unit lies in rows cg*64 + (0..7)
-#pragma unroll
-    for (int k = 0; k < 8; ++k) a2_base[k] = sA2 + operand_offset(cg * 64 + k, ln) - (uint32_t)(k * 128);
     const uint64_t dA2 = smem_desc_sw128(sA2);
-    uint32_t ph_g1 = 0, ph_g2 = 0;
-    bool failed = false;
-    if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0, p.poll_limit);
 
-    int it = 0;
-    for (int tile = first_tile; tile < p.n_tiles; tile += (int)gridDim.x, ++it) {
-        const int s = it & 1;
-        const uint32_t sXs = sX + s * kTileBytes;
-        const uint64_t dX = smem_desc_sw128(sXs);
-        if (tid == 0) {
-            const int next = tile + (int)gridDim.x;      // prefetch the next tile's rows into the other stage
-            if (next < p.n_tiles) {
-                mbar_expect_tx(bar_x[s ^ 1], kTileBytes);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
-            }
-        }
-        failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u, p.poll_limit);
-
-        auto issue_g1 = [&](int q) {     // D1^T = W1_q * X^T
+    if (warp == 8) {
+        // ------------------------------------------------------------------ the issuing thread
+        // The order of the products is fixed (per tile: G1(0) G1(1) G2(0) G1(2) G2(1) G1(3) G2(2) G2(3)), so the
+        // workers only release them one by one: `posted` counts the releases.  Issuing a product keeps the issuing
+        // thread busy for about as long as the tensor pipe needs to execute it, which is why no worker does it.
+        if (lane == 0) {
+            int consumed = 0;
+            bool leave = false;
+            const uint32_t token_limit = p.poll_limit < (1u << 28) ? p.poll_limit << 2 : p.poll_limit;
+            int it = 0;
+            for (int tile = first_tile; tile < p.n_tiles && !leave; tile += (int)gridDim.x, ++it) {
+                const uint64_t dX = smem_desc_sw128(sX + (it & 1) * kTileBytes);
+                for (int step = 0; step < 8 && !leave; ++step) {
+                    uint32_t polls = 0;
+                    while (*reinterpret_cast<volatile int32_t*>(&misc->posted) <= consumed) {
+                        if (*reinterpret_cast<volatile int32_t*>(&misc->stop) != 0 || ++polls > token_limit) { leave = true; break; }
+                        if (polls > 256) __nanosleep(20);
+                    }
+                    if (leave || *reinterpret_cast<volatile int32_t*>(&misc->stop) != 0) { leave = true; break; }
+                    ++consumed;
+                    __threadfence_block();
+                    tc_fence_after();
+                    // steps 0, 1, 3, 5 are first products of blocks 0..3; steps 2, 4, 6, 7 second products of blocks 0..3
+                    const bool first_product = (step == 0) || (step == 1) || (step == 3) || (step == 5);
+                    const int q = first_product ? (step + 1) / 2 : (step == 7 ? 3 : step / 2 - 1);
+                    if (first_product) {             // D1^T = W1_q * X^T
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_bf16_ta(tmem + kColD1, tmem + (uint32_t)(kColW1 + q * 64 + ks * 8), dX + kstep(ks), idesc, ks > 0 ? 1u : 0u);
+                        for (int ks = 0; ks < 8; ++ks)
+                            mma_bf16_ta(tmem + kColD1, tmem + (uint32_t)(kColW1 + q * 64 + ks * 8), dX + kstep(ks), idesc, ks > 0 ? 1u : 0u);
+                        mma_commit(bar_g1);
+                    } else {                         // D2 += A2 * W2_q^T
+                        const uint64_t dW2 = smem_desc_sw128(sW2 + q * kTileBytes);
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            mma_bf16(tmem + kColD2, dA2 + kstep(ks), dW2 + kstep(ks), idesc, (q > 0 || ks > 0) ? 1u : 0u);
+                        mma_commit(bar_g2);
+                    }
+                }
+            }
+            // tensor memory is freed below: every product issued must have completed
+            mma_commit(smem_u32(&misc->bar_drain));
+            mbar_wait(smem_u32(&misc->bar_drain), 0);
+        }
+    } else {
+        // ------------------------------------------------------------------ the eight worker warps
+        auto release_product = [&]() {               // one worker thread, after the barrier that made the operands visible
+            __threadfence_block();
+            *reinterpret_cast<volatile int32_t*>(&misc->posted) = misc->posted + 1;
         };
-        if (tid == 0) {
-            tc_fence_after();
-            issue_g1(0);
-            mma_commit(bar_g1);
-        }
+        uint32_t a2_base[8];                             // where this thread's hidden unit lies in rows cg*64 + (0..7)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a2_base[k] = sA2 + operand_offset(cg * 64 + k, ln) - (uint32_t)(k * 128);
+        uint32_t ph_g1 = 0, ph_g2 = 0;
+        bool failed = false;
+        if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0, p.poll_limit);
 
-        // Per block q of hidden units: the accumulator is read into registers, the next block's first product is
-        // issued at once (it runs while the values are scattered into the operand buffer), then the second
-        // product of this block.  The tensor pipe executes in issue order: G1(0) G1(1) G2(0) G1(2) G2(1) ...
-        for (int q = 0; q < 4; ++q) {
-            failed |= !mbar_wait(bar_g1, ph_g1, p.poll_limit);         // D1^T of block q is complete
-            ph_g1 ^= 1u;
-            tc_fence_after();
-            uint32_t d[64];
-            tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64), d);
-            tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + 32), d + 32);
-            tmem_ld_wait();
-            tc_fence_before();
-            if (q == 0 && tid == 0) bulk_wait_read0();   // the previous tile's store has read the staging buffer
-            __syncthreads();                             // every thread holds its part of D1^T
-            if (tid == 0 && q < 3) {
-                tc_fence_after();
-                issue_g1(q + 1);
-                mma_commit(bar_g1);
+        int it = 0;
+        for (int tile = first_tile; tile < p.n_tiles; tile += (int)gridDim.x, ++it) {
+            const int s = it & 1;
+            const uint32_t sXs = sX + s * kTileBytes;
+            if (!LISTED) {
+                if (tid == 0) {
+                    const int next = tile + (int)gridDim.x;      // prefetch the next tile's rows into the other stage
+                    if (next < p.n_tiles) {
+                        mbar_expect_tx(bar_x[s ^ 1], kTileBytes);
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
+                    }
+                }
+                failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u, p.poll_limit);
+            } else {
+                // listed rows: the workers gather the tile's rows into the same swizzled layout, 16 bytes at a time
+                for (int i = tid; i < kTileM * 16; i += kWorkers) {
+                    const int row = i >> 4, chunk = i & 15;
+                    const int r = tile * kTileM + row;
+                    uint32_t v[4] = {0u, 0u, 0u, 0u};
+                    if (r < p.rows) ld_nc_v4(p.X + (int64_t)p.row_list[p.first + r] * p.ldx + chunk * 8, v);
+                    st_shared_v4(sXs + (uint32_t)((chunk >> 3) * kHalf) + sw128_offset(row, chunk & 7), v);
+                }
+                fence_proxy_async_smem();
             }
-            if (q > 0) {                                 // the previous block's second product has read the buffer
-                failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);
-                ph_g2 ^= 1u;
-            }
-            // rows cg*64 + j: element `ln` of row j lies at a2_base[j & 7] + 128 j (the swizzle depends on j & 7
-            // only, because cg*64 is a multiple of 8); two rows per conversion, ReLU folded into it
-            const float bq = b1v[q];
-#pragma unroll
-            for (int j = 0; j < 64; j += 2)
-                relu_pack_store2(a2_base[j & 7] + (uint32_t)(j * 128), a2_base[(j + 1) & 7] + (uint32_t)((j + 1) * 128),
-                                 __uint_as_float(d[j]) + bq, __uint_as_float(d[j + 1]) + bq);
-            fence_proxy_async_smem();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-                const uint64_t dW2 = smem_desc_sw128(sW2 + q * kTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)           // D2 += A2 * W2_q^T
-                    mma_bf16(tmem + kColD2, dA2 + kstep(ks), dW2 + kstep(ks), idesc, (q > 0 || ks > 0) ? 1u : 0u);
-                mma_commit(bar_g2);
-            }
-        }
-        failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);    // D2 is complete; the activation buffer is free
-        ph_g2 ^= 1u;
-        tc_fence_after();
+            // the X tile has landed for every worker before the first product is released (the barrier also
+            // separates the previous tile's reads of its buffers from this tile's writes)
+            worker_sync();
+            if (tid == 0) release_product();             // G1(0)
 
-        // ---- final epilogue: thread = row `ln`, columns cg*64 .. cg*64+63
-        {
-            float y[64];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t d[32];
-                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64 + half * 32), d);
+            // Per block q of hidden units: the accumulator is read into registers, the next block's first product is
+            // released at once (it runs while the values are scattered into the operand buffer), then the second
+            // product of this block.  The tensor pipe executes in issue order: G1(0) G1(1) G2(0) G1(2) G2(1) ...
+            for (int q = 0; q < 4; ++q) {
+                failed |= !mbar_wait(bar_g1, ph_g1, p.poll_limit);         // D1^T of block q is complete
+                ph_g1 ^= 1u;
+                tc_fence_after();
+                uint32_t d[64];
+                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64), d);
+                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + 32), d + 32);
                 tmem_ld_wait();
+                tc_fence_before();
+                if (!LISTED && q == 0 && tid == 0) bulk_wait_read0();   // the previous tile's store has read the staging buffer
+                worker_sync();                               // every thread holds its part of D1^T
+                if (tid == 0 && q < 3) release_product();    // G1(q + 1)
+                if (q > 0) {                                 // the previous block's second product has read the buffer
+                    failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);
+                    ph_g2 ^= 1u;
+                }
+                // rows cg*64 + j: element `ln` of row j lies at a2_base[j & 7] + 128 j (the swizzle depends on j & 7
+                // only, because cg*64 is a multiple of 8); two rows per conversion, ReLU folded into it
+                const float bq = b1v[q];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) y[half * 32 + j] = __uint_as_float(d[j]);
+                for (int j = 0; j < 64; j += 2)
+                    relu_pack_store2(a2_base[j & 7] + (uint32_t)(j * 128), a2_base[(j + 1) & 7] + (uint32_t)((j + 1) * 128),
+                                     __uint_as_float(d[j]) + bq, __uint_as_float(d[j + 1]) + bq);
+                fence_proxy_async_smem();
+                worker_sync();
+                if (tid == 0) release_product();             // G2(q)
             }
-            tc_fence_before();
-            const float4* b2v = reinterpret_cast<const float4*>(p.b2 + cg * 64);
+            failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);   // D2 is complete; the activation buffer is free
+            ph_g2 ^= 1u;
+            tc_fence_after();
+
+            // ---- final epilogue: thread = row `ln`, columns cg*64 .. cg*64+63
+            {
+                float y[64];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {                // + b2 + the row of X (K-half cg of the X tile)
-                uint32_t w[4];
-                ld_shared_v4(sXs + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
-                const float4 ba = __ldg(b2v + 2 * c), bb = __ldg(b2v + 2 * c + 1);
-                y[c * 8 + 0] += __uint_as_float(w[0] << 16) + ba.x;
-                y[c * 8 + 1] += __uint_as_float(w[0] & 0xffff0000u) + ba.y;
-                y[c * 8 + 2] += __uint_as_float(w[1] << 16) + ba.z;
-                y[c * 8 + 3] += __uint_as_float(w[1] & 0xffff0000u) + ba.w;
-                y[c * 8 + 4] += __uint_as_float(w[2] << 16) + bb.x;
-                y[c * 8 + 5] += __uint_as_float(w[2] & 0xffff0000u) + bb.y;
-                y[c * 8 + 6] += __uint_as_float(w[3] << 16) + bb.z;
-                y[c * 8 + 7] += __uint_as_float(w[3] & 0xffff0000u) + bb.w;
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t d[32];
+                    tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64 + half * 32), d);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) y[half * 32 + j] = __uint_as_float(d[j]);
+                }
+                tc_fence_before();
+                const float4* b2v = reinterpret_cast<const float4*>(p.b2 + cg * 64);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {                // + b2 + the row of X (K-half cg of the X tile)
+                    uint32_t w[4];
+                    ld_shared_v4(sXs + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
+                    const float4 ba = __ldg(b2v + 2 * c), bb = __ldg(b2v + 2 * c + 1);
+                    y[c * 8 + 0] += __uint_as_float(w[0] << 16) + ba.x;
+                    y[c * 8 + 1] += __uint_as_float(w[0] & 0xffff0000u) + ba.y;
+                    y[c * 8 + 2] += __uint_as_float(w[1] << 16) + ba.z;
+                    y[c * 8 + 3] += __uint_as_float(w[1] & 0xffff0000u) + ba.w;
+                    y[c * 8 + 4] += __uint_as_float(w[2] << 16) + bb.x;
+                    y[c * 8 + 5] += __uint_as_float(w[2] & 0xffff0000u) + bb.y;
+                    y[c * 8 + 6] += __uint_as_float(w[3] << 16) + bb.z;
+                    y[c * 8 + 7] += __uint_as_float(w[3] & 0xffff0000u) + bb.w;
+                }
+                // mean and sum of squared deviations of the half-row, merged with the other half-row's
+                float m = 0.0f;
+#pragma unroll
+                for (int j = 0; j < 64; ++j) m += y[j];
+                m *= (1.0f / 64.0f);
+                float m2 = 0.0f;
+#pragma unroll
+                for (int j = 0; j < 64; ++j) m2 += (y[j] - m) * (y[j] - m);
+                st_shared_f2(sA2 + (uint32_t)((ln * 2 + cg) * 8), m, m2);
+                worker_sync();
+                float mo, m2o;
+                ld_shared_f2(sA2 + (uint32_t)((ln * 2 + (cg ^ 1)) * 8), mo, m2o);
+                worker_sync();
+                const float mean = 0.5f * (m + mo);
+                const float var = (m2 + m2o + 32.0f * (m - mo) * (m - mo)) * (1.0f / 128.0f);
+                const float rstd = rsqrtf(var + p.eps);
+                const float4* gv = reinterpret_cast<const float4*>(p.gamma + cg * 64);
+                const float4* bv = reinterpret_cast<const float4*>(p.beta + cg * 64);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float4 ga = __ldg(gv + 2 * c), gb = __ldg(gv + 2 * c + 1);
+                    const float4 ba = __ldg(bv + 2 * c), bb = __ldg(bv + 2 * c + 1);
+                    uint32_t w[4];
+                    w[0] = pack_bf16((y[c * 8 + 0] - mean) * rstd * ga.x + ba.x, (y[c * 8 + 1] - mean) * rstd * ga.y + ba.y);
+                    w[1] = pack_bf16((y[c * 8 + 2] - mean) * rstd * ga.z + ba.z, (y[c * 8 + 3] - mean) * rstd * ga.w + ba.w);
+                    w[2] = pack_bf16((y[c * 8 + 4] - mean) * rstd * gb.x + bb.x, (y[c * 8 + 5] - mean) * rstd * gb.y + bb.y);
+                    w[3] = pack_bf16((y[c * 8 + 6] - mean) * rstd * gb.z + bb.z, (y[c * 8 + 7] - mean) * rstd * gb.w + bb.w);
+                    st_shared_v4(sA2 + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
+                }
             }
-            // mean and sum of squared deviations of the half-row, merged with the other half-row's
-            float m = 0.0f;
-#pragma unroll
-            for (int j = 0; j < 64; ++j) m += y[j];
-            m *= (1.0f / 64.0f);
-            float m2 = 0.0f;
-#pragma unroll
-            for (int j = 0; j < 64; ++j) m2 += (y[j] - m) * (y[j] - m);
-            st_shared_f2(sA2 + (uint32_t)((ln * 2 + cg) * 8), m, m2);
-            __syncthreads();
-            float mo, m2o;
-            ld_shared_f2(sA2 + (uint32_t)((ln * 2 + (cg ^ 1)) * 8), mo, m2o);
-            __syncthreads();
-            const float mean = 0.5f * (m + mo);
-            const float var = (m2 + m2o + 32.0f * (m - mo) * (m - mo)) * (1.0f / 128.0f);
-            const float rstd = rsqrtf(var + p.eps);
-            const float4* gv = reinterpret_cast<const float4*>(p.gamma + cg * 64);
-            const float4* bv = reinterpret_cast<const float4*>(p.beta + cg * 64);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 ga = __ldg(gv + 2 * c), gb = __ldg(gv + 2 * c + 1);
-                const float4 ba = __ldg(bv + 2 * c), bb = __ldg(bv + 2 * c + 1);
-                uint32_t w[4];
-                w[0] = pack_bf16((y[c * 8 + 0] - mean) * rstd * ga.x + ba.x, (y[c * 8 + 1] - mean) * rstd * ga.y + ba.y);
-                w[1] = pack_bf16((y[c * 8 + 2] - mean) * rstd * ga.z + ba.z, (y[c * 8 + 3] - mean) * rstd * ga.w + ba.w);
-                w[2] = pack_bf16((y[c * 8 + 4] - mean) * rstd * gb.x + bb.x, (y[c * 8 + 5] - mean) * rstd * gb.y + bb.y);
-                w[3] = pack_bf16((y[c * 8 + 6] - mean) * rstd * gb.z + bb.z, (y[c * 8 + 7] - mean) * rstd * gb.w + bb.w);
-                st_shared_v4(sA2 + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
+            fence_proxy_async_smem();
+            const bool stop = worker_sync_or(failed);        // also: the X stage may be refilled from here on
+            if (!LISTED) {
+                if (tid == 0 && !stop) {
+                    tma_store_2d(&map_y, 0, tile * kTileM, sA2);
+                    tma_store_2d(&map_y, 64, tile * kTileM, sA2 + kHalf);
+                    bulk_commit();
+                }
+            } else if (!stop) {
+                for (int i = tid; i < kTileM * 16; i += kWorkers) {
+                    const int row = i >> 4, chunk = i & 15;
+                    const int r = tile * kTileM + row;
+                    if (r < p.rows) {
+                        uint32_t v[4];
+                        ld_shared_v4(sA2 + (uint32_t)((chunk >> 3) * kHalf) + sw128_offset(row, chunk & 7), v);
+                        st_global_v4(p.Y + (int64_t)p.row_list[p.first + r] * p.ldy + chunk * 8, v);
+                    }
+                }
+                worker_sync();                               // the staging buffer is rewritten by the next tile
+            }
+            if (stop) {
+                // A wait ran out somewhere in this CTA.  Every worker went through the whole tile (nothing above
+                // branches on `failed`), so all of them are here.  Before the CTA may leave, what it started must
+                // have ended: the weight copy and the copies of this tile's and of the prefetched tile's rows (these
+                // waits keep the default limit: a copy that was started does land); the issuing thread waits for the
+                // products.
+                if (tid == 0) {
+                    if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
+                    mbar_wait(bar_w, 0);
+                    if (!LISTED) {
+                        mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u);
+                        if (tile + (int)gridDim.x < p.n_tiles) mbar_wait(bar_x[s ^ 1], (uint32_t)((it + 1) >> 1) & 1u);
+                    }
+                }
+                break;
             }
         }
-        fence_proxy_async_smem();
-        const bool stop = __syncthreads_or(failed ? 1 : 0) != 0;   // also: the X stage may be refilled from here on
-        if (tid == 0 && !stop) {
-            tma_store_2d(&map_y, 0, tile * kTileM, sA2);
-            tma_store_2d(&map_y, 64, tile * kTileM, sA2 + kHalf);
-            bulk_commit();
-        }
-        if (stop) {
-            // A wait ran out somewhere in this CTA.  Every thread went through the whole tile (nothing above
-            // branches on `failed`), so all of them are here.  Before the CTA may leave, what it started must have
-            // ended: the weight copy, the copies of this tile's and of the prefetched tile's rows, and the MMAs
-            // (these waits keep the default limit: a copy or an MMA that was started does finish).
-            if (tid == 0) {
-                if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
-                mbar_wait(bar_w, 0);
-                mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u);
-                if (tile + (int)gridDim.x < p.n_tiles) mbar_wait(bar_x[s ^ 1], (uint32_t)((it + 1) >> 1) & 1u);
-                mma_commit(smem_u32(&misc->bar_drain));
-                mbar_wait(smem_u32(&misc->bar_drain), 0);
-            }
-            break;
+        if (tid == 0) {
+            *reinterpret_cast<volatile int32_t*>(&misc->stop) = 1;   // releases the issuing thread from its wait
+            bulk_wait_all();
         }
     }
-    if (tid == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
@@ -326,7 +417,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
 // ---- row-wise layer normalisation: half a warp per row, eight columns (16 bytes) per lane -----------
 __global__ void __launch_bounds__(256)
 layernorm_kernel(const __nv_bfloat16* X, int64_t ldx, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, float eps, __nv_bfloat16* Y, int64_t ldy, int n) {   // Y may be X
+                 const float* __restrict__ beta, float eps, __nv_bfloat16* Y, int64_t ldy, int n,
+                 const int32_t* __restrict__ row_list, int list_first) {   // Y may be X; rows from a list if row_list != NULL
     const int sub = threadIdx.x & 15;
     const int groups = (int)((gridDim.x * blockDim.x) >> 4);
     const float4 ga = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * sub), gb = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * sub + 1);
@@ -341,7 +433,7 @@ layernorm_kernel(const __nv_bfloat16* X, int64_t ldx, const float* __restrict__ 
         for (int i = 0; i < 4; ++i) {
             const int row = base_row + hw + i * groups;
             w[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (row < n) w[i] = *reinterpret_cast<const uint4*>(X + (size_t)row * ldx + sub * 8);
+            if (row < n) w[i] = *reinterpret_cast<const uint4*>(X + (size_t)(row_list ? row_list[list_first + row] : row) * ldx + sub * 8);
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -366,7 +458,7 @@ layernorm_kernel(const __nv_bfloat16* X, int64_t ldx, const float* __restrict__ 
             out.y = pack_bf16(x[2] * rstd * ga.z + ba.z, x[3] * rstd * ga.w + ba.w);
             out.z = pack_bf16(x[4] * rstd * gb.x + bb.x, x[5] * rstd * gb.y + bb.y);
             out.w = pack_bf16(x[6] * rstd * gb.z + bb.z, x[7] * rstd * gb.w + bb.w);
-            if (row < n) *reinterpret_cast<uint4*>(Y + (size_t)row * ldy + sub * 8) = out;
+            if (row < n) *reinterpret_cast<uint4*>(Y + (size_t)(row_list ? row_list[list_first + row] : row) * ldy + sub * 8) = out;
         }
     }
 }
@@ -437,6 +529,77 @@ dg4_status check_common(const dg4_graph* g, const dg4_desc* desc, float eps) {
 
 }  // namespace
 
+namespace {
+
+struct RowSet {                       // which rows a call works on: 0 .. rows-1, or row_list[first .. first+rows-1]
+    const int32_t* row_list = nullptr;
+    int32_t first = 0;
+    int32_t rows = 0;
+};
+
+dg4_status layernorm_launch(const void* X, int64_t ldx, const float* gamma, const float* beta, float eps, void* Y,
+                            int64_t ldy, const RowSet& rs, cudaStream_t st) {
+    if (rs.rows <= 0) return DG4_OK;
+    const int blocks = (int)std::min<int64_t>(((int64_t)rs.rows + 15) / 16, 148 * 8);
+    layernorm_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)X, ldx, gamma, beta, eps, (__nv_bfloat16*)Y, ldy,
+                                             rs.rows, rs.row_list, rs.first);
+    DG4_CUDA_TRY(cudaGetLastError());
+    dg4i_count_launch();
+    return DG4_OK;
+}
+
+dg4_status ffn_launch(const dg4_graph* g, const void* X, int64_t ldx, const void* W1, const float* b1, const void* W2,
+                      const float* b2, const float* gamma, const float* beta, float eps, void* Y, int64_t ldy,
+                      const RowSet& rs, cudaStream_t st) {
+    if (rs.rows <= 0) return DG4_OK;
+    int dev = 0;
+    DG4_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_attr_set[dev]) {
+            DG4_CUDA_TRY(cudaFuncSetAttribute(ffn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            DG4_CUDA_TRY(cudaFuncSetAttribute(ffn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            DG4_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+            g_attr_set[dev] = true;
+        }
+    }
+    CUtensorMap map_x, map_w2, map_y;
+    CHECK(make_map(&map_w2, W2, 128, 512, 512));
+    map_x = map_y = map_w2;                      // placeholders when the rows come from a list
+    if (!rs.row_list) {
+        CHECK(make_map(&map_x, X, rs.rows, 128, ldx));
+        CHECK(make_map(&map_y, Y, rs.rows, 128, ldy));
+    }
+    FfnParams p;
+    p.W1 = (const __nv_bfloat16*)W1; p.b1 = b1; p.b2 = b2; p.gamma = gamma; p.beta = beta; p.eps = eps;
+    p.n_tiles = (rs.rows + kTileM - 1) / kTileM;
+    p.status = g->dev_status;
+    p.poll_limit = dg4i_poll_limit();
+    p.row_list = rs.row_list; p.first = rs.first; p.rows = rs.rows;
+    p.X = (const __nv_bfloat16*)X; p.ldx = ldx; p.Y = (__nv_bfloat16*)Y; p.ldy = ldy;
+    const int grid = std::min(p.n_tiles, g_sm_count[dev]);
+    if (rs.row_list) ffn_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(map_x, map_w2, map_y, p);
+    else ffn_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(map_x, map_w2, map_y, p);
+    DG4_CUDA_TRY(cudaGetLastError());
+    dg4i_count_launch();
+    return DG4_OK;
+}
+
+dg4_status check_ffn_args(const void* W1, const float* b1, const void* W2, const float* b2, const float* gamma,
+                          const float* beta, int32_t d_ff) {
+    if (d_ff != 512) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d_ff = %d: only d_ff = 4 d = 512 is supported", d_ff);
+    if (!W1 || !W2) DG4_FAIL(DG4_ERR_INVALID_ARG, "null weight matrix");
+    if (!aligned16(W1) || !aligned16(W2)) DG4_FAIL(DG4_ERR_INVALID_ARG, "weight matrices must be 16-byte aligned");
+    CHECK(check_vec("b1", b1));
+    CHECK(check_vec("b2", b2));
+    CHECK(check_vec("gamma", gamma));
+    CHECK(check_vec("beta", beta));
+    return DG4_OK;
+}
+
+}  // namespace
+
 extern "C" dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,
                                          const float* gamma, const float* beta, float eps, void* Y, int64_t ldy,
                                          void* stream) {
@@ -445,53 +608,78 @@ extern "C" dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc
     CHECK(check_rows("Y", Y, ldy));
     CHECK(check_vec("gamma", gamma));
     CHECK(check_vec("beta", beta));
-    if (g->n == 0) return DG4_OK;
-    const int blocks = (int)std::min<int64_t>(((int64_t)g->n + 15) / 16, 148 * 8);
-    layernorm_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)X, ldx, gamma, beta, eps,
-                                                                (__nv_bfloat16*)Y, ldy, g->n);
-    DG4_CUDA_TRY(cudaGetLastError());
-    dg4i_count_launch();
-    return DG4_OK;
+    RowSet all;
+    all.rows = g->n;
+    return layernorm_launch(X, ldx, gamma, beta, eps, Y, ldy, all, (cudaStream_t)stream);
 }
 
 extern "C" dg4_status dg4_ffn_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx, const void* W1,
                                    const float* b1, const void* W2, const float* b2, const float* gamma,
                                    const float* beta, float eps, int32_t d_ff, void* Y, int64_t ldy, void* stream) {
     CHECK(check_common(g, desc, eps));
-    if (d_ff != 512) DG4_FAIL(DG4_ERR_UNSUPPORTED, "d_ff = %d: only d_ff = 4 d = 512 is supported", d_ff);
+    CHECK(check_ffn_args(W1, b1, W2, b2, gamma, beta, d_ff));
     CHECK(check_rows("X", X, ldx));
     CHECK(check_rows("Y", Y, ldy));
-    if (!W1 || !W2) DG4_FAIL(DG4_ERR_INVALID_ARG, "null weight matrix");
-    if (!aligned16(W1) || !aligned16(W2)) DG4_FAIL(DG4_ERR_INVALID_ARG, "weight matrices must be 16-byte aligned");
-    CHECK(check_vec("b1", b1));
-    CHECK(check_vec("b2", b2));
-    CHECK(check_vec("gamma", gamma));
-    CHECK(check_vec("beta", beta));
-    if (g->n == 0) return DG4_OK;
-    int dev = 0;
-    DG4_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) DG4_FAIL(DG4_ERR_UNSUPPORTED, "device ordinal %d is out of range", dev);
-    {
-        std::lock_guard<std::mutex> lock(g_mu);
-        if (!g_attr_set[dev]) {
-            DG4_CUDA_TRY(cudaFuncSetAttribute(ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-            DG4_CUDA_TRY(cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-            g_attr_set[dev] = true;
+    RowSet all;
+    all.rows = g->n;
+    return ffn_launch(g, X, ldx, W1, b1, W2, b2, gamma, beta, eps, Y, ldy, all, (cudaStream_t)stream);
+}
+
+/* The whole block in level-by-level order (the order of Sec. 1 / Sec. 3.4 applied to the block of Sec. 3.5): one group
+ * of launches per level -- attention for the level's nodes, output projection with residual, LayerNorm, feed-forward
+ * sub-layer with its LayerNorm (rows taken from the level's node list, updated in place), then the K | V rows of the
+ * level are refreshed from the new rows so that higher levels gather block outputs. */
+extern "C" dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                               const void* W_qkv, const void* W_o, const float* ln1_gamma,
+                                               const float* ln1_beta, const void* W1, const float* b1, const void* W2,
+                                               const float* b2, const float* ln2_gamma, const float* ln2_beta, float eps,
+                                               int32_t d_ff, void* workspace, size_t workspace_bytes, void* stream) {
+    CHECK(check_common(g, desc, eps));
+    CHECK(dg4i_check_desc(desc, true));
+    CHECK(check_rows("H", H, ldh));
+    if (!W_qkv || !W_o || !aligned16(W_qkv) || !aligned16(W_o)) DG4_FAIL(DG4_ERR_INVALID_ARG, "W_qkv / W_o null or misaligned");
+    CHECK(check_vec("ln1_gamma", ln1_gamma));
+    CHECK(check_vec("ln1_beta", ln1_beta));
+    CHECK(check_ffn_args(W1, b1, W2, b2, ln2_gamma, ln2_beta, d_ff));
+    if (!workspace) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
+    if ((((uintptr_t)workspace) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+    if (workspace_bytes < dg4_layer_workspace_bytes(g, desc))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", workspace_bytes,
+                 dg4_layer_workspace_bytes(g, desc));
+    cudaStream_t st = (cudaStream_t)stream;
+    __nv_bfloat16* Hb = (__nv_bfloat16*)H;
+    __nv_bfloat16* Q = (__nv_bfloat16*)workspace;
+    __nv_bfloat16* KV = Q + (size_t)g->n * 128;
+    __nv_bfloat16* O = Q + (size_t)g->n * 384;
+    // Q | K | V of every node from the block's input: a node's own query, key and value never change
+    CHECK(dg4_qkv_project(g, desc, H, ldh, W_qkv, Q, 128, KV, 256, KV + 128, 256, stream));
+    const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;
+    for (int l = 0; l < g->n_levels; ++l) {
+        RowSet lev;
+        lev.row_list = g->level_nodes; lev.first = g->h_level_ptr[l]; lev.rows = g->h_level_ptr[l + 1] - lev.first;
+        if (lev.rows <= 0) continue;
+        dg4i_attn_args a;
+        a.Q = Q; a.ldq = 128; a.K = KV; a.ldk = 256; a.V = KV + 128; a.ldv = 256; a.O = O; a.ldo = 128;
+        a.nbr_pad = g->nbr_pad; a.node_list = g->level_nodes; a.first = lev.first; a.count = lev.rows;
+        a.heads = desc->heads; a.max_nbr = g->max_class; a.dtype = desc->dtype; a.scale = desc->scale;
+        dg4i_attn_more more;
+        more.nbr_ptr = g->nbr_ptr; more.nbr_idx = g->nbr_idx;
+        CHECK(dg4i_attn_launch(a, &more, st));
+        dg4i_proj_args o;
+        o.A = O; o.lda = 128; o.W = (const __nv_bfloat16*)W_o; o.n_out = 128;
+        o.out[0] = Hb; o.ldo[0] = ldh; o.out[1] = o.out[2] = nullptr; o.ldo[1] = o.ldo[2] = 0;
+        o.R = Hb; o.ldr = ldh; o.row_list = g->level_nodes; o.first = lev.first; o.rows = lev.rows; o.status = g->dev_status;
+        CHECK(dg4i_proj_launch(o, st));
+        CHECK(layernorm_launch(H, ldh, ln1_gamma, ln1_beta, eps, H, ldh, lev, st));
+        CHECK(ffn_launch(g, H, ldh, W1, b1, W2, b2, ln2_gamma, ln2_beta, eps, H, ldh, lev, st));
+        if (l + 1 < g->n_levels) {
+            dg4i_proj_args k;
+            k.A = Hb; k.lda = ldh; k.W = W_kv; k.n_out = 256;
+            k.out[0] = KV; k.ldo[0] = 256; k.out[1] = KV + 128; k.ldo[1] = 256; k.out[2] = nullptr; k.ldo[2] = 0;
+            k.R = nullptr; k.ldr = 0; k.row_list = g->level_nodes; k.first = lev.first; k.rows = lev.rows; k.status = g->dev_status;
+            CHECK(dg4i_proj_launch(k, st));
         }
     }
-    CUtensorMap map_x, map_w2, map_y;
-    CHECK(make_map(&map_x, X, g->n, 128, ldx));
-    CHECK(make_map(&map_w2, W2, 128, 512, 512));
-    CHECK(make_map(&map_y, Y, g->n, 128, ldy));
-    FfnParams p;
-    p.W1 = (const __nv_bfloat16*)W1; p.b1 = b1; p.b2 = b2; p.gamma = gamma; p.beta = beta; p.eps = eps;
-    p.n_tiles = (g->n + kTileM - 1) / kTileM;
-    p.status = g->dev_status;
-    p.poll_limit = dg4i_poll_limit();
-    const int grid = std::min(p.n_tiles, g_sm_count[dev]);
-    ffn_kernel<<<grid, kThreads, kSmemBytes, (cudaStream_t)stream>>>(map_x, map_w2, map_y, p);
-    DG4_CUDA_TRY(cudaGetLastError());
-    dg4i_count_launch();
     return DG4_OK;
 }
 

@@ -42,7 +42,7 @@ EXPORTS = [
     "dg4_selftest_bounded_wait", "dg4_sparse_attn_additive_fwd", "dg4_graph_partition",
     "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel", "dg4_graph_destroy_async", "dg4_memory_trim",
     "dg4_debug_set_poll_limit", "dg4_debug_override_current_device",
-    "dg4_cone_update_workspace_bytes", "dg4_cone_update_fwd",
+    "dg4_cone_update_workspace_bytes", "dg4_cone_update_fwd", "dg4_block_fwd_levelised",
 ]
 
 
@@ -144,6 +144,9 @@ def load():
     lib.dg4_block_fwd_parallel.restype = ctypes.c_int
     lib.dg4_block_fwd_parallel.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
                                            vp, i64, vp, ctypes.c_size_t, vp]
+    lib.dg4_block_fwd_levelised.restype = ctypes.c_int
+    lib.dg4_block_fwd_levelised.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
+                                            vp, ctypes.c_size_t, vp]
     lib.dg4_cone_update_workspace_bytes.restype = ctypes.c_size_t
     lib.dg4_cone_update_workspace_bytes.argtypes = [vp, dp, ctypes.c_int32]
     lib.dg4_cone_update_fwd.restype = ctypes.c_int
@@ -391,6 +394,16 @@ def dg4_block_fwd_parallel(g: Graph, dsc: dg4_desc, H_in, W_qkv, W_o, ln1_gamma,
                                          _ptr(ln2_gamma), _ptr(ln2_beta), ctypes.c_float(eps), int(W1.shape[0]),
                                          _ptr(H_out), _ld(H_out), _ptr(workspace),
                                          workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def dg4_block_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv, W_o, ln1_gamma, ln1_beta, W1, b1, W2, b2, ln2_gamma,
+                            ln2_beta, eps, workspace, stream=None):
+    """One whole block in level-by-level order, in place on H (one group of launches per level)."""
+    _check(load().dg4_block_fwd_levelised(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), _ptr(W_qkv), _ptr(W_o),
+                                          _ptr(ln1_gamma), _ptr(ln1_beta), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
+                                          _ptr(ln2_gamma), _ptr(ln2_beta), ctypes.c_float(eps), int(W1.shape[0]),
+                                          _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                          _stream(stream)))
 
 
 def dg4_graph_partition(g: Graph, delta: int):

@@ -60,6 +60,12 @@ MUTANTS = [
      "std::memcpy(&cur[(int64_t)i * d], X + (int64_t)S[i] * d, sizeof(double) * d);", "cone_update"),
     ("update_one_layer_only", "            for (int j = 0; j < n_layers; ++j) {\n                orc_layer_parallel(m,", "            for (int j = 0; j < 1; ++j) {\n                orc_layer_parallel(m,", "cone_update"),
     ("update_batches_span_level_groups", "const int b1 = std::min(b0 + batch, (int)group_ptr[l + 1]);", "const int b1 = std::min(b0 + batch, (int)group_ptr[n_levels]);", "cone_update"),
+    ("block_levelised_in_reverse_order", "for (int lev = 0; lev < n_levels; ++lev) {", "for (int lev = n_levels - 1; lev >= 0; --lev) {", "block_levelised"),
+    ("block_levelised_skips_first_norm", "            orc_layernorm(1, d, pre.data(), g1, be1, eps, h1.data());", "            h1 = pre;", "block_levelised"),
+    ("block_levelised_keys_from_attention_sublayer_output", "orc_ffn(1, d, d_ff, h1.data(), W1, b1, W2, b2, g2, be2, eps, rounding, fresh.data() + (int64_t)(i - lo) * d);",
+     "std::memcpy(fresh.data() + (int64_t)(i - lo) * d, h1.data(), sizeof(double) * d);", "block_levelised"),
+    ("block_levelised_without_attention_residual", "project_row(d, d, o.data(), W_o, H + (int64_t)v * d, pre.data());",
+     "project_row(d, d, o.data(), W_o, nullptr, pre.data());", "block_levelised"),
     ("ffn_second_matrix_transposed", "acc += u[h] * W2[(int64_t)o * d_ff + h];", "acc += u[h] * W2[(int64_t)h * d + o];", "ffn"),
 ]
 

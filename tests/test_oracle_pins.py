@@ -603,3 +603,75 @@ def test_ffn_rounding_points():
     ref = orc.round_bf16(orc.layernorm(z, gam, bet, eps=1e-5))
     got = orc.ffn(x, W1, b1, W2, b2, gam, bet, eps=1e-5, rounding="bf16")
     assert np.allclose(got, ref, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- the whole block, level by level
+
+def _block_params(rng, d, d_ff):
+    return dict(Wqkv=0.3 * rng.standard_normal((3 * d, d)), Wo=0.3 * rng.standard_normal((d, d)),
+                g1=1 + 0.2 * rng.standard_normal(d), be1=0.2 * rng.standard_normal(d),
+                W1=0.3 * rng.standard_normal((d_ff, d)), b1=0.2 * rng.standard_normal(d_ff),
+                W2=0.3 * rng.standard_normal((d, d_ff)), b2=0.2 * rng.standard_normal(d),
+                g2=1 + 0.2 * rng.standard_normal(d), be2=0.2 * rng.standard_normal(d))
+
+
+def _block_levelised(H, P, ptr, idx, lptr, lnodes, heads, rounding=None):
+    return orc.block_levelised(H, P["Wqkv"], P["Wo"], P["g1"], P["be1"], P["W1"], P["b1"], P["W2"], P["b2"], P["g2"],
+                               P["be2"], ptr, idx, lptr, lnodes, heads, 0.5, eps=1e-5, rounding=rounding)
+
+
+@pytest.mark.parametrize("rounding", [None, "bf16"])
+def test_block_levelised_equals_bucket_by_bucket_replay_of_library_steps(rounding):
+    """Replay with the routines pinned above: per level, the attention sub-layer of the parallel layer applied to the
+    current rows, LayerNorm, the feed-forward sub-layer; only that level's rows are committed."""
+    rng = np.random.default_rng(41)
+    fanins = random_dag(rng, 6, 80, window=9)
+    n, d, d_ff, heads = len(fanins), 16, 32, 2
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    lptr, lnodes = orc.level_buckets(level)
+    P = _block_params(rng, d, d_ff)
+    if rounding:
+        P = {k: (orc.round_bf16(v) if k.startswith("W") else v) for k, v in P.items()}
+    X = orc.round_bf16(rng.standard_normal((n, d)))
+    rnd = (lambda a: orc.round_bf16(a)) if rounding else (lambda a: a)
+    H = X.copy()
+    for l in range(int(level.max()) + 1):
+        pre = orc.layer_parallel(H, P["Wqkv"], P["Wo"], ptr, idx, heads, 0.5, residual=True, rounding=rounding)
+        h1 = rnd(orc.layernorm(pre, P["g1"], P["be1"], 1e-5))
+        out = orc.ffn(h1, P["W1"], P["b1"], P["W2"], P["b2"], P["g2"], P["be2"], eps=1e-5, rounding=rounding)
+        H[level == l] = out[level == l]
+    got = _block_levelised(X, P, ptr, idx, lptr, lnodes, heads, rounding)
+    assert np.abs(got - H).max() < 1e-12
+    # the level-0 rows are the parallel block's rows; deeper rows are not
+    pre = orc.layer_parallel(X, P["Wqkv"], P["Wo"], ptr, idx, heads, 0.5, residual=True, rounding=rounding)
+    par = orc.ffn(rnd(orc.layernorm(pre, P["g1"], P["be1"], 1e-5)), P["W1"], P["b1"], P["W2"], P["b2"], P["g2"], P["be2"],
+                  eps=1e-5, rounding=rounding)
+    assert (got[level == 0] == par[level == 0]).all() and np.abs(got - par).max() > 1e-6
+
+
+def test_block_levelised_invariants():
+    rng = np.random.default_rng(42)
+    fanins = random_dag(rng, 6, 100, window=9)
+    n, d, d_ff, heads = len(fanins), 16, 32, 2
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    lptr, lnodes = orc.level_buckets(level)
+    P = _block_params(rng, d, d_ff)
+    X = rng.standard_normal((n, d))
+    base = _block_levelised(X, P, ptr, idx, lptr, lnodes, heads)
+    shuffled = lnodes.copy()                               # the order inside a level does not matter
+    for l in range(len(lptr) - 1):
+        shuffled[lptr[l]:lptr[l + 1]] = rng.permutation(lnodes[lptr[l]:lptr[l + 1]])
+    assert (_block_levelised(X, P, ptr, idx, lptr, shuffled, heads) == base).all()
+    m = 60                                                 # a prefix of the ids is closed under fan-in
+    rp2, ci2 = csr_from_fanins(fanins[:m])
+    ptr2, idx2 = orc.neighbourhood(rp2, ci2, 2)
+    lptr2, lnodes2 = orc.level_buckets(level[:m])
+    assert (_block_levelised(X[:m], P, ptr2, idx2, lptr2, lnodes2, heads) == base[:m]).all()
+    # every row went through the last LayerNorm: with gamma = 1 and beta = 0 it has zero mean and unit variance
+    P1 = dict(P, g2=np.ones(d), be2=np.zeros(d))
+    out = _block_levelised(X, P1, ptr, idx, lptr, lnodes, heads)
+    assert np.abs(out.mean(axis=1)).max() < 1e-12 and np.abs(out.var(axis=1) - 1).max() < 1e-3
