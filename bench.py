@@ -376,6 +376,17 @@ def run_ours(args, w):
                        "layernorm_ms": ln_ms, "layernorm_gbs": 512.0 * n / (ln_ms * 1e-3) / 1e9,
                        "block_parallel_ms": blk_ms})
         del w1, w2
+        # the paper's cone depth (k = 8) on the 1M-node circuit: the warp-per-node kernel for wider cones
+        w3 = synth.workload(3)
+        g3 = w3.graph()
+        gr3 = dg4.dg4_graph_create(g3.row_ptr, g3.col_idx, g3.level, 8, 0, local)
+        q3, k3, v3 = ((torch.randn(g3.n, 128, device="cuda") * sdev).to(torch.bfloat16) for sdev in (0.5, 0.5, 1.0))
+        o3 = torch.empty_like(q3)
+        wide_ms = timed3(lambda: dg4.dg4_sparse_attn_fwd(gr3, dsc, q3, k3, v3, o3))
+        extras.update({"wide8_nodes": g3.n, "wide8_entries_per_node": gr3.info.n_nbr / g3.n, "wide8_attn_ms": wide_ms,
+                       "wide8_gather_tbs": gr3.info.n_nbr * 512.0 / (wide_ms * 1e-3) / 1e12})
+        dg4.dg4_graph_destroy(gr3)
+        del q3, k3, v3, o3
 
     # ---- end to end through the C ABI from host buffers -----------------------------------------
     # Every step uploads its circuit (pageable CSR arrays, through dg4_graph_create) and its features (pinned),
