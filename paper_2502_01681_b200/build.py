@@ -34,6 +34,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-pthread", "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc"),
            "-o", LIB] + SOURCES
+    # compile-time switches of the kernels (e.g. DG4_BUILD_DEFINES="-DDG4_ATTN_KV_EVICT_LAST=1"), for measured variants
+    cmd[1:1] = os.environ.get("DG4_BUILD_DEFINES", "").split()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)

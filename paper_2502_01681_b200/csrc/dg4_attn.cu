@@ -218,23 +218,36 @@ __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_ker
                         vq[i] = ld_piece_nc((const char*)a.V + (size_t)u[i] * a.ldv * ES + col);
                     }
                 }
+                // scores of the batch first, then ONE rescale of the running sums to the batch's maximum (rescaling
+                // per neighbour costs a multiply per accumulator and an exponential each time)
+                float s[UN];
 #pragma unroll
                 for (int i = 0; i < UN; ++i) {
                     float dot = (u[i] >= 0) ? Elem<BF16>::dot(qp, kq[i]) : 0.f;
 #pragma unroll
                     for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(hmask, dot, o);
-                    if (u[i] >= 0) {                                           // uniform inside a half
-                        const float s = dot * c;
-                        const float m_new = fmaxf(m, s);
-                        const float keep = fast_exp2(m - m_new);               // 0 on the first neighbour (m = -inf)
-                        const float p = fast_exp2(s - m_new);
-                        float vf[EPP];
-                        Elem<BF16>::unpack(vq[i], vf);
-                        z = z * keep + p;
+                    s[i] = (u[i] >= 0) ? dot * c : -INFINITY;
+                }
+                float m_new = m;
 #pragma unroll
-                        for (int e = 0; e < EPP; ++e) acc[e] = fmaf(p, vf[e], acc[e] * keep);
-                        m = m_new;
+                for (int i = 0; i < UN; ++i) m_new = fmaxf(m_new, s[i]);
+                if (u[0] >= 0) {                                               // uniform inside a half; a batch's first slot is its lowest position
+                    const float keep = fast_exp2(m - m_new);                   // 0 for the first batch (m = -inf)
+                    z *= keep;
+#pragma unroll
+                    for (int e = 0; e < EPP; ++e) acc[e] *= keep;
+#pragma unroll
+                    for (int i = 0; i < UN; ++i) {
+                        if (u[i] >= 0) {
+                            const float p = fast_exp2(s[i] - m_new);
+                            float vf[EPP];
+                            Elem<BF16>::unpack(vq[i], vf);
+                            z += p;
+#pragma unroll
+                            for (int e = 0; e < EPP; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
+                        }
                     }
+                    m = m_new;
                 }
             }
         }
