@@ -244,19 +244,23 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0, p.poll_limit);
 
         int it = 0;
+        bool g1_released = false;        // the first product of the tile about to start was released during the tile before
         for (int tile = first_tile; tile < p.n_tiles; tile += (int)gridDim.x, ++it) {
             const int s = it & 1;
             const uint32_t sXs = sX + s * kTileBytes;
+            const bool has_next = tile + (int)gridDim.x < p.n_tiles;
             if (!LISTED) {
-                if (tid == 0) {
-                    const int next = tile + (int)gridDim.x;      // prefetch the next tile's rows into the other stage
-                    if (next < p.n_tiles) {
-                        mbar_expect_tx(bar_x[s ^ 1], kTileBytes);
-                        for (int h = 0; h < 2; ++h)
-                            tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
-                    }
+                if (tid == 0 && has_next) {                      // prefetch the next tile's rows into the other stage
+                    const int next = tile + (int)gridDim.x;
+                    mbar_expect_tx(bar_x[s ^ 1], kTileBytes);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d(sX + (s ^ 1) * kTileBytes + h * kHalf, &map_x, h * 64, next * kTileM, bar_x[s ^ 1]);
                 }
-                failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u, p.poll_limit);
+                if (!g1_released) {
+                    failed |= !mbar_wait(bar_x[s], (uint32_t)(it >> 1) & 1u, p.poll_limit);
+                    worker_sync();
+                    if (tid == 0) release_product();         // G1(0)
+                }
             } else {
                 // listed rows: the workers gather the tile's rows into the same swizzled layout, 16 bytes at a time
                 for (int i = tid; i < kTileM * 16; i += kWorkers) {
@@ -267,11 +271,9 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     st_shared_v4(sXs + (uint32_t)((chunk >> 3) * kHalf) + sw128_offset(row, chunk & 7), v);
                 }
                 fence_proxy_async_smem();
+                worker_sync();
+                if (tid == 0) release_product();             // G1(0)
             }
-            // the X tile has landed for every worker before the first product is released (the barrier also
-            // separates the previous tile's reads of its buffers from this tile's writes)
-            worker_sync();
-            if (tid == 0) release_product();             // G1(0)
 
             // Per block q of hidden units: the accumulator is read into registers, the next block's first product is
             // released at once (it runs while the values are scattered into the operand buffer), then the second
@@ -303,6 +305,16 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 worker_sync();
                 if (tid == 0) release_product();             // G2(q)
             }
+            // The next tile's rows were requested a tile ago and have landed: its first product may run under this
+            // tile's final epilogue (its accumulator is free: every worker has read block 3's before the last barrier).
+            g1_released = false;
+            if (!LISTED && has_next) {
+                if (tid == 0) {
+                    failed |= !mbar_wait(bar_x[s ^ 1], (uint32_t)((it + 1) >> 1) & 1u, p.poll_limit);
+                    release_product();                       // G1(0) of the next tile
+                }
+                g1_released = true;
+            }
             failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);   // D2 is complete; the activation buffer is free
             ph_g2 ^= 1u;
             tc_fence_after();
@@ -310,13 +322,13 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
             // ---- final epilogue: thread = row `ln`, columns cg*64 .. cg*64+63
             {
                 float y[64];
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t d[32];
-                    tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64 + half * 32), d);
+                {
+                    uint32_t d[64];
+                    tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64), d);
+                    tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD2 + cg * 64 + 32), d + 32);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) y[half * 32 + j] = __uint_as_float(d[j]);
+                    for (int j = 0; j < 64; ++j) y[j] = __uint_as_float(d[j]);
                 }
                 tc_fence_before();
                 const float4* b2v = reinterpret_cast<const float4*>(p.b2 + cg * 64);
@@ -335,13 +347,19 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     y[c * 8 + 7] += __uint_as_float(w[3] & 0xffff0000u) + bb.w;
                 }
                 // mean and sum of squared deviations of the half-row, merged with the other half-row's
-                float m = 0.0f;
+                float ms[4] = {0.0f, 0.0f, 0.0f, 0.0f};               // four partial sums: four independent chains
 #pragma unroll
-                for (int j = 0; j < 64; ++j) m += y[j];
-                m *= (1.0f / 64.0f);
-                float m2 = 0.0f;
+                for (int j = 0; j < 64; j += 4) { ms[0] += y[j]; ms[1] += y[j + 1]; ms[2] += y[j + 2]; ms[3] += y[j + 3]; }
+                const float m = ((ms[0] + ms[1]) + (ms[2] + ms[3])) * (1.0f / 64.0f);
+                float vs[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int j = 0; j < 64; ++j) m2 += (y[j] - m) * (y[j] - m);
+                for (int j = 0; j < 64; j += 4) {
+                    vs[0] = fmaf(y[j] - m, y[j] - m, vs[0]);
+                    vs[1] = fmaf(y[j + 1] - m, y[j + 1] - m, vs[1]);
+                    vs[2] = fmaf(y[j + 2] - m, y[j + 2] - m, vs[2]);
+                    vs[3] = fmaf(y[j + 3] - m, y[j + 3] - m, vs[3]);
+                }
+                const float m2 = (vs[0] + vs[1]) + (vs[2] + vs[3]);
                 st_shared_f2(sA2 + (uint32_t)((ln * 2 + cg) * 8), m, m2);
                 worker_sync();
                 float mo, m2o;
