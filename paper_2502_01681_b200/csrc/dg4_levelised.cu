@@ -76,7 +76,10 @@ constexpr int kOffX = kOffHp + kTileOp;                // input rows of the curr
 constexpr int kOffHres = kOffX + 2 * kTileOp;          // the same rows, plain [kTile][256 B], twice
 constexpr int kOffStage = kOffHres + 2 * kTile * 256;  // staging, plain [kTile][kStageRow]
 constexpr int kOffMisc = kOffStage + kTile * kStageRow;
-constexpr int kSmemBytes = kOffMisc + 256 + 1024;
+constexpr int kWHalf = 128 * 128;                      // K-half of a 128-row weight block: 128 rows x 128 bytes
+constexpr int kWBlock = 2 * kWHalf;                    // a 128 x 128 bf16 block in shared memory (32 KiB)
+constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o | W_k | W_v for the warp-level products
+constexpr int kSmemBytes = kOffWs + 3 * kWBlock + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 static_assert(kWCol0 + 4 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
 static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) == 0, "operand tiles are 1024-byte aligned");
@@ -85,16 +88,17 @@ static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) ==
 // of an SM's shared memory, which rules that out.
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
-enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdWo = 2, kCmdKv = 3, kCmdKvThenQkv = 4 };
+enum : int32_t { kCmdExit = 0, kCmdQkv = 1 };
 
 struct Misc {
-    uint64_t mma0, mma1, mma2, drain;
+    uint64_t mma0, drain;
     uint64_t cmd_bar;                      // the workers' next order for the issuing thread is in `cmd`
     int32_t cmd, cmd_buf;
     uint32_t tmem_base;
     int32_t go, go2;
     int32_t failed;                        // a wait for this CTA's own MMAs ran out: leave at the next level
-    int32_t pre_ok;                        // the layer below has finished the rows of this CTA's next tile
+    int32_t pre_ok;                        // the layer below has finished the rows of this CTA's next tile (checked mid-tile)
+    int32_t pre_early;                     // the same, already known at the top of the tile
     int32_t node[kTile];
 };
 
@@ -160,6 +164,34 @@ __device__ __forceinline__ void give_up(const LevParams& p) {
     if (p.status) atomicCAS(p.status, 0, (int)DG4_ERR_TIMEOUT);
 }
 
+// byte offset of the 16-byte piece `chunk` (0..15) of row `row` in a 128-row weight block (same swizzle)
+__device__ __forceinline__ uint32_t weight_piece(int row, int chunk) {
+    return (uint32_t)((chunk >> 3) * kWHalf) + sw128_offset(row, chunk & 7);
+}
+// warp-level tensor-core product (synchronous: the result is in registers when the instruction retires), used for
+// the two 16-node products that sit on the level-to-level chain
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t* r) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void mma_m16n8k16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void st_shared_b32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_shared_b32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
 // barrier among the eight worker warps only (the issuing warp never joins it)
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 
@@ -183,11 +215,12 @@ levelised_kernel(LevParams p) {
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
     const uint32_t sO = base + kOffO, sHp = base + kOffHp, sX = base + kOffX, sHres = base + kOffHres, sSt = base + kOffStage;
+    const uint32_t sW = base + kOffWs;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = tid >> 4, sub = tid & 15;          // node slot of the tile and lane within the node
     const int grp_base = lane - sub;
     const unsigned gmask = 0xffffu << grp_base;
-    const uint32_t bar0 = smem_u32(&misc->mma0), bar1 = smem_u32(&misc->mma1), bar2 = smem_u32(&misc->mma2);
+    const uint32_t bar0 = smem_u32(&misc->mma0);
 
     // this CTA's layer, its rank among the CTAs of that layer, and how many CTAs each layer has
     const int layer = (int)blockIdx.x % p.n_layers;
@@ -197,8 +230,6 @@ levelised_kernel(LevParams p) {
 
     if (tid == 0) {
         mbar_init(bar0, 1);
-        mbar_init(bar1, 1);
-        mbar_init(bar2, 1);
         mbar_init(smem_u32(&misc->drain), 1);
         mbar_init(smem_u32(&misc->cmd_bar), 1);
         misc->cmd = kCmdExit;
@@ -207,6 +238,7 @@ levelised_kernel(LevParams p) {
         misc->go2 = 1;
         misc->failed = 0;
         misc->pre_ok = 0;
+        misc->pre_early = 0;
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
@@ -235,6 +267,14 @@ levelised_kernel(LevParams p) {
             }
         }
         tmem_st_wait();
+        // W_o, W_k, W_v once more in shared memory (same 128-byte swizzle): the B operands of the warp-level products
+        for (int i = tid; i < 3 * 128 * 16; i += kWorkers) {
+            const int blk = i >> 11, row = (i >> 4) & 127, chunk = i & 15;
+            const __nv_bfloat16* wb = blk == 0 ? p.Wo[layer] : p.Wqkv[layer] + (size_t)blk * 128 * 128;
+            const uint4 v = *reinterpret_cast<const uint4*>(wb + (size_t)row * 128 + chunk * 8);
+            const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+            st_shared_v4(sW + (uint32_t)(blk * kWBlock) + weight_piece(row, chunk), r);
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -275,30 +315,7 @@ levelised_kernel(LevParams p) {
                 const int cmd = *reinterpret_cast<volatile int32_t*>(&misc->cmd);
                 const int b = *reinterpret_cast<volatile int32_t*>(&misc->cmd_buf);
                 if (cmd == kCmdExit) break;
-                if (cmd == kCmdQkv) {
-                    issue_qkv(b);
-                } else if (cmd == kCmdWo) {
-                    // output projection, transposed: D[feature, node] = W_o * O^T
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccO), tmem + (uint32_t)(kWCol0 + kBlkO * kWCols + ks * 8), dO + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
-                    }
-                    mma_commit(bar1);
-                } else {
-                    // from the new rows, transposed: this layer's K | V refresh; right behind it, if ordered, the next
-                    // tile's Q | K | V (it runs while this tile's rows are stored and the level completes)
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
-                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccK2), tmem + (uint32_t)(kWCol0 + kBlkK * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
-                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccV2), tmem + (uint32_t)(kWCol0 + kBlkV * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
-                    }
-                    mma_commit(bar2);
-                    if (cmd == kCmdKvThenQkv) issue_qkv(b);
-                }
+                issue_qkv(b);
             }
             // Tensor memory is freed below: every MMA issued must have completed.  Normally each was waited for by
             // the workers; after a wait that ran out, one may still be in flight.
@@ -314,7 +331,11 @@ levelised_kernel(LevParams p) {
             misc->cmd_buf = b;
             mbar_arrive(smem_u32(&misc->cmd_bar));
         };
-        uint32_t ph0 = 0, ph1 = 0, ph2 = 0;
+        uint32_t ph0 = 0;
+        // lane's place in the warp-level products: g = row of the 8 x 8 sub-matrix it holds, t = column pair
+        const int mg = lane >> 2, mt = lane & 3;
+        const int a_row = lane & 15, a_chunk = lane >> 4;                       // A fragments: the 16-node tile
+        const int b_row = (lane & 7) + ((lane >> 4) << 3), b_chunk = (lane >> 3) & 1;   // B fragments: 16 weight rows
         int last_nonempty = -1, last_participants = 0;
         bool alive = true;
         const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
@@ -382,6 +403,17 @@ levelised_kernel(LevParams p) {
                         v_nx = (more_here && r < n_l) ? p.level_nodes[first + r] : -1;
                     }
                     const bool valid = v >= 0;
+                    // which tile comes next for this CTA, and may its rows be requested already?  Asked twice: at the
+                    // top of the tile (then the rows travel under the gather) and, if the layer below was not ready
+                    // yet, once more in the middle of it
+                    const bool next_level_tile = !more_here && l + 1 < p.n_levels && bid < tiles_next;
+                    const bool want_pre = more_here || next_level_tile;
+                    auto next_rows_ready = [&]() -> int {
+                        if (!want_pre) return 0;
+                        if (next_level_tile && prev_arrive) return ld_acquire(prev_arrive + l + 1) >= prev_target(tiles_next) ? 1 : 0;
+                        return 1;
+                    };
+                    if (waited && tid == 32) misc->pre_early = next_rows_ready();   // visible after the barrier below
 
                     // ---- this tile's own Q | K | V: read from tensor memory if the product was issued during the
                     // tile before, else brought up from scratch below (after the counters)
@@ -421,6 +453,7 @@ levelised_kernel(LevParams p) {
                             if (prev_arrive && !pro_ready) go = wait_counter(prev_arrive + l, prev_target(tiles), p.abort_word, counter_limit);
                             if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                             misc->go2 = go ? 1 : 0;
+                            misc->pre_early = go ? next_rows_ready() : 0;
                         }
                         worker_sync();
                         waited = true;
@@ -456,15 +489,11 @@ levelised_kernel(LevParams p) {
                         for (int j = 1; j < MAXN; ++j)
                             if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
                     }
-                    // which tile comes next for this CTA, and may its rows be requested already?
-                    const bool next_level_tile = !more_here && l + 1 < p.n_levels && bid < tiles_next;
-                    const bool want_pre = more_here || next_level_tile;
                     const int v_pre = more_here ? v_nx : vC;
-                    if (tid == 32) {
-                        int ok = want_pre ? 1 : 0;
-                        if (next_level_tile && prev_arrive) ok = ld_acquire(prev_arrive + l + 1) >= prev_target(tiles_next) ? 1 : 0;
-                        misc->pre_ok = ok;
-                    }
+                    const bool pre_early = want_pre && misc->pre_early != 0;
+                    Piece xpre;
+                    if (pre_early) xpre = load_input(v_pre);                      // the next tile's input rows
+                    else if (tid == 32) misc->pre_ok = next_rows_ready();         // second look; read after the next barrier
                     {   // the node's own query, key and value: from the staging rows
                         const uint32_t row = sSt + (uint32_t)(slot * kStageRow + sub * 16);
                         ld_shared_v4(row, qp.w);
@@ -478,63 +507,77 @@ levelised_kernel(LevParams p) {
                         st_shared_v4(sO + operand_piece(slot, sub), o.w);
                         if (sub == 0) misc->node[slot] = v;
                     }
-                    fence_proxy_async_smem();
                     worker_sync();
 
-                    // ---- output projection, transposed: D[feature, node] = W_o * O^T
-                    if (tid == 0) post(kCmdWo, 0);
-                    // meanwhile: request the next tile's input rows (the layer below has finished them)
-                    const bool pre_ok = want_pre && misc->pre_ok != 0;
-                    Piece xpre;
-                    if (pre_ok) xpre = load_input(v_pre);
-                    if (!mbar_wait(bar1, ph1, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
-                    ph1 ^= 1u;
-                    tc_fence_after();
+                    // ---- output projection for the 16 nodes by warp-level MMAs (m16n8k16): warp w computes output
+                    // features 16w .. 16w+15 for all nodes; the result is in registers when the last one retires
+                    // (the asynchronous tcgen05 path costs an order / commit / barrier round trip per product, which
+                    // at N = 16 is longer than the product itself)
+                    const bool pre_ok = pre_early || (want_pre && misc->pre_ok != 0);
+                    if (pre_ok && !pre_early) xpre = load_input(v_pre);
                     {
-                        uint32_t d[8];
-                        tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * kAccO + cg * 8), d);
-                        tmem_ld_wait();
+                        float acc_o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-                        for (int nn = 0; nn < 8; ++nn) {
-                            const int node = cg * 8 + nn;
-                            const uint16_t rb = p.residual ? ld_shared_b16(sHres_cur + (uint32_t)(node * 256 + feat * 2)) : (uint16_t)0;
-                            const float val = __uint_as_float(d[nn]) + __uint_as_float((uint32_t)rb << 16);
-                            st_shared_b16(sHp + operand_offset(node, feat), bf16_bits(val));
+                        for (int ks = 0; ks < 8; ++ks) {
+                            uint32_t af[4], bf[4];
+                            ldmatrix_x4(sO + operand_piece(a_row, 2 * ks + a_chunk), af);
+                            ldmatrix_x4(sW + weight_piece(16 * warp + b_row, 2 * ks + b_chunk), bf);
+                            mma_m16n8k16(acc_o[0], af, bf[0], bf[1]);
+                            mma_m16n8k16(acc_o[1], af, bf[2], bf[3]);
+                        }
+                        // residual, rounding, new rows into shared memory in operand layout (two features per store)
+#pragma unroll
+                        for (int nt = 0; nt < 2; ++nt) {
+                            const int f = 16 * warp + 8 * nt + 2 * mt;
+#pragma unroll
+                            for (int hrow = 0; hrow < 2; ++hrow) {
+                                const int node = mg + 8 * hrow;
+                                const uint32_t rb = p.residual ? ld_shared_b32(sHres_cur + (uint32_t)(node * 256 + f * 2)) : 0u;
+                                const float lo = acc_o[nt][2 * hrow] + __uint_as_float(rb << 16);
+                                const float hi = acc_o[nt][2 * hrow + 1] + __uint_as_float(rb & 0xffff0000u);
+                                st_shared_b32(sHp + operand_offset(node, f), pack_bf16x2(lo, hi));
+                            }
                         }
                     }
-                    if (pre_ok) stage_input(buf ^ 1, xpre);
-                    tc_fence_before();
-                    fence_proxy_async_smem();
+                    if (pre_ok) {
+                        stage_input(buf ^ 1, xpre);
+                        fence_proxy_async_smem();
+                    }
                     worker_sync();
 
-                    // ---- from the new rows, transposed: this layer's K | V refresh; right behind it, the next tile's
-                    // Q | K | V (it runs while this tile's rows are stored and the level completes)
-                    if (tid == 0) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
-                    // meanwhile: the new rows go to H (16 lanes cover one 256-byte row)
+                    // ---- the next tile's Q | K | V product (tcgen05, issued by the ninth warp; off the chain), the new
+                    // rows to H, and from the new rows this layer's K | V refresh: warp w computes key features
+                    // 16w .. 16w+15 and value features 16w .. 16w+15
+                    if (tid == 0 && pre_ok) post(kCmdQkv, buf ^ 1);
                     const int node_v = misc->node[slot];
                     {
                         uint32_t w4[4];
                         ld_shared_v4(sHp + operand_piece(slot, sub), w4);
                         if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
                     }
-                    if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
-                    ph2 ^= 1u;
-                    tc_fence_after();
                     {
-                        uint32_t d[2][8];
+                        float acc_kv[4][4];
 #pragma unroll
-                        for (int blk = 0; blk < 2; ++blk)
-                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
-                        tmem_ld_wait();
+                        for (int i = 0; i < 4; ++i) acc_kv[i][0] = acc_kv[i][1] = acc_kv[i][2] = acc_kv[i][3] = 0.f;
 #pragma unroll
-                        for (int blk = 0; blk < 2; ++blk) {
-                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
+                        for (int ks = 0; ks < 8; ++ks) {
+                            uint32_t af[4], bk[4], bv[4];
+                            ldmatrix_x4(sHp + operand_piece(a_row, 2 * ks + a_chunk), af);
+                            ldmatrix_x4(sW + (uint32_t)kWBlock + weight_piece(16 * warp + b_row, 2 * ks + b_chunk), bk);
+                            ldmatrix_x4(sW + (uint32_t)(2 * kWBlock) + weight_piece(16 * warp + b_row, 2 * ks + b_chunk), bv);
+                            mma_m16n8k16(acc_kv[0], af, bk[0], bk[1]);
+                            mma_m16n8k16(acc_kv[1], af, bk[2], bk[3]);
+                            mma_m16n8k16(acc_kv[2], af, bv[0], bv[1]);
+                            mma_m16n8k16(acc_kv[3], af, bv[2], bv[3]);
+                        }
 #pragma unroll
-                            for (int nn = 0; nn < 8; ++nn)
-                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
+                        for (int i = 0; i < 4; ++i) {            // i: 0, 1 key features; 2, 3 value features
+                            const int f = 16 * warp + 8 * (i & 1) + 2 * mt;
+                            const uint32_t off = (uint32_t)((i >> 1) * 256 + f * 2);
+                            st_shared_b32(sSt + (uint32_t)(mg * kStageRow) + off, pack_bf16x2(acc_kv[i][0], acc_kv[i][1]));
+                            st_shared_b32(sSt + (uint32_t)((mg + 8) * kStageRow) + off, pack_bf16x2(acc_kv[i][2], acc_kv[i][3]));
                         }
                     }
-                    tc_fence_before();
                     worker_sync();
                     if (node_v >= 0) {
                         const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
