@@ -78,8 +78,8 @@ constexpr int kOffStage = kOffHres + 2 * kTile * 256;  // staging, plain [kTile]
 constexpr int kOffMisc = kOffStage + kTile * kStageRow;
 constexpr int kWHalf = 128 * 128;                      // K-half of a 128-row weight block: 128 rows x 128 bytes
 constexpr int kWBlock = 2 * kWHalf;                    // a 128 x 128 bf16 block in shared memory (32 KiB)
-constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o | W_k | W_v for the warp-level products
-constexpr int kSmemBytes = kOffWs + 3 * kWBlock + 1024;
+constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o for the warp-level output projection
+constexpr int kSmemBytes = kOffWs + kWBlock + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 static_assert(kWCol0 + 4 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
 static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) == 0, "operand tiles are 1024-byte aligned");
@@ -88,10 +88,10 @@ static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) ==
 // of an SM's shared memory, which rules that out.
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
-enum : int32_t { kCmdExit = 0, kCmdQkv = 1 };
+enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdKv = 2, kCmdKvThenQkv = 3 };
 
 struct Misc {
-    uint64_t mma0, drain;
+    uint64_t mma0, mma2, drain;
     uint64_t cmd_bar;                      // the workers' next order for the issuing thread is in `cmd`
     int32_t cmd, cmd_buf;
     uint32_t tmem_base;
@@ -220,7 +220,7 @@ levelised_kernel(LevParams p) {
     const int slot = tid >> 4, sub = tid & 15;          // node slot of the tile and lane within the node
     const int grp_base = lane - sub;
     const unsigned gmask = 0xffffu << grp_base;
-    const uint32_t bar0 = smem_u32(&misc->mma0);
+    const uint32_t bar0 = smem_u32(&misc->mma0), bar2 = smem_u32(&misc->mma2);
 
     // this CTA's layer, its rank among the CTAs of that layer, and how many CTAs each layer has
     const int layer = (int)blockIdx.x % p.n_layers;
@@ -230,6 +230,7 @@ levelised_kernel(LevParams p) {
 
     if (tid == 0) {
         mbar_init(bar0, 1);
+        mbar_init(bar2, 1);
         mbar_init(smem_u32(&misc->drain), 1);
         mbar_init(smem_u32(&misc->cmd_bar), 1);
         misc->cmd = kCmdExit;
@@ -267,13 +268,12 @@ levelised_kernel(LevParams p) {
             }
         }
         tmem_st_wait();
-        // W_o, W_k, W_v once more in shared memory (same 128-byte swizzle): the B operands of the warp-level products
-        for (int i = tid; i < 3 * 128 * 16; i += kWorkers) {
-            const int blk = i >> 11, row = (i >> 4) & 127, chunk = i & 15;
-            const __nv_bfloat16* wb = blk == 0 ? p.Wo[layer] : p.Wqkv[layer] + (size_t)blk * 128 * 128;
-            const uint4 v = *reinterpret_cast<const uint4*>(wb + (size_t)row * 128 + chunk * 8);
+        // W_o once more in shared memory (same 128-byte swizzle): the B operand of the warp-level output projection
+        for (int i = tid; i < 128 * 16; i += kWorkers) {
+            const int row = i >> 4, chunk = i & 15;
+            const uint4 v = *reinterpret_cast<const uint4*>(p.Wo[layer] + (size_t)row * 128 + chunk * 8);
             const uint32_t r[4] = {v.x, v.y, v.z, v.w};
-            st_shared_v4(sW + (uint32_t)(blk * kWBlock) + weight_piece(row, chunk), r);
+            st_shared_v4(sW + weight_piece(row, chunk), r);
         }
     }
     tc_fence_before();
@@ -315,7 +315,21 @@ levelised_kernel(LevParams p) {
                 const int cmd = *reinterpret_cast<volatile int32_t*>(&misc->cmd);
                 const int b = *reinterpret_cast<volatile int32_t*>(&misc->cmd_buf);
                 if (cmd == kCmdExit) break;
-                issue_qkv(b);
+                if (cmd == kCmdQkv) {
+                    issue_qkv(b);
+                } else {
+                    // from the new rows, transposed: this layer's K | V refresh; right behind it, if ordered, the next
+                    // tile's Q | K | V (it runs while this tile's rows are stored and the level completes)
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
+                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccK2), tmem + (uint32_t)(kWCol0 + kBlkK * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                        mma_bf16_ta(tmem + (uint32_t)(kTile * kAccV2), tmem + (uint32_t)(kWCol0 + kBlkV * kWCols + ks * 8), dHp + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                    }
+                    mma_commit(bar2);
+                    if (cmd == kCmdKvThenQkv) issue_qkv(b);
+                }
             }
             // Tensor memory is freed below: every MMA issued must have completed.  Normally each was waited for by
             // the workers; after a wait that ran out, one may still be in flight.
@@ -331,7 +345,7 @@ levelised_kernel(LevParams p) {
             misc->cmd_buf = b;
             mbar_arrive(smem_u32(&misc->cmd_bar));
         };
-        uint32_t ph0 = 0;
+        uint32_t ph0 = 0, ph2 = 0;
         // lane's place in the warp-level products: g = row of the 8 x 8 sub-matrix it holds, t = column pair
         const int mg = lane >> 2, mt = lane & 3;
         const int a_row = lane & 15, a_chunk = lane >> 4;                       // A fragments: the 16-node tile
@@ -539,45 +553,40 @@ levelised_kernel(LevParams p) {
                             }
                         }
                     }
-                    if (pre_ok) {
-                        stage_input(buf ^ 1, xpre);
-                        fence_proxy_async_smem();
-                    }
+                    if (pre_ok) stage_input(buf ^ 1, xpre);
+                    fence_proxy_async_smem();
                     worker_sync();
 
-                    // ---- the next tile's Q | K | V product (tcgen05, issued by the ninth warp; off the chain), the new
-                    // rows to H, and from the new rows this layer's K | V refresh: warp w computes key features
-                    // 16w .. 16w+15 and value features 16w .. 16w+15
-                    if (tid == 0 && pre_ok) post(kCmdQkv, buf ^ 1);
+                    // ---- from the new rows, transposed on the tcgen05 path (issued by the ninth warp): this layer's
+                    // K | V refresh; right behind it the next tile's Q | K | V, which runs while this tile's rows are
+                    // stored and the level completes.  (Measured: for the 8-instruction W_o product the warp-level
+                    // path wins, its fixed cost being nil; for these 16 instructions the asynchronous path does:
+                    // a warp-level m16n8k16 occupies its sub-partition for about 32 clocks.)
+                    if (tid == 0) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
                     const int node_v = misc->node[slot];
                     {
                         uint32_t w4[4];
                         ld_shared_v4(sHp + operand_piece(slot, sub), w4);
                         if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
                     }
+                    if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph2 ^= 1u;
+                    tc_fence_after();
                     {
-                        float acc_kv[4][4];
+                        uint32_t d[2][8];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) acc_kv[i][0] = acc_kv[i][1] = acc_kv[i][2] = acc_kv[i][3] = 0.f;
+                        for (int blk = 0; blk < 2; ++blk)
+                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
+                        tmem_ld_wait();
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {
-                            uint32_t af[4], bk[4], bv[4];
-                            ldmatrix_x4(sHp + operand_piece(a_row, 2 * ks + a_chunk), af);
-                            ldmatrix_x4(sW + (uint32_t)kWBlock + weight_piece(16 * warp + b_row, 2 * ks + b_chunk), bk);
-                            ldmatrix_x4(sW + (uint32_t)(2 * kWBlock) + weight_piece(16 * warp + b_row, 2 * ks + b_chunk), bv);
-                            mma_m16n8k16(acc_kv[0], af, bk[0], bk[1]);
-                            mma_m16n8k16(acc_kv[1], af, bk[2], bk[3]);
-                            mma_m16n8k16(acc_kv[2], af, bv[0], bv[1]);
-                            mma_m16n8k16(acc_kv[3], af, bv[2], bv[3]);
-                        }
+                        for (int blk = 0; blk < 2; ++blk) {
+                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {            // i: 0, 1 key features; 2, 3 value features
-                            const int f = 16 * warp + 8 * (i & 1) + 2 * mt;
-                            const uint32_t off = (uint32_t)((i >> 1) * 256 + f * 2);
-                            st_shared_b32(sSt + (uint32_t)(mg * kStageRow) + off, pack_bf16x2(acc_kv[i][0], acc_kv[i][1]));
-                            st_shared_b32(sSt + (uint32_t)((mg + 8) * kStageRow) + off, pack_bf16x2(acc_kv[i][2], acc_kv[i][3]));
+                            for (int nn = 0; nn < 8; ++nn)
+                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
                         }
                     }
+                    tc_fence_before();
                     worker_sync();
                     if (node_v >= 0) {
                         const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
