@@ -170,6 +170,10 @@ __device__ __forceinline__ uint32_t weight_piece(int row, int chunk) {
 }
 // warp-level tensor-core product (synchronous: the result is in registers when the instruction retires), used for
 // the two 16-node products that sit on the level-to-level chain
+__device__ __forceinline__ void prefetch_l2(const void* ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
+
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t* r) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
@@ -395,12 +399,18 @@ levelised_kernel(LevParams p) {
         for (int l = 0; l < p.n_levels && alive; ++l) {
             const int first = lp0;
             const int n_l = lp1 - lp0;
-            // issue the next load of every pipelined chain; the results are first used one level later
-            const int lp4 = lp_at(l + 4);
-            const int vB = stage_node(lp2, lp3);
-            const int padC = pad_of(vC);
+            // the next load of every pipelined chain (results first used one level later) is issued together with
+            // the tile's gather loads, whose latency the tile waits out anyway: issued here at the top, the first
+            // wait on anything else would also wait for them
+            int lp4 = 0, vB = -1, padC = 0;
+            auto issue_chains = [&]() {
+                lp4 = lp_at(l + 4);
+                vB = stage_node(lp2, lp3);
+                padC = pad_of(vC);
+            };
             const int tiles = (n_l + kTile - 1) / kTile;
             const int tiles_next = (lp2 - lp1 + kTile - 1) / kTile;      // tiles of level l + 1
+            if (!(n_l > 0 && bid < tiles)) issue_chains();
             if (n_l > 0 && bid < tiles) {
                 bool waited = false;
                 int v_nx = -1, pad_nx = 0;           // index chain of this CTA's next tile in a wide level
@@ -503,6 +513,7 @@ levelised_kernel(LevParams p) {
                         for (int j = 1; j < MAXN; ++j)
                             if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
                     }
+                    if (tile == bid) issue_chains();
                     const int v_pre = more_here ? v_nx : vC;
                     const bool pre_early = want_pre && misc->pre_early != 0;
                     Piece xpre;
@@ -568,6 +579,26 @@ levelised_kernel(LevParams p) {
                         uint32_t w4[4];
                         ld_shared_v4(sHp + operand_piece(slot, sub), w4);
                         if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
+                    }
+                    if (!more_here) {
+                        // While the product runs: ask L2 for the lines the coming levels' first loads will want (a
+                        // prefetch has no destination register, so nothing ever waits for it).  Without this the
+                        // index-chain loads and the neighbours' K | V rows of a large circuit come from DRAM, and
+                        // that latency is on the level-to-level chain.
+                        const int r3 = bid * kTile + slot;
+                        if (sub == 0 && r3 < lp4 - lp3) prefetch_l2(p.level_nodes + lp3 + r3);     // node id, level l+3
+                        if (vB >= 0) {                                                            // level l+2's node
+                            if (sub == 0) prefetch_l2(p.nbr_pad + (size_t)vB * W);
+                            if ((sub & 1) == 0) prefetch_l2((const char*)p.H + (size_t)vB * p.ldh * 2 + sub * 16);
+                        }
+                        if (vC >= 0) {                                                            // level l+1's node
+                            const int cnt_c = __shfl_sync(gmask, padC, grp_base);
+#pragma unroll
+                            for (int j = 1; j < MAXN; ++j) {
+                                const int uj = __shfl_sync(gmask, padC, grp_base + j);
+                                if (j < cnt_c) prefetch_l2(kv_tab + (size_t)uj * 512 + sub * 32);
+                            }
+                        }
                     }
                     if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
