@@ -13,19 +13,23 @@
 //   1. gather the K | V rows of every OTHER neighbour from layer k's K|V table (16 lanes per node, 16 bytes per
 //      lane), compute scores, softmax and the weighted value sum in registers, and write the 16 x 128
 //      attention tile into shared memory in operand layout;
-//   2. output projection, transposed again: D[feature, node] = W_o * O^T, so a small tile costs a fraction of a
-//      128-row tile and all warps take part in the epilogue (128 TMEM lanes x 16 columns);
+//   2. output projection by warp-level MMAs (mma.sync m16n8k16, W_o in shared memory): warp w computes output
+//      features 16w .. 16w+15 of all 16 nodes, and the result is in registers when the last instruction retires.
+//      This product sits on the level-to-level chain, and an asynchronous tcgen05 group costs an order / issue /
+//      commit / barrier / tcgen05.ld round trip that for its 8 instructions is longer than the product itself;
 //   3. add the residual (the input rows still in shared memory), round to bf16, write the new rows to H and --
 //      in operand layout again -- to shared memory;
-//   4. from the new rows, transposed: the tile's K | V rows of layer k, stored to the table so that higher levels
-//      gather updated rows.
+//   4. from the new rows, transposed (tcgen05.mma, 16 instructions: here the asynchronous path is the cheaper
+//      one): the tile's K | V rows of layer k, stored to the table so that higher levels gather updated rows.
+//      While that product runs, the lanes ask L2 (prefetch, nothing waits for it) for what the coming levels'
+//      first loads will want: node ids, neighbour-table entries, input rows, the next level's neighbours' K | V.
 // The prologue of a CTA's NEXT tile is folded into the main part of the current one: the next tile's rows are
 // requested once the layer below is known to have finished them, they are written to the second input buffer
 // before the barrier that precedes step 4, and their Q | K | V product is issued right behind step 4's MMAs, so
 // it runs while the CTA stores its rows, arrives and waits for the level to complete.  The level-to-level chain
 // is then wait -> gather -> W_o -> K|V refresh -> arrive; the projections of the next tile hide in the hand-off.
 // A CTA that has no tile in a level but has one in the next does that prologue while it is idle.
-// The MMAs are issued by a thread of a ninth warp that does nothing else: issuing an M128 x N16 x K16 instruction
+// The tcgen05 MMAs are issued by a thread of a ninth warp that does nothing else: issuing an M128 x N16 x K16 instruction
 // occupies the issuing thread for about as long as the tensor pipe needs to execute it, so a worker thread that
 // issued the next tile's 24 instructions would hold up its own warp's epilogue (and with it the level) for their
 // whole duration.  The workers hand the issuing thread one order at a time (a word in shared memory and an
@@ -33,9 +37,9 @@
 //
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
-// to layers round-robin; each keeps its layer's W_o, W_k, W_v and W_q resident in TENSOR memory (four blocks
-// of 128 lanes x 64 columns beside the accumulators) and issues its MMAs with the A operand read from there, so
-// the weights are never re-read from shared memory and shared memory holds only the node-side tiles.  With n
+// to layers round-robin; each keeps its layer's W_k, W_v and W_q resident in TENSOR memory (blocks of 128 lanes
+// x 64 columns beside the accumulators) and issues its tcgen05 MMAs with the A operand read from there, so
+// those weights are never re-read from shared memory, which holds the node-side tiles and W_o.  With n
 // layers the dependent chain is n_levels + n - 1 tile steps long instead of n * n_levels, while computing exactly
 // what n successive level-by-level sweeps compute.
 //
@@ -64,10 +68,10 @@ constexpr int kThreads = kWorkers + 32;      // and a ninth warp whose first lan
 constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
 constexpr int kTileOp = 2 * kBHalf;          // a kTile x 128 bf16 tile in operand layout (4 KiB)
 constexpr int kTmemCols = 512;
-constexpr int kAccO = 0, kAccK2 = 1, kAccV2 = 2, kAccQ = 3, kAccK = 4, kAccV = 5;   // accumulators of kTile columns
-constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks W_o | W_k | W_v | W_q
+constexpr int kAccK2 = 1, kAccV2 = 2, kAccQ = 3, kAccK = 4, kAccV = 5;   // accumulators of kTile columns (slot 0 unused)
+constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks ( - | W_k | W_v | W_q )
 constexpr int kWCols = 64;                   // a 128 x 128 bf16 block: 128 lanes x 64 columns of two elements
-constexpr int kBlkO = 0, kBlkK = 1, kBlkV = 2, kBlkQ = 3;
+constexpr int kBlkK = 1, kBlkV = 2, kBlkQ = 3;            // weight blocks in tensor memory (slot 0 unused)
 constexpr int kStageRow = 768 + 16;          // staging per node: Q 256 | K 256 | V 256 (+ padding against bank conflicts)
 
 constexpr int kOffO = 0;                               // attention tile (operand layout)
@@ -129,11 +133,6 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t* r) {
 }
 __device__ __forceinline__ void st_shared_b16(uint32_t addr, uint16_t v) {
     asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
-}
-__device__ __forceinline__ uint16_t ld_shared_b16(uint32_t addr) {
-    uint16_t v;
-    asm volatile("ld.shared.b16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
-    return v;
 }
 __device__ __forceinline__ void st_global_v4(void* p, const uint32_t* r) {
     asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
@@ -259,9 +258,8 @@ levelised_kernel(LevParams p) {
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
     if (warp < 8) {
-        for (int blk = 0; blk < 4; ++blk) {
-            const __nv_bfloat16* wb = blk == kBlkO ? p.Wo[layer]
-                                     : blk == kBlkQ ? p.Wqkv[layer]
+        for (int blk = kBlkK; blk <= kBlkQ; ++blk) {
+            const __nv_bfloat16* wb = blk == kBlkQ ? p.Wqkv[layer]
                                                     : p.Wqkv[layer] + (size_t)blk * 128 * 128;     // kBlkK = 1, kBlkV = 2
             const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
 #pragma unroll
@@ -286,7 +284,7 @@ levelised_kernel(LevParams p) {
 
     const uint32_t idesc = idesc_bf16_f32(128, kTile);
     // matrix descriptors of the node-side operands; stepping along K only adds to the address field
-    const uint64_t dO = smem_desc_sw128(sO), dHp = smem_desc_sw128(sHp);
+    const uint64_t dHp = smem_desc_sw128(sHp);
     const uint64_t dX[2] = {smem_desc_sw128(sX), smem_desc_sw128(sX + kTileOp)};
     // issues Q | K | V = W * X^T for the rows in input buffer b (one thread)
     auto issue_qkv = [&](int b) {
