@@ -372,9 +372,13 @@ def run_ours(args, w):
         ln_ms = timed3(lambda: dg4.dg4_layernorm_fwd(gr, dsc, x_dev, gam, bet, 1e-5, o_v))
         blk_ms = timed3(lambda: dg4.dg4_block_fwd_parallel(gr, dsc, x_dev, wq[0], wo[0], gam, bet, w1, b1, w2, b2, gam,
                                                            bet, 1e-5, h_par, ws))
+        # the all-parallel layer in its opt-in one-kernel form (K|V projection + fused kernel), for comparison
+        # with the three kernels timed inside the step
+        dsc_fused = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, fused_layer=True)
+        fused_ms = timed3(lambda: dg4.dg4_layer_fwd_parallel(gr, dsc_fused, x_dev, wq[0], wo[0], h_par, ws))
         extras.update({"ffn_ms": ffn_ms, "ffn_tflops": 4.0 * 128 * 512 * n / (ffn_ms * 1e-3) / 1e12,
                        "layernorm_ms": ln_ms, "layernorm_gbs": 512.0 * n / (ln_ms * 1e-3) / 1e9,
-                       "block_parallel_ms": blk_ms})
+                       "block_parallel_ms": blk_ms, "parallel_layer_fused_ms": fused_ms})
         del w1, w2
         # the paper's cone depth (k = 8) on the 1M-node circuit: the warp-per-node kernel for wider cones
         w3 = synth.workload(3)

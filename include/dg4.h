@@ -48,8 +48,12 @@ typedef enum { DG4_F32 = 0, DG4_BF16 = 1 } dg4_dtype;
 
 enum {
     DG4_FLAG_RESIDUAL = 1,     /* output projection adds the layer's input row                */
-    DG4_FLAG_LEVEL_LAUNCHES = 2 /* levelised layer: one group of kernel launches per level instead of the
+    DG4_FLAG_LEVEL_LAUNCHES = 2, /* levelised layer: one group of kernel launches per level instead of the
                                   single persistent kernel (same results; kept for comparison)   */
+    DG4_FLAG_FUSED_LAYER = 4   /* all-parallel layer: the K|V projection followed by ONE kernel (queries from
+                                  the X tiles, attention, output projection, residual; Q and O never reach
+                                  memory) instead of three kernels.  Same results bit for bit; measured a
+                                  little slower to equal, so it is not the default.  bf16, two hops at most */
 };
 
 /* Per-call description of the attention layer. */
@@ -266,6 +270,9 @@ size_t dg4_layer_workspace_bytes(const dg4_graph* g, const dg4_desc* desc);
  * restricted to cone_k(v)): QKV projection -> sparse attention -> output projection (+ residual),
  * every node reading the same input H_in.   H_in, H_out: device [n, d] bf16; they may be the same buffer
  * only if ldh == ldho (rows are then updated in place after all reads of the layer's input are done).
+ * With DG4_FLAG_FUSED_LAYER (bf16, heads a power of two up to 16, cones of two hops at most; ignored otherwise) the
+ * layer runs as the K|V projection followed by one kernel that never writes Q or O to memory; the rows it
+ * produces are the same bit for bit.
  */
 dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc* desc,
                                   const void* H_in, int64_t ldh, const void* W_qkv, const void* W_o,

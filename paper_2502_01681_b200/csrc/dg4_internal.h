@@ -38,6 +38,12 @@ dg4_status dg4i_check_tensor(const char* name, const void* p, int64_t ld, int el
 uint32_t dg4i_poll_limit();
 #define DG4I_DEFAULT_POLL_LIMIT (1u << 24)
 
+// ---- tensor maps -----------------------------------------------------------------------------------
+// Tensor map over a [rows, 128] bf16 row-major matrix with leading dimension ld (elements): box = 64 columns x
+// box_rows rows, 128-byte swizzle, rows past the end read as zero and are clipped on store (dg4_project.cu).
+struct CUtensorMap_st;
+dg4_status dg4i_make_row_map(CUtensorMap_st* map, const void* base, int64_t rows, int64_t ld, int box_rows);
+
 // ---- launch accounting (every kernel launch of the library bumps this counter) ------------------
 void dg4i_count_launch(int n = 1);
 
@@ -131,6 +137,14 @@ struct dg4i_proj_args {
     int32_t* status = nullptr;         // device status word: receives DG4_ERR_TIMEOUT if a bounded wait runs out
 };
 dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st);
+
+// The all-nodes-parallel layer behind its K | V projection as one kernel (dg4_fused.cu): Q from the X tiles,
+// attention, output projection (+ residual) per 128-node tile.  Supported for bf16, heads a power of two up to
+// 16, and graphs with the fixed-width neighbour table (two hops at most).
+bool dg4i_fused_layer_supported(const dg4_graph* g, const dg4_desc* desc);
+dg4_status dg4i_fused_layer_launch(const dg4_graph* g, const dg4_desc* desc, const __nv_bfloat16* X, int64_t ldx,
+                                   const __nv_bfloat16* KV, const __nv_bfloat16* W_q, const __nv_bfloat16* W_o,
+                                   __nv_bfloat16* H_out, int64_t ldho, int32_t* status, cudaStream_t st);
 
 // Persistent levelised kernel over n_layers layers run as a wavefront.  KV[k] ([n, 256] bf16, contents irrelevant on
 // entry) receives layer k's K | V rows of the nodes as they are updated.  H is updated in place.  `sync` is zeroed

@@ -242,6 +242,18 @@ extern "C" dg4_status dg4_layer_fwd_parallel(const dg4_graph* g, const dg4_desc*
     Workspace w = carve(workspace, g->n);
     int32_t* status_word = g->dev_status;
 
+    if ((desc->flags & DG4_FLAG_FUSED_LAYER) && dg4i_fused_layer_supported(g, desc)) {
+        // K | V of every node first (every node may be gathered by any other), then one kernel for the rest:
+        // queries from the X tiles, attention, output projection, residual -- Q and O never leave the chip
+        dg4i_proj_args kv;
+        kv.A = (const __nv_bfloat16*)H_in; kv.lda = ldh; kv.W = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128; kv.n_out = 256;
+        kv.out[0] = w.KV; kv.ldo[0] = 256; kv.out[1] = w.KV + 128; kv.ldo[1] = 256; kv.out[2] = nullptr; kv.ldo[2] = 0;
+        kv.R = nullptr; kv.ldr = 0; kv.row_list = nullptr; kv.first = 0; kv.rows = g->n; kv.status = status_word;
+        CHECK(dg4i_proj_launch(kv, st));
+        return dg4i_fused_layer_launch(g, desc, (const __nv_bfloat16*)H_in, ldh, w.KV, (const __nv_bfloat16*)W_qkv,
+                                       (const __nv_bfloat16*)W_o, (__nv_bfloat16*)H_out, ldho, status_word, st);
+    }
+
     dg4i_proj_args p;
     p.A = (const __nv_bfloat16*)H_in; p.lda = ldh; p.W = (const __nv_bfloat16*)W_qkv; p.n_out = 384;
     p.out[0] = w.Q; p.ldo[0] = 128; p.out[1] = w.KV; p.ldo[1] = 256; p.out[2] = w.KV + 128; p.ldo[2] = 256;

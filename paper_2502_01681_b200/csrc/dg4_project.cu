@@ -379,14 +379,14 @@ dg4_status get_encoder(EncodeTiledFn* fn) {
     return DG4_OK;
 }
 
-// [rows, 128] bf16 row-major with leading dimension ld; box = 64 columns x 128 rows, 128-byte swizzle.
-dg4_status make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) {
+// [rows, 128] bf16 row-major with leading dimension ld; box = 64 columns x box_rows rows, 128-byte swizzle.
+dg4_status make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld, int box_rows = 128) {
     EncodeTiledFn enc;
     dg4_status s = get_encoder(&enc);
     if (s != DG4_OK) return s;
     cuuint64_t dims[2] = {128, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)(ld * 2)};
-    cuuint32_t box[2] = {64, 128};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -396,6 +396,10 @@ dg4_status make_map(CUtensorMap* m, const void* base, int64_t rows, int64_t ld) 
 }
 
 }  // namespace
+
+dg4_status dg4i_make_row_map(CUtensorMap_st* map, const void* base, int64_t rows, int64_t ld, int box_rows) {
+    return make_map(map, base, rows, ld, box_rows);
+}
 
 dg4_status dg4i_proj_launch(const dg4i_proj_args& a, cudaStream_t st) {
     if (a.rows <= 0) return DG4_OK;

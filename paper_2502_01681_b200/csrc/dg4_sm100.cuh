@@ -39,6 +39,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     }
     return mbar_test(bar, parity);
 }
+// For roles that wait long and need no prompt wake-up (a producer or an epilogue a whole tile ahead of its
+// consumer): the hardware suspends the thread inside try_wait for up to the hinted time instead of having it
+// spin, so the waiting warps leave the issue slots to the warps that share their scheduler.  `limit` counts
+// polls of about `kRelaxedWaitNs` each; callers pass the launch's poll limit, which is scaled down accordingly.
+constexpr uint32_t kRelaxedWaitNs = 640;
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, uint32_t limit = kDefaultPollLimit) {
+    const uint32_t tries = (limit >> 4) + 1u;          // 16 ordinary polls of ~40 ns are about one suspended wait
+    for (uint32_t i = 0; i < tries; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(kRelaxedWaitNs) : "memory");
+        if (ok) return true;
+    }
+    return mbar_test(bar, parity);
+}
+__device__ __forceinline__ bool mbar_wait_relaxed_warp(uint32_t bar, uint32_t parity, uint32_t limit = kDefaultPollLimit) {
+    return __all_sync(0xffffffffu, mbar_wait_relaxed(bar, parity, limit) ? 1 : 0) != 0;
+}
 // The same for a whole (converged) warp, with one answer for all 32 lanes: true only if every lane saw the phase
 // complete.  Code that follows may then branch on the result and still execute warp-wide instructions together.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, uint32_t limit = kDefaultPollLimit) {

@@ -30,6 +30,7 @@ DG4_ERR_TIMEOUT = -8
 DG4_F32, DG4_BF16 = 0, 1
 DG4_FLAG_RESIDUAL = 1
 DG4_FLAG_LEVEL_LAUNCHES = 2
+DG4_FLAG_FUSED_LAYER = 4
 
 (DG4_ARR_NBR_PTR, DG4_ARR_NBR_IDX, DG4_ARR_LEVEL_PTR, DG4_ARR_LEVEL_NODES, DG4_ARR_PERM, DG4_ARR_CLASS_PTR,
  DG4_ARR_LEVEL_PERM, DG4_ARR_LEVEL_CLASS_PTR, DG4_ARR_NBR_PAD) = range(9)
@@ -187,8 +188,9 @@ def _ld(t):
 
 
 def desc(heads: int, dtype: int, scale: float, residual: bool = False, d: int = 128,
-         level_launches: bool = False) -> dg4_desc:
-    flags = (DG4_FLAG_RESIDUAL if residual else 0) | (DG4_FLAG_LEVEL_LAUNCHES if level_launches else 0)
+         level_launches: bool = False, fused_layer: bool = False) -> dg4_desc:
+    flags = ((DG4_FLAG_RESIDUAL if residual else 0) | (DG4_FLAG_LEVEL_LAUNCHES if level_launches else 0)
+             | (DG4_FLAG_FUSED_LAYER if fused_layer else 0))
     return dg4_desc(d, heads, dtype, flags, float(scale))
 
 

@@ -91,6 +91,11 @@ def test_waits_that_run_out_wind_the_kernels_down_and_report_timeout():
         gr, ws = fresh()                                # feed-forward kernel
         dg4.dg4_ffn_fwd(gr, dsc, x, w1, b1, w2, vec, vec, vec, 1e-5, y)
         assert dg4.dg4_graph_poll_status(gr) == dg4.DG4_ERR_TIMEOUT
+        gr, ws = fresh()                                # one-kernel form of the parallel layer (behind its K|V projection)
+        h = x.clone()
+        dg4.dg4_layer_fwd_parallel(gr, dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True, fused_layer=True),
+                                   h, dwq, dwo, h, ws)
+        assert dg4.dg4_graph_poll_status(gr) == dg4.DG4_ERR_TIMEOUT
         gr, ws = fresh()                                # persistent levelised kernel (its table-filling projection too)
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         h = x.clone()
@@ -106,8 +111,14 @@ def test_waits_that_run_out_wind_the_kernels_down_and_report_timeout():
     h = x.clone()
     dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dwq] * 3, [dwo] * 3, ws, status)
     dg4.dg4_qkv_project(gr, dsc, x, dwq, q, k, v)
+    hf = x.clone()
+    dg4.dg4_layer_fwd_parallel(gr, dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True, fused_layer=True),
+                               hf, dwq, dwo, hf, ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and dg4.dg4_graph_poll_status(gr) == 0
+    want_par = orc.layer_parallel(f64_of_bits(xb), wq, wo, *orc.neighbourhood(g.row_ptr, g.col_idx, w.hops), w.heads,
+                                  w.scale, residual=True, rounding="bf16")
+    assert rel_row_err(host_f64_of_bf16(hf), want_par).max() <= BF16_ROW_TOL
     ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
     lptr, lnodes = orc.level_buckets(g.level)
     want = f64_of_bits(xb)

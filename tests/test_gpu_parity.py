@@ -241,7 +241,8 @@ def _weights(w, layers):
 
 
 def _run_layers_gpu(gr, w, xb, weights, mode):
-    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, level_launches=(mode == "level-launches"))
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, level_launches=(mode == "level-launches"),
+                   fused_layer=(mode == "fused"))
     ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, len(weights))),
                      dtype=torch.uint8, device="cuda")
     h = dev_bf16(xb).clone()
@@ -253,22 +254,23 @@ def _run_layers_gpu(gr, w, xb, weights, mode):
         assert int(status.item()) == 0
         return host_f64_of_bf16(h)
     for (wq_bits, _, wo_bits, _) in weights:
-        if mode == "parallel":
+        if mode in ("parallel", "fused"):
             dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), h, ws)
         else:
             dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), ws, status)
             assert int(status.item()) == 0
     torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(gr) == 0
     return host_f64_of_bf16(h)
 
 
 def _run_layers_checker(g, w, xb, weights, mode):
     ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
     h = f64_of_bits(xb)
-    if mode != "parallel":
+    if mode not in ("parallel", "fused"):
         lptr, lnodes = orc.level_buckets(g.level)
     for (_, wq, _, wo) in weights:
-        if mode == "parallel":
+        if mode in ("parallel", "fused"):
             h = orc.layer_parallel(h, wq, wo, ptr, idx, w.heads, w.scale, residual=w.residual, rounding="bf16")
         else:
             h = orc.layer_levelised(h, wq, wo, ptr, idx, lptr, lnodes, w.heads, w.scale, residual=w.residual,
@@ -277,6 +279,7 @@ def _run_layers_checker(g, w, xb, weights, mode):
 
 
 @pytest.mark.parametrize("cfg,shrink,mode", [(2, 1, "parallel"), (2, 7, "parallel"), (5, 200, "parallel"),
+                                             (2, 1, "fused"), (2, 7, "fused"), (5, 200, "fused"), (4, 5, "fused"),
                                              (4, 20, "levelised"), (5, 400, "levelised"), (2, 10, "levelised"),
                                              (4, 5, "levelised"), (5, 50, "levelised"),
                                              (4, 20, "level-launches"), (5, 400, "level-launches"),
@@ -292,6 +295,37 @@ def test_layers_match_checker(cfg, shrink, mode):
     want = _run_layers_checker(g, w, xb, weights, mode)
     err = rel_row_err(got, want)
     assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
+
+
+@pytest.mark.parametrize("n_gates,heads,residual", [(1, 8, True), (63, 8, True), (128, 2, False), (129, 8, True),
+                                                    (20000, 16, True), (33333, 1, False)])
+def test_fused_layer_is_bit_identical_to_the_three_kernels(n_gates, heads, residual):
+    """The one-kernel form of the all-parallel layer computes the same products with the same roundings in the
+    same order: its rows must equal the three-kernel path's bit for bit (and that path is checked against the
+    oracle above), for ragged sizes, in place and out of place."""
+    rng = np.random.default_rng(n_gates + heads)
+    fanins = random_dag(rng, 17, n_gates, window=500)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    n = len(fanins)
+    gr = dg4.dg4_graph_create(rp, ci, level, 2, 0)
+    x = dev_bf16(synth.normal_bf16_bits(11, 1, (n, 128), 1.0))
+    wq = dev_bf16(bf16_weights(synth.normal_f32(11, 2, (384, 128), 0.08))[0])
+    wo = dev_bf16(bf16_weights(synth.normal_f32(11, 3, (128, 128), 0.08))[0])
+    scale = 1.0 / np.sqrt(128 // heads)
+    outs = []
+    for fused in (False, True):
+        dsc = dg4.desc(heads, dg4.DG4_BF16, scale, residual=residual, fused_layer=fused)
+        ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+        h = torch.zeros_like(x)
+        dg4.dg4_layer_fwd_parallel(gr, dsc, x, wq, wo, h, ws)
+        inplace = x.clone()
+        dg4.dg4_layer_fwd_parallel(gr, dsc, inplace, wq, wo, inplace, ws)
+        torch.cuda.synchronize()
+        assert dg4.dg4_graph_poll_status(gr) == 0
+        assert bool((h.view(torch.int16) == inplace.view(torch.int16)).all())
+        outs.append(h.view(torch.int16).clone())
+    assert bool((outs[0] == outs[1]).all()), int((outs[0] != outs[1]).any(dim=1).sum())
 
 
 def test_levelised_differs_from_parallel_and_is_repeatable():
@@ -358,7 +392,8 @@ def test_bounded_wait_runs_out_and_reports_timeout():
 
 @pytest.mark.parametrize("hops,heads,residual,mode", [(1, 1, True, "wavefront"), (2, 4, False, "wavefront"),
                                                       (2, 16, True, "wavefront"), (1, 2, False, "parallel"),
-                                                      (2, 16, True, "parallel"), (1, 4, True, "level-launches")])
+                                                      (2, 16, True, "parallel"), (1, 4, True, "level-launches"),
+                                                      (1, 2, False, "fused"), (2, 16, True, "fused"), (2, 1, True, "fused")])
 def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
     rng = np.random.default_rng(1000 * hops + heads)
     fanins = random_dag(rng, 40, 6000, window=300)
@@ -370,11 +405,12 @@ def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
     weights = [bf16_weights(synth.normal_f32(7, 10 + l, (384, 128), 0.05)) +
                bf16_weights(synth.normal_f32(7, 20 + l, (128, 128), 0.05)) for l in range(2)]
     scale = 1.0 / np.sqrt(128 // heads)
-    dsc = dg4.desc(heads, dg4.DG4_BF16, scale, residual=residual, level_launches=(mode == "level-launches"))
+    dsc = dg4.desc(heads, dg4.DG4_BF16, scale, residual=residual, level_launches=(mode == "level-launches"),
+                   fused_layer=(mode == "fused"))
     ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, 2)),
                      dtype=torch.uint8, device="cuda")
     h = dev_bf16(xb).clone()
-    if mode == "parallel":
+    if mode in ("parallel", "fused"):
         for w_ in weights:
             dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(w_[0]), dev_bf16(w_[2]), h, ws)
     else:
@@ -385,7 +421,7 @@ def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
     lptr, lnodes = orc.level_buckets(level)
     want = f64_of_bits(xb)
     for (_, wq, _, wo) in weights:
-        if mode == "parallel":
+        if mode in ("parallel", "fused"):
             want = orc.layer_parallel(want, wq, wo, ptr, idx, heads, scale, residual=residual, rounding="bf16")
         else:
             want = orc.layer_levelised(want, wq, wo, ptr, idx, lptr, lnodes, heads, scale, residual=residual,
