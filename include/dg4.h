@@ -120,8 +120,7 @@ int64_t dg4_launch_count(void);
  *   hops        1 (fan-ins + self), 2 (2-hop fan-in cone + self), or 3 .. 8 (wider cones, the paper uses k = 8:
  *               up to 2^(hops+1)-1 members).  For hops > 2 only the neighbourhood CSR and the level buckets are
  *               built (no fixed-width table, no class orderings: exporting those returns DG4_ERR_UNSUPPORTED),
- *               the lists must stay below 2^31 entries, dg4_graph_rebuild is not available, and the levelised
- *               layer runs only with DG4_FLAG_LEVEL_LAUNCHES.
+ *               the lists must stay below 2^31 entries and dg4_graph_rebuild is not available.
  *   perm_chunk  0 (one chunk) or a positive multiple of 1024
  *   device      CUDA ordinal; made current for the duration of the call and restored
  *   out         receives the handle; untouched on error

@@ -280,8 +280,6 @@ extern "C" dg4_status dg4_layer_fwd_levelised(const dg4_graph* g, const dg4_desc
     if (device_status) DG4_CUDA_TRY(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
     int32_t* status_word = device_status ? device_status : g->dev_status;
 
-    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
-        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layer needs DG4_FLAG_LEVEL_LAUNCHES");
     if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES)) {
         // one persistent kernel walks the levels; it projects each tile's own Q | K | V on the fly and fills the
         // K | V table as nodes are updated
@@ -354,8 +352,6 @@ extern "C" dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_des
                  layers_workspace_bytes(g, n_layers));
     cudaStream_t st = (cudaStream_t)stream;
 
-    if (g->wide && !(desc->flags & DG4_FLAG_LEVEL_LAUNCHES))
-        DG4_FAIL(DG4_ERR_UNSUPPORTED, "cones wider than two hops: the levelised layers need DG4_FLAG_LEVEL_LAUNCHES");
     if (desc->flags & DG4_FLAG_LEVEL_LAUNCHES) {       // comparison driver: layer after layer, a launch group per level
         for (int k = 0; k < n_layers; ++k)
             CHECK(dg4_layer_fwd_levelised(g, desc, H, ldh, W_qkv[k], W_o[k], workspace, workspace_bytes_, device_status, stream));

@@ -35,6 +35,11 @@
 // whole duration.  The workers hand the issuing thread one order at a time (a word in shared memory and an
 // mbarrier arrival) and wait only for the completion barrier of the product they need next.
 //
+// Cones wider than two hops (MAXN = 0) come as lists instead of the fixed-width table: step 1 then walks a node's
+// list in batches of four entries with an online softmax, two batches in flight.  A tile's time is then the serial
+// walk of its longest list, so narrow levels are spread over all of the layer's CTAs and the slots a tile has
+// left over take replicas of its nodes, each walking a share of the list; the shares are merged in shared memory.
+//
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
 // to layers round-robin; each keeps its layer's W_k, W_v and W_q resident in TENSOR memory (blocks of 128 lanes
@@ -62,7 +67,8 @@ namespace {
 using namespace sm100;
 using namespace attn;
 
-constexpr int kTile = 16;                    // nodes per tile
+constexpr int kTile = 16;                    // node slots per tile
+constexpr int kMergeRow = 12;                // floats a lane parks for the merge of a split list: m, z, 8 sums (+ padding)
 constexpr int kWorkers = kTile * 16;         // 16 lanes per node: eight warps that gather, attend and run the epilogues
 constexpr int kThreads = kWorkers + 32;      // and a ninth warp whose first lane issues every tcgen05.mma
 constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand tile
@@ -79,7 +85,8 @@ constexpr int kOffHp = kOffO + kTileOp;                // new rows (operand layo
 constexpr int kOffX = kOffHp + kTileOp;                // input rows of the current and of the next tile (operand layout)
 constexpr int kOffHres = kOffX + 2 * kTileOp;          // the same rows, plain [kTile][256 B], twice
 constexpr int kOffStage = kOffHres + 2 * kTile * 256;  // staging, plain [kTile][kStageRow]
-constexpr int kOffMisc = kOffStage + kTile * kStageRow;
+constexpr int kOffMerge = kOffStage + kTile * kStageRow;        // wide cones: partial softmaxes of a node's replicas
+constexpr int kOffMisc = kOffMerge + kWorkers * kMergeRow * 4;
 constexpr int kWHalf = 128 * 128;                      // K-half of a 128-row weight block: 128 rows x 128 bytes
 constexpr int kWBlock = 2 * kWHalf;                    // a 128 x 128 bf16 block in shared memory (32 KiB)
 constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o for the warp-level output projection
@@ -112,7 +119,9 @@ struct LevParams {
     const __nv_bfloat16* Wqkv[DG4I_MAX_LAYERS];  // [384, 128] per layer
     __nv_bfloat16* H;                      // [n, ldh], updated in place by every layer in turn
     int64_t ldh;
-    const int32_t* nbr_pad;                // [n, pad_width]
+    const int32_t* nbr_pad;                // [n, pad_width] (cones of at most two hops)
+    const int32_t* nbr_ptr;                // [n + 1], [n_nbr]: the cones as lists (wider cones)
+    const int32_t* nbr_idx;
     const int32_t* level_ptr;
     const int32_t* level_nodes;
     int32_t n_levels;
@@ -213,7 +222,9 @@ template <int LPH, int MAXN>
 __global__ void __launch_bounds__(kThreads, 1)
 levelised_kernel(LevParams p) {
     extern __shared__ uint8_t smem_raw[];
-    constexpr int W = MAXN + 1;                          // width of a neighbour-table entry
+    constexpr bool WIDE = (MAXN == 0);                   // cones wider than two hops: CSR lists instead of the table
+    constexpr int NK = WIDE ? 1 : MAXN;
+    constexpr int W = WIDE ? 2 : MAXN + 1;               // words of a node's index entry: table row, or its list bounds
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     Misc* misc = reinterpret_cast<Misc*>(base_ptr + kOffMisc);
@@ -360,7 +371,20 @@ levelised_kernel(LevParams p) {
         int32_t* my_arrive = p.arrive + (size_t)layer * p.n_levels;
         const int32_t* prev_arrive = layer > 0 ? p.arrive + (size_t)(layer - 1) * p.n_levels : nullptr;
         const int prev_ctas = layer > 0 ? ctas_of(layer - 1) : 0;
-        auto prev_target = [&](int tiles_of_level) { return tiles_of_level < prev_ctas ? tiles_of_level : prev_ctas; };
+        // Nodes per tile of a level.  With the fixed-width table: 16, on as few CTAs as that takes (spreading a
+        // narrow level over all CTAs was measured 2 % slower: more arrivals per level, nothing saved).  With cone
+        // lists, where a tile's time is the serial walk of its longest list, a level narrower than ctas x 16
+        // nodes is spread over all the layer's CTAs, and the slots a tile has left over take REPLICAS of its
+        // nodes: replica q of `parts` walks every parts-th batch of the list, and the partial softmaxes are
+        // merged through shared memory.
+        auto per_tile = [&](int n_level, int ctas) {
+            if (!WIDE) return kTile;
+            const int t = (n_level + ctas - 1) / ctas;
+            return t < 1 ? 1 : (t > kTile ? kTile : t);
+        };
+        auto tiles_of = [&](int n_level, int ctas) { const int t = per_tile(n_level, ctas); return (n_level + t - 1) / t; };
+        // arrivals on the layer below's counter for a level of n_level nodes (one per CTA that owns a tile of it)
+        auto prev_target = [&](int n_level) { const int t = tiles_of(n_level, prev_ctas); return t < prev_ctas ? t : prev_ctas; };
 
         // this lane's piece of node v's input row (zero for an empty slot) into input buffer b, both layouts
         auto stage_input = [&](int b, const Piece& x) {
@@ -382,11 +406,15 @@ levelised_kernel(LevParams p) {
         // so a plain load at the top of a level would cost a trip to L2 on the level-to-level chain.
         auto lp_at = [&](int lv) { return p.level_ptr[lv < p.n_levels ? lv : p.n_levels]; };
         auto stage_node = [&](int lv_first, int lv_end) -> int {   // node of (first tile of this CTA, this slot) of a level
-            const int r = bid * kTile + slot;
-            return (r < lv_end - lv_first) ? p.level_nodes[lv_first + r] : -1;
+            const int t = per_tile(lv_end - lv_first, nctas);
+            const int r = bid * t + slot % t;
+            return (slot / t < kTile / t && r < lv_end - lv_first) ? p.level_nodes[lv_first + r] : -1;
         };
         int lp0 = lp_at(0), lp1 = lp_at(1), lp2 = lp_at(2), lp3 = lp_at(3);
-        auto pad_of = [&](int v) -> int { return (v >= 0 && sub < W) ? p.nbr_pad[(size_t)v * W + sub] : 0; };
+        auto pad_of = [&](int v) -> int {
+            if (v < 0 || sub >= W) return 0;
+            return WIDE ? p.nbr_ptr[v + sub] : p.nbr_pad[(size_t)v * W + sub];
+        };
         int v0 = stage_node(lp0, lp1);                     // level l  : node id and this lane's table word
         int pad0 = pad_of(v0);
         int vC = stage_node(lp1, lp2);                     // level l+1: node id
@@ -406,8 +434,9 @@ levelised_kernel(LevParams p) {
                 vB = stage_node(lp2, lp3);
                 padC = pad_of(vC);
             };
-            const int tiles = (n_l + kTile - 1) / kTile;
-            const int tiles_next = (lp2 - lp1 + kTile - 1) / kTile;      // tiles of level l + 1
+            const int T_l = per_tile(n_l, nctas);                         // nodes per tile in this level
+            const int tiles = (n_l + T_l - 1) / T_l;
+            const int tiles_next = tiles_of(lp2 - lp1, nctas);            // tiles of level l + 1
             if (!(n_l > 0 && bid < tiles)) issue_chains();
             if (n_l > 0 && bid < tiles) {
                 bool waited = false;
@@ -421,8 +450,8 @@ levelised_kernel(LevParams p) {
                     }
                     const bool more_here = tile + nctas < tiles;
                     {
-                        const int r = (tile + nctas) * kTile + slot;
-                        v_nx = (more_here && r < n_l) ? p.level_nodes[first + r] : -1;
+                        const int r = (tile + nctas) * T_l + slot % T_l;
+                        v_nx = (more_here && slot / T_l < kTile / T_l && r < n_l) ? p.level_nodes[first + r] : -1;
                     }
                     const bool valid = v >= 0;
                     // which tile comes next for this CTA, and may its rows be requested already?  Asked twice: at the
@@ -432,7 +461,7 @@ levelised_kernel(LevParams p) {
                     const bool want_pre = more_here || next_level_tile;
                     auto next_rows_ready = [&]() -> int {
                         if (!want_pre) return 0;
-                        if (next_level_tile && prev_arrive) return ld_acquire(prev_arrive + l + 1) >= prev_target(tiles_next) ? 1 : 0;
+                        if (next_level_tile && prev_arrive) return ld_acquire(prev_arrive + l + 1) >= prev_target(lp2 - lp1) ? 1 : 0;
                         return 1;
                     };
                     if (waited && tid == 32) misc->pre_early = next_rows_ready();   // visible after the barrier below
@@ -472,7 +501,7 @@ levelised_kernel(LevParams p) {
                             misc->go = go ? 1 : 0;
                         } else if (tid == 32) {
                             bool go = true;
-                            if (prev_arrive && !pro_ready) go = wait_counter(prev_arrive + l, prev_target(tiles), p.abort_word, counter_limit);
+                            if (prev_arrive && !pro_ready) go = wait_counter(prev_arrive + l, prev_target(n_l), p.abort_word, counter_limit);
                             if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                             misc->go2 = go ? 1 : 0;
                             misc->pre_early = go ? next_rows_ready() : 0;
@@ -496,39 +525,161 @@ levelised_kernel(LevParams p) {
                     const uint32_t sHres_cur = sHres + (uint32_t)(buf * kTile * 256);
 
                     // ---- gather and attend
-                    Piece kq[MAXN], vq[MAXN], qp;
-                    int u[MAXN];
-                    const int cnt = valid ? __shfl_sync(gmask, pad, grp_base) : 1;
-                    u[0] = v;
-#pragma unroll
-                    for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(gmask, pad, grp_base + j);
                     float acc[8];
-                    if (valid) {
-#pragma unroll
-                        for (int j = 1; j < MAXN; ++j)
-                            if (j < cnt) vq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + 256 + sub * 16);
-#pragma unroll
-                        for (int j = 1; j < MAXN; ++j)
-                            if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
-                    }
-                    if (tile == bid) issue_chains();
+                    Piece xpre;
                     const int v_pre = more_here ? v_nx : vC;
                     const bool pre_early = want_pre && misc->pre_early != 0;
-                    Piece xpre;
-                    if (pre_early) xpre = load_input(v_pre);                      // the next tile's input rows
-                    else if (tid == 32) misc->pre_ok = next_rows_ready();         // second look; read after the next barrier
-                    {   // the node's own query, key and value: from the staging rows
-                        const uint32_t row = sSt + (uint32_t)(slot * kStageRow + sub * 16);
-                        ld_shared_v4(row, qp.w);
-                        ld_shared_v4(row + 256, kq[0].w);
-                        ld_shared_v4(row + 512, vq[0].w);
+                    if constexpr (!WIDE) {
+                        Piece kq[NK], vq[NK], qp;
+                        int u[NK];
+                        const int cnt = valid ? __shfl_sync(gmask, pad, grp_base) : 1;
+                        u[0] = v;
+#pragma unroll
+                        for (int j = 1; j < MAXN; ++j) u[j] = __shfl_sync(gmask, pad, grp_base + j);
+                        if (valid) {
+#pragma unroll
+                            for (int j = 1; j < MAXN; ++j)
+                                if (j < cnt) vq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + 256 + sub * 16);
+#pragma unroll
+                            for (int j = 1; j < MAXN; ++j)
+                                if (j < cnt) kq[j] = ld_piece_cg(kv_tab + (size_t)u[j] * 512 + sub * 16);
+                        }
+                        if (tile == bid) issue_chains();
+                        if (pre_early) xpre = load_input(v_pre);                      // the next tile's input rows
+                        else if (tid == 32) misc->pre_ok = next_rows_ready();         // second look; read after the next barrier
+                        {   // the node's own query, key and value: from the staging rows
+                            const uint32_t row = sSt + (uint32_t)(slot * kStageRow + sub * 16);
+                            ld_shared_v4(row, qp.w);
+                            ld_shared_v4(row + 256, kq[0].w);
+                            ld_shared_v4(row + 512, vq[0].w);
+                        }
+                        attend<true, LPH, NK>(qp, kq, vq, cnt, p.scale, gmask, acc);
+                    } else {
+                        // cones wider than two hops: the node's list (CSR, the node itself included) is walked 16
+                        // entries at a time -- one entry per lane of the node's group -- with four neighbours' rows
+                        // in flight and an online softmax (running maximum and sum in log2 units, one rescale per
+                        // batch of four).  The node's own entry takes the key and value projected on chip.
+                        const int beg = valid ? __shfl_sync(gmask, pad, grp_base) : 0;
+                        const int cnt = valid ? __shfl_sync(gmask, pad, grp_base + 1) - beg : 0;
+                        if (tile == bid) issue_chains();
+                        if (pre_early) xpre = load_input(v_pre);
+                        else if (tid == 32) misc->pre_ok = next_rows_ready();
+                        Piece qp, k_own, v_own;
+                        {
+                            const uint32_t row = sSt + (uint32_t)(slot * kStageRow + sub * 16);
+                            ld_shared_v4(row, qp.w);
+                            ld_shared_v4(row + 256, k_own.w);
+                            ld_shared_v4(row + 512, v_own.w);
+                        }
+                        constexpr int UN = 4;
+                        const float c = p.scale * 1.4426950408889634f;
+                        const int parts = kTile / T_l, part = slot / T_l;      // replicas of a node, and which one this is
+                        float m = -INFINITY, z = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                        // Batches of UN entries; this replica takes batches part, part + parts, ...  A 16-lane load
+                        // brings the entries of four of its batches (one group), one group ahead of their use; the
+                        // rows of batch k+1 are requested before batch k is consumed.
+                        const int n_batches = (cnt + UN - 1) / UN;
+                        const int nb = part < n_batches ? (n_batches - part + parts - 1) / parts : 0;   // this replica's
+                        auto idx_group = [&](int j) -> int {
+                            const int pos = (part + (4 * j + (sub >> 2)) * parts) * UN + (sub & 3);
+                            return pos < cnt ? p.nbr_idx[beg + pos] : -1;
+                        };
+                        int g0 = nb > 0 ? idx_group(0) : -1, g1 = nb > 4 ? idx_group(1) : -1;
+                        auto issue = [&](int k, int* u, Piece* kq, Piece* vq) {
+                            const int j = k >> 2;
+                            if ((k & 3) == 0 && k > 0 && 4 * (j + 1) < nb) {       // entering group j: fetch group j+1
+                                if (j & 1) g0 = idx_group(j + 1); else g1 = idx_group(j + 1);
+                            }
+                            const int src = (j & 1) ? g1 : g0;
+#pragma unroll
+                            for (int i = 0; i < UN; ++i) u[i] = __shfl_sync(gmask, src, grp_base + (k & 3) * 4 + i);
+#pragma unroll
+                            for (int i = 0; i < UN; ++i) {
+                                if (u[i] >= 0 && u[i] != v) {
+                                    kq[i] = ld_piece_cg(kv_tab + (size_t)u[i] * 512 + sub * 16);
+                                    vq[i] = ld_piece_cg(kv_tab + (size_t)u[i] * 512 + 256 + sub * 16);
+                                }
+                            }
+                        };
+                        auto consume = [&](const int* u, Piece* kq, Piece* vq) {
+                            float sc[UN];
+#pragma unroll
+                            for (int i = 0; i < UN; ++i) {
+                                if (u[i] == v) { kq[i] = k_own; vq[i] = v_own; }
+                                float dot = (u[i] >= 0) ? Elem<true>::dot(qp, kq[i]) : 0.f;
+#pragma unroll
+                                for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(gmask, dot, o);
+                                sc[i] = (u[i] >= 0) ? dot * c : -INFINITY;
+                            }
+                            float m_new = m;
+#pragma unroll
+                            for (int i = 0; i < UN; ++i) m_new = fmaxf(m_new, sc[i]);
+                            const float keep = fast_exp2(m - m_new);            // 0 for the first batch (m = -inf)
+                            z *= keep;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[e] *= keep;
+#pragma unroll
+                            for (int i = 0; i < UN; ++i) {
+                                if (u[i] >= 0) {
+                                    const float pw = fast_exp2(sc[i] - m_new);
+                                    float vf[8];
+                                    Elem<true>::unpack(vq[i], vf);
+                                    z += pw;
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) acc[e] = fmaf(pw, vf[e], acc[e]);
+                                }
+                            }
+                            m = m_new;
+                        };
+                        {
+                            Piece kA[UN], vA[UN], kB[UN], vB[UN];
+                            int uA[UN], uB[UN];
+                            if (nb > 0) issue(0, uA, kA, vA);
+                            for (int k = 0; k < nb; k += 2) {
+                                if (k + 1 < nb) issue(k + 1, uB, kB, vB);
+                                consume(uA, kA, vA);
+                                if (k + 2 < nb) issue(k + 2, uA, kA, vA);
+                                if (k + 1 < nb) consume(uB, kB, vB);
+                            }
+                        }
+                        // merge the replicas' partial softmaxes into replica 0 (a replica that saw nothing has m = -inf)
+                        float* mine = reinterpret_cast<float*>(base_ptr + kOffMerge) + (size_t)tid * kMergeRow;
+                        mine[0] = m; mine[1] = z;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) mine[2 + e] = acc[e];
+                        worker_sync();
+                        if (part == 0) {
+                            for (int q = 1; q < parts; ++q) {
+                                const float* other = mine + (size_t)q * T_l * 16 * kMergeRow;
+                                const float m2 = other[0], z2 = other[1];
+                                if (m2 == -INFINITY) continue;
+                                const float mm = fmaxf(m, m2);
+                                const float w1 = fast_exp2(m - mm), w2 = fast_exp2(m2 - mm);
+                                z = z * w1 + z2 * w2;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) acc[e] = acc[e] * w1 + other[2 + e] * w2;
+                                m = mm;
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[e] = 0.f;           // a replica's row of the O tile is never used
+                            z = 1.f;
+                        }
+                        if (cnt == 1 && part == 0) {
+                            Elem<true>::unpack(v_own, acc);                     // softmax over one element: weight exactly 1
+                        } else if (cnt > 1 && part == 0) {
+                            const float inv = fast_rcp(z);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[e] *= inv;
+                        }
                     }
-                    attend<true, LPH, MAXN>(qp, kq, vq, cnt, p.scale, gmask, acc);
                     pad_nx = pad_of(v_nx);           // its node id has arrived by now; the entry is used by the next tile
                     {
                         Piece o = Elem<true>::pack(acc);
                         st_shared_v4(sO + operand_piece(slot, sub), o.w);
-                        if (sub == 0) misc->node[slot] = v;
+                        if (sub == 0) misc->node[slot] = (WIDE && slot / T_l != 0) ? -1 : v;   // replicas store nothing
                     }
                     worker_sync();
 
@@ -583,13 +734,14 @@ levelised_kernel(LevParams p) {
                         // prefetch has no destination register, so nothing ever waits for it).  Without this the
                         // index-chain loads and the neighbours' K | V rows of a large circuit come from DRAM, and
                         // that latency is on the level-to-level chain.
-                        const int r3 = bid * kTile + slot;
-                        if (sub == 0 && r3 < lp4 - lp3) prefetch_l2(p.level_nodes + lp3 + r3);     // node id, level l+3
+                        const int t3 = per_tile(lp4 - lp3, nctas);
+                        const int r3 = bid * t3 + slot;
+                        if (sub == 0 && slot < t3 && r3 < lp4 - lp3) prefetch_l2(p.level_nodes + lp3 + r3);   // node ids, level l+3
                         if (vB >= 0) {                                                            // level l+2's node
-                            if (sub == 0) prefetch_l2(p.nbr_pad + (size_t)vB * W);
+                            if (sub == 0) prefetch_l2(WIDE ? (const void*)(p.nbr_ptr + vB) : (const void*)(p.nbr_pad + (size_t)vB * W));
                             if ((sub & 1) == 0) prefetch_l2((const char*)p.H + (size_t)vB * p.ldh * 2 + sub * 16);
                         }
-                        if (vC >= 0) {                                                            // level l+1's node
+                        if (!WIDE && vC >= 0) {                                                   // level l+1's node
                             const int cnt_c = __shfl_sync(gmask, padC, grp_base);
 #pragma unroll
                             for (int j = 1; j < MAXN; ++j) {
@@ -639,7 +791,7 @@ levelised_kernel(LevParams p) {
                 // ---- no tile in this level but one in the next: bring that tile up while there is nothing else to do
                 if (tid == 32) {
                     bool go = true;
-                    if (prev_arrive) go = wait_counter(prev_arrive + l + 1, prev_target(tiles_next), p.abort_word, counter_limit);
+                    if (prev_arrive) go = wait_counter(prev_arrive + l + 1, prev_target(lp2 - lp1), p.abort_word, counter_limit);
                     if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                     misc->go2 = go ? 1 : 0;
                 }
@@ -736,11 +888,13 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     }
     DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, n_layers), st));
     p.H = H; p.ldh = ldh;
-    p.nbr_pad = g->nbr_pad; p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
+    p.nbr_pad = g->nbr_pad; p.nbr_ptr = g->nbr_ptr; p.nbr_idx = g->nbr_idx;
+    p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
     p.n_levels = g->n_levels; p.n_layers = n_layers;
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status; p.poll_limit = dg4i_poll_limit();
     const int grid = g_sm_count[dev];
+    if (g->wide) return launch_heads<0>(desc->heads, p, grid, st);
     if (g->max_class <= 3) return launch_heads<3>(desc->heads, p, grid, st);
     return launch_heads<7>(desc->heads, p, grid, st);
 }

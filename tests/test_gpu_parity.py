@@ -501,35 +501,49 @@ def test_wide_cone_attention_matches_checker(dtype, hops, heads):
         assert rel_row_err(got, want).max() <= BF16_ROW_TOL
 
 
-def test_wide_cone_layers_parallel_and_level_launches():
-    rng = np.random.default_rng(31)
+@pytest.mark.parametrize("hops,heads", [(4, 8), (8, 8), (3, 1), (6, 16)])
+def test_wide_cone_layers_in_every_order(hops, heads):
+    """Cones of 3 to 8 hops through the layer calls: all nodes at once, level by level with one launch group per
+    level, level by level in the persistent kernel (which walks the cone lists with an online softmax), and two
+    layers as a wavefront."""
+    rng = np.random.default_rng(31 + hops)
     fanins = random_dag(rng, 30, 2500, window=60)
     rp, ci = csr_from_fanins(fanins)
     level = levels_of(fanins)
-    n, hops, heads = len(fanins), 4, 8
+    n = len(fanins)
+    scale = 1.0 / np.sqrt(128 // heads)
     gr = dg4.dg4_graph_create(rp, ci, level, hops, 0)
     xb = synth.normal_bf16_bits(8, 1, (n, 128), 1.0)
-    wqb, wq = bf16_weights(synth.normal_f32(8, 2, (384, 128), 0.05))
-    wob, wo = bf16_weights(synth.normal_f32(8, 3, (128, 128), 0.05))
+    weights = [bf16_weights(synth.normal_f32(8, 2 + 2 * l, (384, 128), 0.05)) +
+               bf16_weights(synth.normal_f32(8, 3 + 2 * l, (128, 128), 0.05)) for l in range(2)]
+    (wqb, wq, wob, wo) = weights[0]
     ptr, idx = orc.neighbourhood(rp, ci, hops)
     lptr, lnodes = orc.level_buckets(level)
-    for mode in ("parallel", "level-launches"):
-        dsc = dg4.desc(heads, dg4.DG4_BF16, 0.25, residual=True, level_launches=(mode == "level-launches"))
-        ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    want_par = orc.layer_parallel(f64_of_bits(xb), wq, wo, ptr, idx, heads, scale, residual=True, rounding="bf16")
+    want_lev = orc.layer_levelised(f64_of_bits(xb), wq, wo, ptr, idx, lptr, lnodes, heads, scale, residual=True,
+                                   rounding="bf16")
+    want_lev2 = orc.layer_levelised(want_lev, weights[1][1], weights[1][3], ptr, idx, lptr, lnodes, heads, scale,
+                                    residual=True, rounding="bf16")
+    for mode in ("parallel", "level-launches", "persistent", "wavefront"):
+        dsc = dg4.desc(heads, dg4.DG4_BF16, scale, residual=True, level_launches=(mode == "level-launches"))
+        ws = torch.empty(max(dg4.dg4_layer_workspace_bytes(gr, dsc), dg4.dg4_layers_workspace_bytes(gr, dsc, 2)),
+                         dtype=torch.uint8, device="cuda")
         h = dev_bf16(xb).clone()
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
         if mode == "parallel":
             dg4.dg4_layer_fwd_parallel(gr, dsc, h, dev_bf16(wqb), dev_bf16(wob), h, ws)
-            want = orc.layer_parallel(f64_of_bits(xb), wq, wo, ptr, idx, heads, 0.25, residual=True, rounding="bf16")
+            want = want_par
+        elif mode == "wavefront":
+            dg4.dg4_layers_fwd_levelised(gr, dsc, h, [dev_bf16(w_[0]) for w_ in weights],
+                                         [dev_bf16(w_[2]) for w_ in weights], ws, status)
+            want = want_lev2
         else:
-            dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wqb), dev_bf16(wob), ws)
-            want = orc.layer_levelised(f64_of_bits(xb), wq, wo, ptr, idx, lptr, lnodes, heads, 0.25, residual=True,
-                                       rounding="bf16")
+            dg4.dg4_layer_fwd_levelised(gr, dsc, h, dev_bf16(wqb), dev_bf16(wob), ws, status)
+            want = want_lev
         torch.cuda.synchronize()
-        assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL, mode
-    # the persistent level kernel holds at most 7 neighbours in registers: wider cones are refused, not mangled
-    with pytest.raises(dg4.Dg4Error) as e:
-        dg4.dg4_layer_fwd_levelised(gr, dg4.desc(heads, dg4.DG4_BF16, 0.25), h, dev_bf16(wqb), dev_bf16(wob), ws)
-    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+        assert int(status.item()) == 0 and dg4.dg4_graph_poll_status(gr) == 0, mode
+        err = rel_row_err(host_f64_of_bf16(h), want)
+        assert err.max() <= BF16_ROW_TOL, (mode, err.max(), int(err.argmax()))
 
 
 @pytest.mark.parametrize("hops,delta", [(8, 6), (3, 2), (2, 1), (1, 1)])
