@@ -33,7 +33,10 @@
 // occupies the issuing thread for about as long as the tensor pipe needs to execute it, so a worker thread that
 // issued the next tile's 24 instructions would hold up its own warp's epilogue (and with it the level) for their
 // whole duration.  The workers hand the issuing thread one order at a time (a word in shared memory and an
-// mbarrier arrival) and wait only for the completion barrier of the product they need next.
+// mbarrier arrival) and wait only for the completion barrier of the product they need next.  Both sides wait
+// suspended (try_wait with a time hint) rather than polling: a polling warp takes issue slots from the warp that
+// shares its scheduler -- from the issuing thread while the workers wait for its product, from the workers'
+// attention while the issuing thread waits for an order (measured: 2 % of the whole sweep).
 //
 // Cones wider than two hops (MAXN = 0) come as lists instead of the fixed-width table: step 1 then walks a node's
 // list in batches of four entries with an online softmax, two batches in flight.  A tile's time is then the serial
@@ -316,7 +319,7 @@ levelised_kernel(LevParams p) {
             uint32_t phc = 0;
             int strikes = 0;
             for (;;) {
-                if (!mbar_wait(cmd_bar, phc, p.poll_limit)) {
+                if (!mbar_wait_relaxed(cmd_bar, phc, p.poll_limit)) {
                     // no order for a long time: normal while the CTA idles through levels in which it has no tile,
                     // unless the run was aborted meanwhile; a bound on the total keeps even that wait finite
                     if (ld_acquire(p.abort_word) != 0) break;
@@ -469,7 +472,7 @@ levelised_kernel(LevParams p) {
                     // ---- this tile's own Q | K | V: read from tensor memory if the product was issued during the
                     // tile before, else brought up from scratch below (after the counters)
                     auto epilogue_qkv = [&]() {
-                        if (!mbar_wait(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                        if (!mbar_wait_relaxed(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                         ph0 ^= 1u;
                         tc_fence_after();
                         uint32_t d[3][8];
@@ -750,7 +753,7 @@ levelised_kernel(LevParams p) {
                             }
                         }
                     }
-                    if (!mbar_wait(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
                     tc_fence_after();
                     {
