@@ -177,7 +177,9 @@ __global__ void __launch_bounds__(DG4_ATTN_THREADS, DG4_ATTN_MIN_BLOCKS) sparse_
 // keeps an online softmax (running maximum and sum, in log2 units) over the neighbours its half has seen and the
 // matching weighted sum of its value piece; the halves are merged at the end.  Four neighbours per half are in
 // flight at a time.
-template <bool BF16, int LPH>
+// ADDITIVE: scores are LeakyReLU(S_src[u, head] + S_dst[v, head]) from node-level scalars instead of q . k (no
+// query or key rows are read).
+template <bool BF16, int LPH, bool ADDITIVE>
 __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_kernel(dg4i_attn_args a, dg4i_attn_more x) {
     constexpr int G = BF16 ? 16 : 32;              // lanes per row
     constexpr int HALVES = 32 / G;                 // neighbours a warp handles side by side
@@ -195,7 +197,10 @@ __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_ker
         const int v = a.node_list ? a.node_list[a.first + slot] : a.first + slot;
         const int beg = x.nbr_ptr[v];
         const int cnt = x.nbr_ptr[v + 1] - beg;
-        const Piece qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
+        Piece qp;
+        float sd = 0.f;
+        if (ADDITIVE) sd = __ldg(x.s_dst + (size_t)v * a.heads + sub / LPH);
+        else qp = ld_piece_stream((const char*)a.Q + (size_t)v * a.ldq * ES + col);
         float m = -INFINITY, z = 0.f, acc[EPP];
 #pragma unroll
         for (int i = 0; i < EPP; ++i) acc[i] = 0.f;
@@ -214,7 +219,8 @@ __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_ker
 #pragma unroll
                 for (int i = 0; i < UN; ++i) {
                     if (u[i] >= 0) {
-                        kq[i] = ld_piece_nc((const char*)a.K + (size_t)u[i] * a.ldk * ES + col);
+                        if (ADDITIVE) kq[i].w[0] = __float_as_uint(__ldg(x.s_src + (size_t)u[i] * a.heads + sub / LPH));
+                        else kq[i] = ld_piece_nc((const char*)a.K + (size_t)u[i] * a.ldk * ES + col);
                         vq[i] = ld_piece_nc((const char*)a.V + (size_t)u[i] * a.ldv * ES + col);
                     }
                 }
@@ -223,10 +229,16 @@ __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_ker
                 float s[UN];
 #pragma unroll
                 for (int i = 0; i < UN; ++i) {
-                    float dot = (u[i] >= 0) ? Elem<BF16>::dot(qp, kq[i]) : 0.f;
+                    if (ADDITIVE) {
+                        float e = __uint_as_float(kq[i].w[0]) + sd;
+                        e = (e > 0.f ? e : x.slope * e) * 1.4426950408889634f;
+                        s[i] = (u[i] >= 0) ? e : -INFINITY;
+                    } else {
+                        float dot = (u[i] >= 0) ? Elem<BF16>::dot(qp, kq[i]) : 0.f;
 #pragma unroll
-                    for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(hmask, dot, o);
-                    s[i] = (u[i] >= 0) ? dot * c : -INFINITY;
+                        for (int o = LPH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(hmask, dot, o);
+                        s[i] = (u[i] >= 0) ? dot * c : -INFINITY;
+                    }
                 }
                 float m_new = m;
 #pragma unroll
@@ -276,29 +288,29 @@ __global__ void __launch_bounds__(256, DG4_WIDE_MIN_BLOCKS) sparse_attn_wide_ker
     }
 }
 
-template <bool BF16, int LPH>
+template <bool BF16, int LPH, bool ADDITIVE>
 dg4_status launch_wide(const dg4i_attn_args& a, const dg4i_attn_more& x, cudaStream_t st) {
     int dev = 0, sms = 0;
     DG4_CUDA_TRY(cudaGetDevice(&dev));
     DG4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int64_t needed = ((int64_t)a.count + 7) / 8;
     const int64_t resident = (int64_t)sms * DG4_WIDE_MIN_BLOCKS;
-    sparse_attn_wide_kernel<BF16, LPH><<<(unsigned)(needed < resident ? needed : resident), 256, 0, st>>>(a, x);
+    sparse_attn_wide_kernel<BF16, LPH, ADDITIVE><<<(unsigned)(needed < resident ? needed : resident), 256, 0, st>>>(a, x);
     dg4i_count_launch();
     DG4_CUDA_TRY(cudaGetLastError());
     return DG4_OK;
 }
 
-template <bool BF16>
+template <bool BF16, bool ADDITIVE>
 dg4_status launch_wide_heads(const dg4i_attn_args& a, const dg4i_attn_more& x, cudaStream_t st) {
     constexpr int G = BF16 ? 16 : 32;
     switch (G / a.heads) {
-        case 1: return launch_wide<BF16, 1>(a, x, st);
-        case 2: return launch_wide<BF16, 2>(a, x, st);
-        case 4: return launch_wide<BF16, 4>(a, x, st);
-        case 8: return launch_wide<BF16, 8>(a, x, st);
-        case 16: return launch_wide<BF16, 16>(a, x, st);
-        case 32: if (G == 32) return launch_wide<BF16, (G == 32 ? 32 : 16)>(a, x, st);
+        case 1: return launch_wide<BF16, 1, ADDITIVE>(a, x, st);
+        case 2: return launch_wide<BF16, 2, ADDITIVE>(a, x, st);
+        case 4: return launch_wide<BF16, 4, ADDITIVE>(a, x, st);
+        case 8: return launch_wide<BF16, 8, ADDITIVE>(a, x, st);
+        case 16: return launch_wide<BF16, 16, ADDITIVE>(a, x, st);
+        case 32: if (G == 32) return launch_wide<BF16, (G == 32 ? 32 : 16), ADDITIVE>(a, x, st);
     }
     DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d is not supported for this dtype", a.heads);
 }
@@ -357,9 +369,8 @@ dg4_status attn_dispatch(const dg4i_attn_args& a, const dg4i_attn_more* x, cudaS
     if (a.heads < 1 || a.heads > G || (G % a.heads) != 0)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "heads = %d: must divide %d", a.heads, G);
     if (a.max_nbr > 7) {
-        if (ADDITIVE) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the additive-score variant supports cones of at most two hops");
         if (!x || !x->nbr_ptr || !x->nbr_idx) DG4_FAIL(DG4_ERR_INVALID_ARG, "wider cones need the CSR neighbour lists");
-        return bf16 ? launch_wide_heads<true>(a, *x, st) : launch_wide_heads<false>(a, *x, st);
+        return bf16 ? launch_wide_heads<true, ADDITIVE>(a, *x, st) : launch_wide_heads<false, ADDITIVE>(a, *x, st);
     }
     if (a.max_nbr <= 3) return bf16 ? launch_for_heads<true, 3, ADDITIVE>(a, x, st) : launch_for_heads<false, 3, ADDITIVE>(a, x, st);
     return bf16 ? launch_for_heads<true, 7, ADDITIVE>(a, x, st) : launch_for_heads<false, 7, ADDITIVE>(a, x, st);

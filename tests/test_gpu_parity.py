@@ -431,7 +431,8 @@ def test_layers_other_head_counts_and_no_residual(hops, heads, residual, mode):
 
 
 @pytest.mark.parametrize("dtype,hops,heads", [("f32", 1, 4), ("f32", 2, 8), ("bf16", 2, 8), ("bf16", 1, 1),
-                                              ("bf16", 2, 16), ("f32", 2, 32)])
+                                              ("bf16", 2, 16), ("f32", 2, 32),
+                                              ("bf16", 4, 8), ("bf16", 8, 2), ("f32", 5, 4), ("f32", 8, 32)])
 def test_additive_score_attention_matches_checker(dtype, hops, heads):
     rng = np.random.default_rng(7000 + heads + hops)
     fanins = random_dag(rng, 40, 5000, window=200)
