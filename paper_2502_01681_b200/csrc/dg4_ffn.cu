@@ -669,6 +669,18 @@ extern "C" dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc
     __nv_bfloat16* Q = (__nv_bfloat16*)workspace;
     __nv_bfloat16* KV = Q + (size_t)g->n * 128;
     __nv_bfloat16* O = Q + (size_t)g->n * 384;
+    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES) && !g->wide &&
+        (size_t)g->n * 256 >= dg4i_levelised_sync_bytes(g, 2)) {
+        // one persistent kernel: attention-stage and feed-forward-stage CTAs hand the levels to one another (the
+        // counters live where the launch-group driver keeps its Q table, which this path does not need)
+        dg4i_block_tail tail;
+        tail.ln1_gamma = ln1_gamma; tail.ln1_beta = ln1_beta; tail.W1 = (const __nv_bfloat16*)W1; tail.b1 = b1;
+        tail.W2 = (const __nv_bfloat16*)W2; tail.b2 = b2; tail.ln2_gamma = ln2_gamma; tail.ln2_beta = ln2_beta; tail.eps = eps;
+        __nv_bfloat16* kv1[1] = {KV};
+        const __nv_bfloat16* wq1[1] = {(const __nv_bfloat16*)W_qkv};
+        const __nv_bfloat16* wo1[1] = {(const __nv_bfloat16*)W_o};
+        return dg4i_levelised_launch(g, desc, 1, kv1, Hb, ldh, wq1, wo1, (int32_t*)workspace, g->dev_status, st, &tail);
+    }
     // Q | K | V of every node from the block's input: a node's own query, key and value never change
     CHECK(dg4_qkv_project(g, desc, H, ldh, W_qkv, Q, 128, KV, 256, KV + 128, 256, stream));
     const __nv_bfloat16* W_kv = (const __nv_bfloat16*)W_qkv + (size_t)128 * 128;

@@ -151,7 +151,17 @@ dg4_status dg4i_fused_layer_launch(const dg4_graph* g, const dg4_desc* desc, con
 // by the call and must hold dg4i_levelised_sync_bytes() bytes.
 #define DG4I_MAX_LAYERS 8
 size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers);
+// With `block` (one layer, cones of at most two hops): the whole Transformer block level by level -- half of the
+// CTAs run the attention sub-layer of each level, the other half its LayerNorm, feed-forward sub-layer, LayerNorm
+// and the K | V refresh from the block's output rows.  `sync` then holds dg4i_levelised_sync_bytes(g, 2) bytes.
+struct dg4i_block_tail {
+    const float* ln1_gamma; const float* ln1_beta;
+    const __nv_bfloat16* W1; const float* b1;          // [512, 128], [512]
+    const __nv_bfloat16* W2; const float* b2;          // [128, 512], [128]
+    const float* ln2_gamma; const float* ln2_beta;
+    float eps;
+};
 dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers,
                                  __nv_bfloat16* const* KV, __nv_bfloat16* H, int64_t ldh,
                                  const __nv_bfloat16* const* W_qkv, const __nv_bfloat16* const* W_o, int32_t* sync,
-                                 int32_t* status, cudaStream_t st);
+                                 int32_t* status, cudaStream_t st, const dg4i_block_tail* block = nullptr);

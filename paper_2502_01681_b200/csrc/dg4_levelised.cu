@@ -43,6 +43,13 @@
 // walk of its longest list, so narrow levels are spread over all of the layer's CTAs and the slots a tile has
 // left over take replicas of its nodes, each walking a share of the list; the shares are merged in shared memory.
 //
+// The whole Transformer block level by level (block mode, Sec. 3.5 with the order of Sec. 1 / Sec. 3.4): the CTAs are
+// dealt alternately to an attention stage -- the tile described above without step 4 -- and a feed-forward stage,
+// which keeps W1 in tensor memory and W2 in shared memory and turns the attention stage's rows of a level into
+// the block's output rows (LayerNorm, two transposed products with bias / ReLU between them, residual, LayerNorm)
+// and refreshes the level's K | V rows from THOSE.  The two stages hand each level to one another through the
+// same counters the layers of a wavefront use.
+//
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
 // to layers round-robin; each keeps its layer's W_k, W_v and W_q resident in TENSOR memory (blocks of 128 lanes
@@ -78,7 +85,10 @@ constexpr int kBHalf = kTile * 128;          // K-half of a kTile-row operand ti
 constexpr int kTileOp = 2 * kBHalf;          // a kTile x 128 bf16 tile in operand layout (4 KiB)
 constexpr int kTmemCols = 512;
 constexpr int kAccK2 = 1, kAccV2 = 2, kAccQ = 3, kAccK = 4, kAccV = 5;   // accumulators of kTile columns (slot 0 unused)
-constexpr int kWCol0 = 6 * kTile;            // first column of the weight blocks ( - | W_k | W_v | W_q )
+constexpr int kWCol0 = 64;                   // weight blocks at kWCol0 + blk * 64: W_k at 128, W_v at 192, W_q at 256
+// a CTA that runs the feed-forward stage of the block instead keeps W1 where W_q would be (four blocks from column
+// 256) and has its own accumulators beside K2 | V2: the four hidden blocks and the second product
+constexpr int kColW1 = 256, kColD1 = 3 * kTile, kColD2 = 7 * kTile;
 constexpr int kWCols = 64;                   // a 128 x 128 bf16 block: 128 lanes x 64 columns of two elements
 constexpr int kBlkK = 1, kBlkV = 2, kBlkQ = 3;            // weight blocks in tensor memory (slot 0 unused)
 constexpr int kStageRow = 768 + 16;          // staging per node: Q 256 | K 256 | V 256 (+ padding against bank conflicts)
@@ -89,23 +99,26 @@ constexpr int kOffX = kOffHp + kTileOp;                // input rows of the curr
 constexpr int kOffHres = kOffX + 2 * kTileOp;          // the same rows, plain [kTile][256 B], twice
 constexpr int kOffStage = kOffHres + 2 * kTile * 256;  // staging, plain [kTile][kStageRow]
 constexpr int kOffMerge = kOffStage + kTile * kStageRow;        // wide cones: partial softmaxes of a node's replicas
-constexpr int kOffMisc = kOffMerge + kWorkers * kMergeRow * 4;
+constexpr int kOffAct = ((kOffMerge + kWorkers * kMergeRow * 4 + 1023) / 1024) * 1024;   // feed-forward stage: hidden activations, 4 tiles
+constexpr int kOffS32 = kOffAct + 4 * kTileOp;                  // feed-forward stage: second product in fp32, [kTile][128]
+constexpr int kOffMisc = kOffS32 + kTile * 128 * 4;
 constexpr int kWHalf = 128 * 128;                      // K-half of a 128-row weight block: 128 rows x 128 bytes
 constexpr int kWBlock = 2 * kWHalf;                    // a 128 x 128 bf16 block in shared memory (32 KiB)
-constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o for the warp-level output projection
-constexpr int kSmemBytes = kOffWs + kWBlock + 1024;
+constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o for the warp-level output projection; W2 (4 blocks) in a feed-forward CTA
+constexpr int kSmemBytes = kOffWs + 4 * kWBlock + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-static_assert(kWCol0 + 4 * kWCols <= kTmemCols, "tensor memory budget of one CTA");
+static_assert(kWCol0 + 4 * kWCols <= kTmemCols && kColW1 + 4 * kWCols <= kTmemCols && 6 * kTile <= kWCol0 + kWCols &&
+              kColD2 + kTile <= kWCol0 + kWCols, "tensor memory budget of one CTA");
 static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) == 0, "operand tiles are 1024-byte aligned");
 // Every CTA allocates all of its SM's tensor memory, so two CTAs must never share an SM (the second one's
 // allocation would wait for the first, which waits for the second's levels): the launch asks for more than half
 // of an SM's shared memory, which rules that out.
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
 
-enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdKv = 2, kCmdKvThenQkv = 3 };
+enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdKv = 2, kCmdKvThenQkv = 3, kCmdFfn1 = 4, kCmdFfn2 = 5 };
 
 struct Misc {
-    uint64_t mma0, mma2, drain;
+    uint64_t mma0, mma1, mma2, drain;
     uint64_t cmd_bar;                      // the workers' next order for the issuing thread is in `cmd`
     int32_t cmd, cmd_buf;
     uint32_t tmem_base;
@@ -135,6 +148,17 @@ struct LevParams {
     int32_t* abort_word;                   // zero on entry
     int32_t* status;
     uint32_t poll_limit;                   // polls after which a wait gives up
+    // The whole Transformer block level by level (block != 0, n_layers == 2): the CTAs of "layer" 0 run the
+    // attention sub-layer of a level, those of "layer" 1 its LayerNorm, feed-forward sub-layer, LayerNorm and the
+    // K | V refresh from the block's output rows; the two hand each level to one another through the counters.
+    int32_t block;
+    float eps;
+    const float* ln1_gamma; const float* ln1_beta;
+    const __nv_bfloat16* W1;               // [512, 128]
+    const float* b1;                       // [512]
+    const __nv_bfloat16* W2;               // [128, 512]
+    const float* b2;                       // [128]
+    const float* ln2_gamma; const float* ln2_beta;
 };
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
@@ -248,6 +272,7 @@ levelised_kernel(LevParams p) {
     if (tid == 0) {
         mbar_init(bar0, 1);
         mbar_init(bar2, 1);
+        mbar_init(smem_u32(&misc->mma1), 1);
         mbar_init(smem_u32(&misc->drain), 1);
         mbar_init(smem_u32(&misc->cmd_bar), 1);
         misc->cmd = kCmdExit;
@@ -271,7 +296,30 @@ levelised_kernel(LevParams p) {
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
-    if (warp < 8) {
+    const bool ffn_stage = p.block != 0 && layer == 1;
+    if (warp < 8 && ffn_stage) {
+        // W_k, W_v as everywhere; W1's four blocks of 128 hidden units in tensor memory; W2 in shared memory as
+        // four 128 x 128 blocks (block c = hidden units 128c .. 128c+127) in the swizzled K-major layout
+        for (int blk = 1; blk <= 6; ++blk) {
+            const __nv_bfloat16* wb = blk <= 2 ? p.Wqkv[layer] + (size_t)blk * 128 * 128 : p.W1 + (size_t)(blk - 3) * 128 * 128;
+            const uint32_t col0 = blk <= 2 ? (uint32_t)(kWCol0 + blk * kWCols) : (uint32_t)(kColW1 + (blk - 3) * kWCols);
+            const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint4 lo = src[2 * c], hi = src[2 * c + 1];
+                const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                tmem_st_32x8(tmem + lane_base + col0 + (uint32_t)(cg * 32 + c * 8), r);
+            }
+        }
+        tmem_st_wait();
+        for (int i = tid; i < 4 * 128 * 16; i += kWorkers) {
+            const int c = i >> 11, row = (i >> 4) & 127, chunk = i & 15;
+            const uint4 v = *reinterpret_cast<const uint4*>(p.W2 + (size_t)row * 512 + c * 128 + chunk * 8);
+            const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+            st_shared_v4(sW + (uint32_t)(c * kWBlock) + weight_piece(row, chunk), r);
+        }
+        fence_proxy_async_smem();
+    } else if (warp < 8) {
         for (int blk = kBlkK; blk <= kBlkQ; ++blk) {
             const __nv_bfloat16* wb = blk == kBlkQ ? p.Wqkv[layer]
                                                     : p.Wqkv[layer] + (size_t)blk * 128 * 128;     // kBlkK = 1, kBlkV = 2
@@ -333,6 +381,29 @@ levelised_kernel(LevParams p) {
                 if (cmd == kCmdExit) break;
                 if (cmd == kCmdQkv) {
                     issue_qkv(b);
+                } else if (cmd == kCmdFfn1) {
+                    // hidden^T = W1 * Y1^T, four blocks of 128 hidden units (rows in input buffer 0)
+                    tc_fence_after();
+#pragma unroll
+                    for (int blk = 0; blk < 4; ++blk)
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t b_off = (uint32_t)((ks >> 2) * kBHalf + (ks & 3) * 32);
+                            mma_bf16_ta(tmem + (uint32_t)(kColD1 + blk * kTile), tmem + (uint32_t)(kColW1 + blk * kWCols + ks * 8), dX[0] + (b_off >> 4), idesc, ks > 0 ? 1u : 0u);
+                        }
+                    mma_commit(bar0);
+                } else if (cmd == kCmdFfn2) {
+                    // out^T = W2 * act^T: W2's block c from shared memory as the A operand, the activation tile c as B
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint32_t a_off = (uint32_t)(c * kWBlock + (ks >> 2) * kWHalf + (ks & 3) * 32);
+                            const uint32_t b_off = (uint32_t)(c * kTileOp + (ks >> 2) * kBHalf + (ks & 3) * 32);
+                            mma_bf16(tmem + (uint32_t)kColD2, smem_desc_sw128(sW + a_off), smem_desc_sw128(base + kOffAct + b_off), idesc, (c > 0 || ks > 0) ? 1u : 0u);
+                        }
+                    mma_commit(smem_u32(&misc->mma1));
                 } else {
                     // from the new rows, transposed: this layer's K | V refresh; right behind it, if ordered, the next
                     // tile's Q | K | V (it runs while this tile's rows are stored and the level completes)
@@ -366,7 +437,7 @@ levelised_kernel(LevParams p) {
         const int mg = lane >> 2, mt = lane & 3;
         const int a_row = lane & 15, a_chunk = lane >> 4;                       // A fragments: the 16-node tile
         const int b_row = (lane & 7) + ((lane >> 4) << 3), b_chunk = (lane >> 3) & 1;   // B fragments: 16 weight rows
-        int last_nonempty = -1, last_participants = 0;
+        int last_nonempty = -1, last_participants = 0, last_participants_ffn = 0;
         bool alive = true;
         const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
 
@@ -422,6 +493,159 @@ levelised_kernel(LevParams p) {
         int pad0 = pad_of(v0);
         int vC = stage_node(lp1, lp2);                     // level l+1: node id
 
+        if (ffn_stage) {
+            // ------------------------------------------------------------ a block's feed-forward stage
+            // Per tile of 16 nodes of a level whose attention stage has arrived: rows a (attention sub-layer output)
+            // -> LayerNorm -> y1 (bf16) -> hidden^T = W1 y1^T (four blocks) -> + b1, ReLU, bf16 -> out^T = W2 act^T
+            // -> + b2 + y1 -> LayerNorm -> block output rows (bf16) to H -> K | V refresh from them -> arrive.
+            // Lanes own 8 features of a node in the row-wise parts and one feature (hidden unit) of 8 nodes in the
+            // epilogues that read tensor memory; the two views meet in shared memory.
+            const uint32_t bar1 = smem_u32(&misc->mma1);
+            const uint32_t sAct = base + kOffAct, sS32 = base + kOffS32;
+            uint32_t ph1 = 0;
+            float g1[8], be1[8], g2[8], be2[8], bo[8], bh[4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                g1[i] = __ldg(p.ln1_gamma + sub * 8 + i); be1[i] = __ldg(p.ln1_beta + sub * 8 + i);
+                g2[i] = __ldg(p.ln2_gamma + sub * 8 + i); be2[i] = __ldg(p.ln2_beta + sub * 8 + i);
+                bo[i] = __ldg(p.b2 + sub * 8 + i);
+            }
+#pragma unroll
+            for (int blk = 0; blk < 4; ++blk) bh[blk] = __ldg(p.b1 + blk * 128 + feat);
+            auto layer_norm = [&](float* x, const float* g, const float* b) {     // over the node's 128 features (16 lanes)
+                float sum = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sum += x[i];
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(gmask, sum, o);
+                const float mean = sum * (1.0f / 128.0f);
+                float sq = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { x[i] -= mean; sq += x[i] * x[i]; }
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(gmask, sq, o);
+                const float rstd = rsqrtf(sq * (1.0f / 128.0f) + p.eps);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) x[i] = x[i] * rstd * g[i] + b[i];
+            };
+            for (int l = 0; l < p.n_levels && alive; ++l) {
+                const int first = p.level_ptr[l];
+                const int n_l = p.level_ptr[l + 1] - first;
+                const int tiles = (n_l + kTile - 1) / kTile;
+                if (n_l <= 0 || bid >= tiles) continue;
+                bool waited = false;
+                for (int tile = bid; tile < tiles; tile += nctas) {
+                    const int r = tile * kTile + slot;
+                    const int v = r < n_l ? p.level_nodes[first + r] : -1;
+                    if (!waited) {                     // the attention stage has stored this level's rows
+                        if (tid == 0) {
+                            bool go = misc->failed == 0;
+                            if (go) go = wait_counter(prev_arrive + l, prev_target(n_l), p.abort_word, counter_limit);
+                            if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                            misc->go = go ? 1 : 0;
+                        }
+                        worker_sync();
+                        waited = true;
+                        if (!misc->go) { alive = false; break; }
+                    }
+                    // ---- first LayerNorm, rows into the operand tile
+                    float x[8];
+                    {
+                        const Piece a = load_input(v);
+                        Elem<true>::unpack(a, x);
+                    }
+                    layer_norm(x, g1, be1);
+                    const Piece y1 = Elem<true>::pack(x);
+                    st_shared_v4(sX + operand_piece(slot, sub), y1.w);
+                    if (sub == 0) misc->node[slot] = v;
+                    fence_proxy_async_smem();
+                    worker_sync();
+                    if (tid == 0) post(kCmdFfn1, 0);
+                    // ---- hidden units: + b1, ReLU, bf16, into the four activation tiles (operand layout)
+                    if (!mbar_wait_relaxed(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph0 ^= 1u;
+                    tc_fence_after();
+#pragma unroll
+                    for (int blk = 0; blk < 4; ++blk) {
+                        uint32_t d[8];
+                        tmem_ld_32x8(tmem + lane_base + (uint32_t)(kColD1 + blk * kTile + cg * 8), d);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int nn = 0; nn < 8; ++nn) {
+                            const float hval = fmaxf(__uint_as_float(d[nn]) + bh[blk], 0.f);
+                            st_shared_b16(sAct + (uint32_t)(blk * kTileOp) + operand_offset(cg * 8 + nn, feat), bf16_bits(hval));
+                        }
+                    }
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    worker_sync();
+                    if (tid == 0) post(kCmdFfn2, 0);
+                    // ---- second product out of tensor memory into [node][feature] fp32
+                    if (!mbar_wait_relaxed(bar1, ph1, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph1 ^= 1u;
+                    tc_fence_after();
+                    {
+                        uint32_t d[8];
+                        tmem_ld_32x8(tmem + lane_base + (uint32_t)(kColD2 + cg * 8), d);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int nn = 0; nn < 8; ++nn) st_shared_b32(sS32 + (uint32_t)(((cg * 8 + nn) * 128 + feat) * 4), d[nn]);
+                    }
+                    tc_fence_before();
+                    worker_sync();
+                    // ---- + b2 + y1, second LayerNorm, the block's output rows
+                    {
+                        uint32_t w8[8];
+                        ld_shared_v4(sS32 + (uint32_t)((slot * 128 + sub * 8) * 4), w8);
+                        ld_shared_v4(sS32 + (uint32_t)((slot * 128 + sub * 8 + 4) * 4), w8 + 4);
+                        float y[8];
+                        Elem<true>::unpack(y1, y);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(w8[i]) + bo[i] + y[i];
+                    }
+                    layer_norm(x, g2, be2);
+                    const Piece out = Elem<true>::pack(x);
+                    if (v >= 0) st_global_v4((char*)p.H + (size_t)v * p.ldh * 2 + sub * 16, out.w);
+                    st_shared_v4(sHp + operand_piece(slot, sub), out.w);
+                    fence_proxy_async_smem();
+                    worker_sync();
+                    // ---- K | V of the new rows into the table
+                    if (tid == 0) post(kCmdKv, 0);
+                    if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                    ph2 ^= 1u;
+                    tc_fence_after();
+                    {
+                        uint32_t d[2][8];
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk)
+                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int blk = 0; blk < 2; ++blk) {
+                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
+#pragma unroll
+                            for (int nn = 0; nn < 8; ++nn)
+                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
+                        }
+                    }
+                    tc_fence_before();
+                    worker_sync();
+                    if (v >= 0) {
+                        const uint32_t row = sSt + (uint32_t)(slot * kStageRow);
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
+                            st_global_v4((char*)p.KV[layer] + (size_t)v * 512 + (sub + 16 * h) * 16, w4);
+                        }
+                    }
+                    worker_sync();
+                }
+                if (!alive) break;
+                if (tid == 64) red_release_add(my_arrive + l, 1);
+            }
+            if (tid == 0) post(kCmdExit, 0);
+        } else {
         bool pro_ready = false;      // the Q | K | V product of this CTA's next tile has been issued (rows in buffer `buf`)
         int buf = 0;
 
@@ -498,7 +722,11 @@ levelised_kernel(LevParams p) {
                         if (tid == 0) {
                             bool go = true;
                             if (misc->failed) go = false;
-                            if (go && last_nonempty >= 0) go = wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
+                            // (as a block's attention stage: the level below is complete when the feed-forward stage has
+                            // refreshed its K | V rows)
+                            if (go && last_nonempty >= 0)
+                                go = p.block ? wait_counter(p.arrive + p.n_levels + last_nonempty, last_participants_ffn, p.abort_word, counter_limit)
+                                             : wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
                             if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                             if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
                             misc->go = go ? 1 : 0;
@@ -725,7 +953,12 @@ levelised_kernel(LevParams p) {
                     // stored and the level completes.  (Measured: for the 8-instruction W_o product the warp-level
                     // path wins, its fixed cost being nil; for these 16 instructions the asynchronous path does:
                     // a warp-level m16n8k16 occupies its sub-partition for about 32 clocks.)
-                    if (tid == 0) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
+                    // (as a block's attention stage there is no refresh here: the feed-forward stage does it, from the
+                    // block's output rows)
+                    if (tid == 0) {
+                        if (!p.block) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
+                        else if (pre_ok) post(kCmdQkv, buf ^ 1);
+                    }
                     const int node_v = misc->node[slot];
                     {
                         uint32_t w4[4];
@@ -753,6 +986,7 @@ levelised_kernel(LevParams p) {
                             }
                         }
                     }
+                    if (!p.block) {
                     if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
                     tc_fence_after();
@@ -780,6 +1014,7 @@ levelised_kernel(LevParams p) {
                             ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
                             st_global_v4((char*)p.KV[layer] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
                         }
+                    }
                     }
                     worker_sync();    // the tile's shared buffers may be overwritten from here on
                     pro_ready = pre_ok;
@@ -809,6 +1044,7 @@ levelised_kernel(LevParams p) {
             if (n_l > 0) {
                 last_nonempty = l;
                 last_participants = tiles < nctas ? tiles : nctas;
+                if (p.block) { const int t1 = tiles_of(n_l, ctas_of(1)); last_participants_ffn = t1 < ctas_of(1) ? t1 : ctas_of(1); }
             }
             // rotate the pipeline by one level
             v0 = vC; pad0 = padC;
@@ -816,6 +1052,7 @@ levelised_kernel(LevParams p) {
             lp0 = lp1; lp1 = lp2; lp2 = lp3; lp3 = lp4;
         }
         if (tid == 0) post(kCmdExit, 0);
+        }
     }
 
     tc_fence_before();
@@ -866,7 +1103,7 @@ size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers) {
 dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n_layers,
                                  __nv_bfloat16* const* KV, __nv_bfloat16* H, int64_t ldh,
                                  const __nv_bfloat16* const* W_qkv, const __nv_bfloat16* const* W_o, int32_t* sync,
-                                 int32_t* status, cudaStream_t st) {
+                                 int32_t* status, cudaStream_t st, const dg4i_block_tail* block) {
     if (n_layers < 1 || n_layers > DG4I_MAX_LAYERS)
         DG4_FAIL(DG4_ERR_UNSUPPORTED, "n_layers = %d: between 1 and %d layers per call", n_layers, DG4I_MAX_LAYERS);
     int dev = 0;
@@ -889,13 +1126,24 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         p.Wqkv[k] = W_qkv[kk];
         p.KV[k] = KV[kk];
     }
-    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, n_layers), st));
+    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, block ? 2 : n_layers), st));
     p.H = H; p.ldh = ldh;
     p.nbr_pad = g->nbr_pad; p.nbr_ptr = g->nbr_ptr; p.nbr_idx = g->nbr_idx;
     p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
     p.n_levels = g->n_levels; p.n_layers = n_layers;
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status; p.poll_limit = dg4i_poll_limit();
+    p.block = 0; p.eps = 0.f;
+    p.ln1_gamma = p.ln1_beta = p.b1 = p.b2 = p.ln2_gamma = p.ln2_beta = nullptr; p.W1 = p.W2 = nullptr;
+    if (block) {
+        // two kinds of CTA, dealt alternately: attention stage ("layer" 0) and feed-forward stage ("layer" 1)
+        if (n_layers != 1) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the block runs one layer per call");
+        if (g->wide) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the persistent block kernel takes cones of at most two hops");
+        if (g_sm_count[dev] < 2) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer than two SMs");
+        p.block = 1; p.n_layers = 2; p.eps = block->eps; p.residual = 1;
+        p.ln1_gamma = block->ln1_gamma; p.ln1_beta = block->ln1_beta; p.W1 = block->W1; p.b1 = block->b1;
+        p.W2 = block->W2; p.b2 = block->b2; p.ln2_gamma = block->ln2_gamma; p.ln2_beta = block->ln2_beta;
+    }
     const int grid = g_sm_count[dev];
     if (g->wide) return launch_heads<0>(desc->heads, p, grid, st);
     if (g->max_class <= 3) return launch_heads<3>(desc->heads, p, grid, st);

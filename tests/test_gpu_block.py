@@ -124,15 +124,19 @@ def test_block_matches_checker(hops, heads, n):
     assert rel_row_err(host_f64_of_bf16(out), want).max() <= BF16_ROW_TOL
 
 
-@pytest.mark.parametrize("hops,heads,n,window", [(1, 8, 900, 40), (2, 4, 3000, 64), (4, 8, 1500, 50)])
-def test_block_in_level_order_matches_checker(hops, heads, n, window):
-    """The whole block level by level (dg4_block_fwd_levelised): higher levels read the block outputs of lower ones."""
+@pytest.mark.parametrize("driver", ["persistent", "level-launches"])
+@pytest.mark.parametrize("hops,heads,n,window", [(1, 8, 900, 40), (2, 4, 3000, 64), (4, 8, 1500, 50), (2, 16, 20000, 3000),
+                                                 (1, 1, 31, 4)])
+def test_block_in_level_order_matches_checker(hops, heads, n, window, driver):
+    """The whole block level by level (dg4_block_fwd_levelised): higher levels read the block outputs of lower ones.
+    Two drivers: one persistent kernel whose attention-stage and feed-forward-stage CTAs hand the levels to one
+    another (cones of at most two hops), and one group of launches per level."""
     fanins = random_dag(np.random.default_rng(31 + hops), 30, n - 30, window=window)
     rp, ci = csr_from_fanins(fanins)
     level = levels_of(fanins)
     g = dg4.dg4_graph_create(rp, ci, level, hops, 0)
     scale = 1.0 / np.sqrt(128 // heads)
-    dsc = dg4.desc(heads, dg4.DG4_BF16, scale)
+    dsc = dg4.desc(heads, dg4.DG4_BF16, scale, level_launches=(driver == "level-launches"))
     xb = synth.normal_bf16_bits(26, 1, (n, 128), 1.0)
     wq_bits, wq = bf16_weights(synth.normal_f32(26, 2, (384, 128), 0.08))
     wo_bits, wo = bf16_weights(synth.normal_f32(26, 3, (128, 128), 0.08))
@@ -141,9 +145,12 @@ def test_block_in_level_order_matches_checker(hops, heads, n, window):
     host, dev = _ffn_params(26)
     ws = torch.empty(dg4.dg4_layer_workspace_bytes(g, dsc), dtype=torch.uint8, device="cuda")
     h = dev_bf16(xb).clone()
+    launches = dg4.dg4_launch_count()
     dg4.dg4_block_fwd_levelised(g, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), dg1, dbe1, *dev, EPS, ws)
     torch.cuda.synchronize()
     assert dg4.dg4_graph_poll_status(g) == 0
+    if driver == "persistent" and hops <= 2:
+        assert dg4.dg4_launch_count() - launches == 1       # one kernel for the whole block
     ptr, idx = orc.neighbourhood(rp, ci, hops)
     lptr, lnodes = orc.level_buckets(level)
     w1, b1, w2, b2, g2, be2 = host
@@ -157,6 +164,40 @@ def test_block_in_level_order_matches_checker(hops, heads, n, window):
     torch.cuda.synchronize()
     lvl0 = torch.from_numpy(np.nonzero(level == 0)[0]).cuda()
     assert torch.equal(h[lvl0], out[lvl0]) and not torch.equal(h, out)
+
+
+def test_block_in_level_order_with_empty_levels_and_many_tiles_per_level():
+    """A layering with gaps (every level number tripled) and levels wider than the feed-forward stage's CTAs x 16
+    nodes: both drivers give the same rows bit for bit (same arithmetic, same order), and they match the oracle."""
+    fanins = random_dag(np.random.default_rng(77), 3000, 9000, window=6000)
+    rp, ci = csr_from_fanins(fanins)
+    level = (levels_of(fanins) * 3).astype(np.int32)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, level, 2, 0)
+    assert np.bincount(level).max() > 75 * 16
+    heads, scale = 8, 0.25
+    xb = synth.normal_bf16_bits(27, 1, (n, 128), 1.0)
+    wq_bits, wq = bf16_weights(synth.normal_f32(27, 2, (384, 128), 0.08))
+    wo_bits, wo = bf16_weights(synth.normal_f32(27, 3, (128, 128), 0.08))
+    g1, dg1 = _vec(27, 4, 128, 0.2, 1.0)
+    be1, dbe1 = _vec(27, 5, 128, 0.2)
+    host, dev = _ffn_params(27)
+    outs = []
+    for launches in (False, True):
+        dsc = dg4.desc(heads, dg4.DG4_BF16, scale, level_launches=launches)
+        ws = torch.empty(dg4.dg4_layer_workspace_bytes(g, dsc), dtype=torch.uint8, device="cuda")
+        h = dev_bf16(xb).clone()
+        dg4.dg4_block_fwd_levelised(g, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), dg1, dbe1, *dev, EPS, ws)
+        torch.cuda.synchronize()
+        assert dg4.dg4_graph_poll_status(g) == 0
+        outs.append(h)
+    ptr, idx = orc.neighbourhood(rp, ci, 2)
+    lptr, lnodes = orc.level_buckets(level)
+    w1, b1, w2, b2, g2, be2 = host
+    want = orc.block_levelised(f64_of_bits(xb), wq, wo, g1, be1, w1, b1, w2, b2, g2, be2, ptr, idx, lptr, lnodes, heads,
+                               scale, eps=EPS, rounding="bf16")
+    for h in outs:
+        assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
 
 
 def test_block_calls_reject_bad_arguments():

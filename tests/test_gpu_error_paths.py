@@ -96,6 +96,11 @@ def test_waits_that_run_out_wind_the_kernels_down_and_report_timeout():
         dg4.dg4_layer_fwd_parallel(gr, dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=True, fused_layer=True),
                                    h, dwq, dwo, h, ws)
         assert dg4.dg4_graph_poll_status(gr) == dg4.DG4_ERR_TIMEOUT
+        gr, ws = fresh()                                # the block level by level as one persistent kernel
+        h = x.clone()
+        dg4.dg4_block_fwd_levelised(gr, dsc, h, dwq, dwo, vec, vec * 0, w1, b1, w2, vec * 0, vec, vec * 0, 1e-5, ws)
+        torch.cuda.synchronize()
+        assert dg4.dg4_graph_poll_status(gr) == dg4.DG4_ERR_TIMEOUT
         gr, ws = fresh()                                # persistent levelised kernel (its table-filling projection too)
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         h = x.clone()
