@@ -365,11 +365,11 @@ dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, vo
  * dg4_block_fwd_levelised: the same block in the paper's level-by-level order (Sec. 1 and Sec. 3.4 for the order,
  * Sec. 3.5 for the block), in place on H: levels 0, 1, ... in turn; a node takes its query and its own key / value
  * from its row as it was when the call started, and the key / value of every other member of N(v) from that node's
- * row as already replaced by this call, i.e. from its BLOCK output.  For cones of at most two hops the block runs
+ * row as already replaced by this call, i.e. from its BLOCK output.  The block runs
  * as ONE persistent cooperative kernel: half of its CTAs take the attention sub-layer of each level, the other half
  * the LayerNorm, feed-forward sub-layer, LayerNorm and the K | V refresh from the block's output rows, and the two
  * hand the levels to one another through per-level counters (every wait bounded; DG4_ERR_TIMEOUT in the handle's
- * status word if one runs out).  With DG4_FLAG_LEVEL_LAUNCHES, or for wider cones: one group of kernel launches
+ * status word if one runs out).  With DG4_FLAG_LEVEL_LAUNCHES: one group of kernel launches
  * per level (the level's rows are taken through the handle's level buckets).  Same results either way.
  */
 dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,

@@ -669,8 +669,7 @@ extern "C" dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc
     __nv_bfloat16* Q = (__nv_bfloat16*)workspace;
     __nv_bfloat16* KV = Q + (size_t)g->n * 128;
     __nv_bfloat16* O = Q + (size_t)g->n * 384;
-    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES) && !g->wide &&
-        (size_t)g->n * 256 >= dg4i_levelised_sync_bytes(g, 2)) {
+    if (!(desc->flags & DG4_FLAG_LEVEL_LAUNCHES) && (size_t)g->n * 256 >= dg4i_levelised_sync_bytes(g, 2)) {
         // one persistent kernel: attention-stage and feed-forward-stage CTAs hand the levels to one another (the
         // counters live where the launch-group driver keeps its Q table, which this path does not need)
         dg4i_block_tail tail;

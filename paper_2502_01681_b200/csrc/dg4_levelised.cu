@@ -1044,7 +1044,10 @@ levelised_kernel(LevParams p) {
             if (n_l > 0) {
                 last_nonempty = l;
                 last_participants = tiles < nctas ? tiles : nctas;
-                if (p.block) { const int t1 = tiles_of(n_l, ctas_of(1)); last_participants_ffn = t1 < ctas_of(1) ? t1 : ctas_of(1); }
+                if (p.block) {      // the feed-forward stage always fills 16-node tiles
+                    const int t1 = (n_l + kTile - 1) / kTile;
+                    last_participants_ffn = t1 < ctas_of(1) ? t1 : ctas_of(1);
+                }
             }
             // rotate the pipeline by one level
             v0 = vC; pad0 = padC;
@@ -1138,7 +1141,6 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     if (block) {
         // two kinds of CTA, dealt alternately: attention stage ("layer" 0) and feed-forward stage ("layer" 1)
         if (n_layers != 1) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the block runs one layer per call");
-        if (g->wide) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the persistent block kernel takes cones of at most two hops");
         if (g_sm_count[dev] < 2) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer than two SMs");
         p.block = 1; p.n_layers = 2; p.eps = block->eps; p.residual = 1;
         p.ln1_gamma = block->ln1_gamma; p.ln1_beta = block->ln1_beta; p.W1 = block->W1; p.b1 = block->b1;
