@@ -387,6 +387,19 @@ dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, voi
                                    const void* W1, const float* b1, const void* W2, const float* b2,
                                    const float* ln2_gamma, const float* ln2_beta, float eps, int32_t d_ff,
                                    void* workspace, size_t workspace_bytes, void* stream);
+/* Several blocks in level-by-level order in one call, as ONE wavefront (block k+1 takes a level as soon as block k
+ * has finished it): the same result as n_blocks successive dg4_block_fwd_levelised calls, bit for bit, with a
+ * dependent chain n_levels + 2 n_blocks - 1 stage steps long instead of n_blocks * 2 * n_levels.  Every parameter
+ * of the single-block call becomes a host array of n_blocks device pointers (1 .. 8 blocks); eps and d_ff are
+ * shared.  workspace: at least dg4_blocks_workspace_bytes() bytes, 256-byte aligned.  Always the persistent kernel. */
+size_t dg4_blocks_workspace_bytes(const dg4_graph* g, const dg4_desc* desc, int32_t n_blocks);
+dg4_status dg4_blocks_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh, int32_t n_blocks,
+                                    const void* const* W_qkv, const void* const* W_o,
+                                    const float* const* ln1_gamma, const float* const* ln1_beta,
+                                    const void* const* W1, const float* const* b1, const void* const* W2,
+                                    const float* const* b2, const float* const* ln2_gamma,
+                                    const float* const* ln2_beta, float eps, int32_t d_ff, void* workspace,
+                                    size_t workspace_bytes, void* stream);
 
 /*
  * Diagnostic (the paper has no counterpart): launches one small CTA that waits, with the same bounded wait the

@@ -712,6 +712,57 @@ extern "C" dg4_status dg4_block_fwd_levelised(const dg4_graph* g, const dg4_desc
     return DG4_OK;
 }
 
+extern "C" size_t dg4_blocks_workspace_bytes(const dg4_graph* g, const dg4_desc* desc, int32_t n_blocks) {
+    (void)desc;
+    if (!g || n_blocks < 1 || n_blocks > DG4I_MAX_LAYERS) return 0;
+    const size_t tables = (((size_t)g->n * 512 + 255) / 256) * 256 * (size_t)n_blocks;
+    return tables + ((dg4i_levelised_sync_bytes(g, 2 * n_blocks) + 255) / 256) * 256;
+}
+
+/* Several blocks in level-by-level order as ONE wavefront: the attention stage and the feed-forward stage of every
+ * block are pipeline stages of one persistent kernel; block k+1 takes a level as soon as block k has finished it. */
+extern "C" dg4_status dg4_blocks_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, void* H, int64_t ldh,
+                                                int32_t n_blocks, const void* const* W_qkv, const void* const* W_o,
+                                                const float* const* ln1_gamma, const float* const* ln1_beta,
+                                                const void* const* W1, const float* const* b1, const void* const* W2,
+                                                const float* const* b2, const float* const* ln2_gamma,
+                                                const float* const* ln2_beta, float eps, int32_t d_ff, void* workspace,
+                                                size_t workspace_bytes, void* stream) {
+    CHECK(check_common(g, desc, eps));
+    CHECK(dg4i_check_desc(desc, true));
+    CHECK(check_rows("H", H, ldh));
+    if (n_blocks < 1 || n_blocks > DG4I_MAX_LAYERS)
+        DG4_FAIL(DG4_ERR_UNSUPPORTED, "n_blocks = %d: between 1 and %d blocks per call", n_blocks, DG4I_MAX_LAYERS);
+    if (!W_qkv || !W_o || !ln1_gamma || !ln1_beta || !W1 || !b1 || !W2 || !b2 || !ln2_gamma || !ln2_beta)
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "null parameter array");
+    dg4i_block_tail tails[DG4I_MAX_LAYERS];
+    const __nv_bfloat16* wq[DG4I_MAX_LAYERS];
+    const __nv_bfloat16* wo[DG4I_MAX_LAYERS];
+    __nv_bfloat16* kv[DG4I_MAX_LAYERS];
+    if (!workspace) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is null");
+    if ((((uintptr_t)workspace) & 255u) != 0) DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace is not 256-byte aligned");
+    if (workspace_bytes < dg4_blocks_workspace_bytes(g, desc, n_blocks))
+        DG4_FAIL(DG4_ERR_INVALID_ARG, "workspace of %zu bytes is below the %zu bytes needed", workspace_bytes,
+                 dg4_blocks_workspace_bytes(g, desc, n_blocks));
+    const size_t table = (((size_t)g->n * 512 + 255) / 256) * 256;
+    for (int k = 0; k < n_blocks; ++k) {
+        if (!W_qkv[k] || !W_o[k] || !aligned16(W_qkv[k]) || !aligned16(W_o[k]))
+            DG4_FAIL(DG4_ERR_INVALID_ARG, "W_qkv / W_o of block %d null or misaligned", k);
+        CHECK(check_vec("ln1_gamma", ln1_gamma[k]));
+        CHECK(check_vec("ln1_beta", ln1_beta[k]));
+        CHECK(check_ffn_args(W1[k], b1[k], W2[k], b2[k], ln2_gamma[k], ln2_beta[k], d_ff));
+        tails[k].ln1_gamma = ln1_gamma[k]; tails[k].ln1_beta = ln1_beta[k];
+        tails[k].W1 = (const __nv_bfloat16*)W1[k]; tails[k].b1 = b1[k];
+        tails[k].W2 = (const __nv_bfloat16*)W2[k]; tails[k].b2 = b2[k];
+        tails[k].ln2_gamma = ln2_gamma[k]; tails[k].ln2_beta = ln2_beta[k]; tails[k].eps = eps;
+        wq[k] = (const __nv_bfloat16*)W_qkv[k]; wo[k] = (const __nv_bfloat16*)W_o[k];
+        kv[k] = (__nv_bfloat16*)((char*)workspace + table * (size_t)k);
+    }
+    int32_t* sync = (int32_t*)((char*)workspace + table * (size_t)n_blocks);
+    return dg4i_levelised_launch(g, desc, n_blocks, kv, (__nv_bfloat16*)H, ldh, wq, wo, sync, g->dev_status,
+                                 (cudaStream_t)stream, tails);
+}
+
 extern "C" dg4_status dg4_block_fwd_parallel(const dg4_graph* g, const dg4_desc* desc, const void* H_in, int64_t ldh,
                                               const void* W_qkv, const void* W_o, const float* ln1_gamma,
                                               const float* ln1_beta, const void* W1, const float* b1, const void* W2,

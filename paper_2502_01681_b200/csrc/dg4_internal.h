@@ -151,9 +151,10 @@ dg4_status dg4i_fused_layer_launch(const dg4_graph* g, const dg4_desc* desc, con
 // by the call and must hold dg4i_levelised_sync_bytes() bytes.
 #define DG4I_MAX_LAYERS 8
 size_t dg4i_levelised_sync_bytes(const dg4_graph* g, int n_layers);
-// With `block` (one layer, cones of at most two hops): the whole Transformer block level by level -- half of the
-// CTAs run the attention sub-layer of each level, the other half its LayerNorm, feed-forward sub-layer, LayerNorm
-// and the K | V refresh from the block's output rows.  `sync` then holds dg4i_levelised_sync_bytes(g, 2) bytes.
+// With `block` (an array of n_layers entries): whole Transformer blocks level by level -- for every block one group
+// of CTAs runs the attention sub-layer of each level, another its LayerNorm, feed-forward sub-layer, LayerNorm
+// and the K | V refresh from the block's output rows; the stages of all blocks form one wavefront.  `sync` then
+// holds dg4i_levelised_sync_bytes(g, 2 * n_layers) bytes.
 struct dg4i_block_tail {
     const float* ln1_gamma; const float* ln1_beta;
     const __nv_bfloat16* W1; const float* b1;          // [512, 128], [512]

@@ -151,14 +151,16 @@ struct LevParams {
     // The whole Transformer block level by level (block != 0, n_layers == 2): the CTAs of "layer" 0 run the
     // attention sub-layer of a level, those of "layer" 1 its LayerNorm, feed-forward sub-layer, LayerNorm and the
     // K | V refresh from the block's output rows; the two hand each level to one another through the counters.
+    // Several blocks: n_layers == 2 x blocks, "layer" 2k is block k's attention stage, 2k+1 its feed-forward stage,
+    // and the stages of all blocks form one wavefront.
     int32_t block;
     float eps;
-    const float* ln1_gamma; const float* ln1_beta;
-    const __nv_bfloat16* W1;               // [512, 128]
-    const float* b1;                       // [512]
-    const __nv_bfloat16* W2;               // [128, 512]
-    const float* b2;                       // [128]
-    const float* ln2_gamma; const float* ln2_beta;
+    const float* ln1_gamma[DG4I_MAX_LAYERS]; const float* ln1_beta[DG4I_MAX_LAYERS];
+    const __nv_bfloat16* W1[DG4I_MAX_LAYERS];              // [512, 128]
+    const float* b1[DG4I_MAX_LAYERS];                      // [512]
+    const __nv_bfloat16* W2[DG4I_MAX_LAYERS];              // [128, 512]
+    const float* b2[DG4I_MAX_LAYERS];                      // [128]
+    const float* ln2_gamma[DG4I_MAX_LAYERS]; const float* ln2_beta[DG4I_MAX_LAYERS];
 };
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint32_t* r) {
@@ -296,12 +298,13 @@ levelised_kernel(LevParams p) {
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
-    const bool ffn_stage = p.block != 0 && layer == 1;
+    const bool ffn_stage = p.block != 0 && (layer & 1) != 0;
+    const int wl = p.block ? layer >> 1 : layer;         // whose weights and K | V table this CTA works with
     if (warp < 8 && ffn_stage) {
         // W_k, W_v as everywhere; W1's four blocks of 128 hidden units in tensor memory; W2 in shared memory as
         // four 128 x 128 blocks (block c = hidden units 128c .. 128c+127) in the swizzled K-major layout
         for (int blk = 1; blk <= 6; ++blk) {
-            const __nv_bfloat16* wb = blk <= 2 ? p.Wqkv[layer] + (size_t)blk * 128 * 128 : p.W1 + (size_t)(blk - 3) * 128 * 128;
+            const __nv_bfloat16* wb = blk <= 2 ? p.Wqkv[wl] + (size_t)blk * 128 * 128 : p.W1[wl] + (size_t)(blk - 3) * 128 * 128;
             const uint32_t col0 = blk <= 2 ? (uint32_t)(kWCol0 + blk * kWCols) : (uint32_t)(kColW1 + (blk - 3) * kWCols);
             const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
 #pragma unroll
@@ -314,15 +317,15 @@ levelised_kernel(LevParams p) {
         tmem_st_wait();
         for (int i = tid; i < 4 * 128 * 16; i += kWorkers) {
             const int c = i >> 11, row = (i >> 4) & 127, chunk = i & 15;
-            const uint4 v = *reinterpret_cast<const uint4*>(p.W2 + (size_t)row * 512 + c * 128 + chunk * 8);
+            const uint4 v = *reinterpret_cast<const uint4*>(p.W2[wl] + (size_t)row * 512 + c * 128 + chunk * 8);
             const uint32_t r[4] = {v.x, v.y, v.z, v.w};
             st_shared_v4(sW + (uint32_t)(c * kWBlock) + weight_piece(row, chunk), r);
         }
         fence_proxy_async_smem();
     } else if (warp < 8) {
         for (int blk = kBlkK; blk <= kBlkQ; ++blk) {
-            const __nv_bfloat16* wb = blk == kBlkQ ? p.Wqkv[layer]
-                                                    : p.Wqkv[layer] + (size_t)blk * 128 * 128;     // kBlkK = 1, kBlkV = 2
+            const __nv_bfloat16* wb = blk == kBlkQ ? p.Wqkv[wl]
+                                                    : p.Wqkv[wl] + (size_t)blk * 128 * 128;     // kBlkK = 1, kBlkV = 2
             const uint4* src = reinterpret_cast<const uint4*>(wb + (size_t)feat * 128 + cg * 64);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -335,7 +338,7 @@ levelised_kernel(LevParams p) {
         // W_o once more in shared memory (same 128-byte swizzle): the B operand of the warp-level output projection
         for (int i = tid; i < 128 * 16; i += kWorkers) {
             const int row = i >> 4, chunk = i & 15;
-            const uint4 v = *reinterpret_cast<const uint4*>(p.Wo[layer] + (size_t)row * 128 + chunk * 8);
+            const uint4 v = *reinterpret_cast<const uint4*>(p.Wo[wl] + (size_t)row * 128 + chunk * 8);
             const uint32_t r[4] = {v.x, v.y, v.z, v.w};
             st_shared_v4(sW + weight_piece(row, chunk), r);
         }
@@ -441,7 +444,7 @@ levelised_kernel(LevParams p) {
         bool alive = true;
         const uint32_t counter_limit = p.poll_limit > 4u ? p.poll_limit >> 2 : 1u;   // a counter poll is a trip to L2
 
-        const char* kv_tab = (const char*)p.KV[layer];
+        const char* kv_tab = (const char*)p.KV[wl];
         int32_t* my_arrive = p.arrive + (size_t)layer * p.n_levels;
         const int32_t* prev_arrive = layer > 0 ? p.arrive + (size_t)(layer - 1) * p.n_levels : nullptr;
         const int prev_ctas = layer > 0 ? ctas_of(layer - 1) : 0;
@@ -458,7 +461,11 @@ levelised_kernel(LevParams p) {
         };
         auto tiles_of = [&](int n_level, int ctas) { const int t = per_tile(n_level, ctas); return (n_level + t - 1) / t; };
         // arrivals on the layer below's counter for a level of n_level nodes (one per CTA that owns a tile of it)
-        auto prev_target = [&](int n_level) { const int t = tiles_of(n_level, prev_ctas); return t < prev_ctas ? t : prev_ctas; };
+        // (a feed-forward stage always fills 16-node tiles)
+        auto prev_target = [&](int n_level) {
+            const int t = (p.block && !ffn_stage) ? (n_level + kTile - 1) / kTile : tiles_of(n_level, prev_ctas);
+            return t < prev_ctas ? t : prev_ctas;
+        };
 
         // this lane's piece of node v's input row (zero for an empty slot) into input buffer b, both layouts
         auto stage_input = [&](int b, const Piece& x) {
@@ -506,12 +513,12 @@ levelised_kernel(LevParams p) {
             float g1[8], be1[8], g2[8], be2[8], bo[8], bh[4];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                g1[i] = __ldg(p.ln1_gamma + sub * 8 + i); be1[i] = __ldg(p.ln1_beta + sub * 8 + i);
-                g2[i] = __ldg(p.ln2_gamma + sub * 8 + i); be2[i] = __ldg(p.ln2_beta + sub * 8 + i);
-                bo[i] = __ldg(p.b2 + sub * 8 + i);
+                g1[i] = __ldg(p.ln1_gamma[wl] + sub * 8 + i); be1[i] = __ldg(p.ln1_beta[wl] + sub * 8 + i);
+                g2[i] = __ldg(p.ln2_gamma[wl] + sub * 8 + i); be2[i] = __ldg(p.ln2_beta[wl] + sub * 8 + i);
+                bo[i] = __ldg(p.b2[wl] + sub * 8 + i);
             }
 #pragma unroll
-            for (int blk = 0; blk < 4; ++blk) bh[blk] = __ldg(p.b1 + blk * 128 + feat);
+            for (int blk = 0; blk < 4; ++blk) bh[blk] = __ldg(p.b1[wl] + blk * 128 + feat);
             auto layer_norm = [&](float* x, const float* g, const float* b) {     // over the node's 128 features (16 lanes)
                 float sum = 0.f;
 #pragma unroll
@@ -636,7 +643,7 @@ levelised_kernel(LevParams p) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
-                            st_global_v4((char*)p.KV[layer] + (size_t)v * 512 + (sub + 16 * h) * 16, w4);
+                            st_global_v4((char*)p.KV[wl] + (size_t)v * 512 + (sub + 16 * h) * 16, w4);
                         }
                     }
                     worker_sync();
@@ -725,7 +732,7 @@ levelised_kernel(LevParams p) {
                             // (as a block's attention stage: the level below is complete when the feed-forward stage has
                             // refreshed its K | V rows)
                             if (go && last_nonempty >= 0)
-                                go = p.block ? wait_counter(p.arrive + p.n_levels + last_nonempty, last_participants_ffn, p.abort_word, counter_limit)
+                                go = p.block ? wait_counter(p.arrive + (size_t)(layer + 1) * p.n_levels + last_nonempty, last_participants_ffn, p.abort_word, counter_limit)
                                              : wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
                             if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                             if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
@@ -1012,7 +1019,7 @@ levelised_kernel(LevParams p) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {        // this layer's K | V row
                             ld_shared_v4(row + (uint32_t)((sub + 16 * h) * 16), w4);
-                            st_global_v4((char*)p.KV[layer] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
+                            st_global_v4((char*)p.KV[wl] + (size_t)node_v * 512 + (sub + 16 * h) * 16, w4);
                         }
                     }
                     }
@@ -1046,7 +1053,7 @@ levelised_kernel(LevParams p) {
                 last_participants = tiles < nctas ? tiles : nctas;
                 if (p.block) {      // the feed-forward stage always fills 16-node tiles
                     const int t1 = (n_l + kTile - 1) / kTile;
-                    last_participants_ffn = t1 < ctas_of(1) ? t1 : ctas_of(1);
+                    last_participants_ffn = t1 < ctas_of(layer + 1) ? t1 : ctas_of(layer + 1);
                 }
             }
             // rotate the pipeline by one level
@@ -1129,7 +1136,7 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         p.Wqkv[k] = W_qkv[kk];
         p.KV[k] = KV[kk];
     }
-    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, block ? 2 : n_layers), st));
+    DG4_CUDA_TRY(cudaMemsetAsync(sync, 0, dg4i_levelised_sync_bytes(g, block ? 2 * n_layers : n_layers), st));
     p.H = H; p.ldh = ldh;
     p.nbr_pad = g->nbr_pad; p.nbr_ptr = g->nbr_ptr; p.nbr_idx = g->nbr_idx;
     p.level_ptr = g->level_ptr; p.level_nodes = g->level_nodes;
@@ -1137,14 +1144,18 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status; p.poll_limit = dg4i_poll_limit();
     p.block = 0; p.eps = 0.f;
-    p.ln1_gamma = p.ln1_beta = p.b1 = p.b2 = p.ln2_gamma = p.ln2_beta = nullptr; p.W1 = p.W2 = nullptr;
+    for (int k = 0; k < DG4I_MAX_LAYERS; ++k) {
+        p.ln1_gamma[k] = p.ln1_beta[k] = p.b1[k] = p.b2[k] = p.ln2_gamma[k] = p.ln2_beta[k] = nullptr;
+        p.W1[k] = p.W2[k] = nullptr;
+    }
     if (block) {
-        // two kinds of CTA, dealt alternately: attention stage ("layer" 0) and feed-forward stage ("layer" 1)
-        if (n_layers != 1) DG4_FAIL(DG4_ERR_UNSUPPORTED, "the block runs one layer per call");
-        if (g_sm_count[dev] < 2) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer than two SMs");
-        p.block = 1; p.n_layers = 2; p.eps = block->eps; p.residual = 1;
-        p.ln1_gamma = block->ln1_gamma; p.ln1_beta = block->ln1_beta; p.W1 = block->W1; p.b1 = block->b1;
-        p.W2 = block->W2; p.b2 = block->b2; p.ln2_gamma = block->ln2_gamma; p.ln2_beta = block->ln2_beta;
+        // two kinds of CTA per block, dealt round-robin: attention stage ("layer" 2k) and feed-forward stage (2k+1)
+        if (g_sm_count[dev] < 2 * n_layers) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer SMs than stages");
+        p.block = 1; p.n_layers = 2 * n_layers; p.eps = block[0].eps; p.residual = 1;
+        for (int k = 0; k < n_layers; ++k) {
+            p.ln1_gamma[k] = block[k].ln1_gamma; p.ln1_beta[k] = block[k].ln1_beta; p.W1[k] = block[k].W1; p.b1[k] = block[k].b1;
+            p.W2[k] = block[k].W2; p.b2[k] = block[k].b2; p.ln2_gamma[k] = block[k].ln2_gamma; p.ln2_beta[k] = block[k].ln2_beta;
+        }
     }
     const int grid = g_sm_count[dev];
     if (g->wide) return launch_heads<0>(desc->heads, p, grid, st);

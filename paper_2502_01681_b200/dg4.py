@@ -44,6 +44,7 @@ EXPORTS = [
     "dg4_layernorm_fwd", "dg4_ffn_fwd", "dg4_block_fwd_parallel", "dg4_graph_destroy_async", "dg4_memory_trim",
     "dg4_debug_set_poll_limit", "dg4_debug_override_current_device",
     "dg4_cone_update_workspace_bytes", "dg4_cone_update_fwd", "dg4_block_fwd_levelised",
+    "dg4_blocks_workspace_bytes", "dg4_blocks_fwd_levelised",
 ]
 
 
@@ -148,6 +149,12 @@ def load():
     lib.dg4_block_fwd_levelised.restype = ctypes.c_int
     lib.dg4_block_fwd_levelised.argtypes = [vp, dp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, cf, ctypes.c_int32,
                                             vp, ctypes.c_size_t, vp]
+    lib.dg4_blocks_workspace_bytes.restype = ctypes.c_size_t
+    lib.dg4_blocks_workspace_bytes.argtypes = [vp, dp, ctypes.c_int32]
+    pvp = ctypes.POINTER(vp)
+    lib.dg4_blocks_fwd_levelised.restype = ctypes.c_int
+    lib.dg4_blocks_fwd_levelised.argtypes = [vp, dp, vp, i64, ctypes.c_int32, pvp, pvp, pvp, pvp, pvp, pvp, pvp, pvp, pvp, pvp,
+                                             cf, ctypes.c_int32, vp, ctypes.c_size_t, vp]
     lib.dg4_cone_update_workspace_bytes.restype = ctypes.c_size_t
     lib.dg4_cone_update_workspace_bytes.argtypes = [vp, dp, ctypes.c_int32]
     lib.dg4_cone_update_fwd.restype = ctypes.c_int
@@ -406,6 +413,21 @@ def dg4_block_fwd_levelised(g: Graph, dsc: dg4_desc, H, W_qkv, W_o, ln1_gamma, l
                                           _ptr(ln2_gamma), _ptr(ln2_beta), ctypes.c_float(eps), int(W1.shape[0]),
                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
                                           _stream(stream)))
+
+
+def dg4_blocks_workspace_bytes(g: Graph, dsc: dg4_desc, n_blocks: int) -> int:
+    return int(load().dg4_blocks_workspace_bytes(g.handle, ctypes.byref(dsc), n_blocks))
+
+
+def dg4_blocks_fwd_levelised(g: Graph, dsc: dg4_desc, H, blocks, eps, workspace, stream=None):
+    """Several whole blocks level by level as one wavefront, in place on H.  `blocks`: one tuple per block,
+    (W_qkv, W_o, ln1_gamma, ln1_beta, W1, b1, W2, b2, ln2_gamma, ln2_beta), device tensors."""
+    n = len(blocks)
+    arr = ctypes.c_void_p * n
+    cols = [arr(*[blk[i].data_ptr() for blk in blocks]) for i in range(10)]
+    _check(load().dg4_blocks_fwd_levelised(g.handle, ctypes.byref(dsc), _ptr(H), _ld(H), n, *cols, ctypes.c_float(eps),
+                                           int(blocks[0][4].shape[0]), _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def dg4_graph_partition(g: Graph, delta: int):

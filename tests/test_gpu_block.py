@@ -200,6 +200,49 @@ def test_block_in_level_order_with_empty_levels_and_many_tiles_per_level():
         assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
 
 
+@pytest.mark.parametrize("hops,n_blocks", [(2, 3), (1, 2), (4, 2)])
+def test_blocks_as_one_wavefront_equal_successive_blocks(hops, n_blocks):
+    """dg4_blocks_fwd_levelised: the stages of all blocks as one wavefront give, bit for bit, what one
+    dg4_block_fwd_levelised call per block gives; and that matches the oracle applied block after block."""
+    fanins = random_dag(np.random.default_rng(91 + hops), 60, 6000, window=150)
+    rp, ci = csr_from_fanins(fanins)
+    level = levels_of(fanins)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, level, hops, 0)
+    heads, scale = 8, 0.25
+    dsc = dg4.desc(heads, dg4.DG4_BF16, scale)
+    xb = synth.normal_bf16_bits(28, 1, (n, 128), 1.0)
+    host_blocks, dev_blocks = [], []
+    for k in range(n_blocks):
+        wq_bits, wq = bf16_weights(synth.normal_f32(28, 10 * k + 2, (384, 128), 0.08))
+        wo_bits, wo = bf16_weights(synth.normal_f32(28, 10 * k + 3, (128, 128), 0.08))
+        g1, dg1 = _vec(28, 10 * k + 4, 128, 0.2, 1.0)
+        be1, dbe1 = _vec(28, 10 * k + 5, 128, 0.2)
+        host, dev = _ffn_params(28 + k)
+        host_blocks.append((wq, wo, g1, be1) + tuple(host))
+        dev_blocks.append((dev_bf16(wq_bits), dev_bf16(wo_bits), dg1, dbe1) + tuple(dev))
+    ws = torch.empty(max(dg4.dg4_blocks_workspace_bytes(g, dsc, n_blocks), dg4.dg4_layer_workspace_bytes(g, dsc)),
+                     dtype=torch.uint8, device="cuda")
+    h = dev_bf16(xb).clone()
+    launches = dg4.dg4_launch_count()
+    dg4.dg4_blocks_fwd_levelised(g, dsc, h, dev_blocks, EPS, ws)
+    torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(g) == 0 and dg4.dg4_launch_count() - launches == 1
+    h2 = dev_bf16(xb).clone()
+    for blk in dev_blocks:
+        dg4.dg4_block_fwd_levelised(g, dsc, h2, *blk, EPS, ws)
+    torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(g) == 0
+    assert torch.equal(h.view(torch.int16), h2.view(torch.int16))
+    ptr, idx = orc.neighbourhood(rp, ci, hops)
+    lptr, lnodes = orc.level_buckets(level)
+    want = f64_of_bits(xb)
+    for (wq, wo, g1, be1, w1, b1, w2, b2, g2, be2) in host_blocks:
+        want = orc.block_levelised(want, wq, wo, g1, be1, w1, b1, w2, b2, g2, be2, ptr, idx, lptr, lnodes, heads, scale,
+                                   eps=EPS, rounding="bf16")
+    assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
+
+
 def test_block_calls_reject_bad_arguments():
     n = 64
     g = _edgeless(n)
