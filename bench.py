@@ -376,6 +376,27 @@ def run_ours(args, w):
         # with the three kernels timed inside the step
         dsc_fused = dg4.desc(w.heads, dg4.DG4_BF16, w.scale, residual=w.residual, fused_layer=True)
         fused_ms = timed3(lambda: dg4.dg4_layer_fwd_parallel(gr, dsc_fused, x_dev, wq[0], wo[0], h_par, ws))
+        # the whole block level by level: one block, and three blocks as one wavefront (persistent kernel whose
+        # attention-stage and feed-forward-stage CTAs hand the levels to one another), in place on a copy of X
+        blocks3 = [(wq[l], wo[l], gam, bet, w1, b1, w2, b2, gam, bet) for l in range(3)]
+        ws_blk = torch.empty(max(dg4.dg4_blocks_workspace_bytes(gr, dsc, 3), dg4.dg4_layer_workspace_bytes(gr, dsc)),
+                             dtype=torch.uint8, device="cuda")
+
+        def timed1(fn):
+            h_par.copy_(x_dev)
+            fn()
+            h_par.copy_(x_dev)
+            t0, t1 = ev(), ev()
+            t0.record(stream)
+            fn()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1)
+
+        block_lev_ms = timed1(lambda: dg4.dg4_block_fwd_levelised(gr, dsc, h_par, *blocks3[0], 1e-5, ws_blk))
+        blocks3_lev_ms = timed1(lambda: dg4.dg4_blocks_fwd_levelised(gr, dsc, h_par, blocks3, 1e-5, ws_blk))
+        del ws_blk
+        extras.update({"block_levelised_ms": block_lev_ms, "blocks3_levelised_ms": blocks3_lev_ms})
         extras.update({"ffn_ms": ffn_ms, "ffn_tflops": 4.0 * 128 * 512 * n / (ffn_ms * 1e-3) / 1e12,
                        "layernorm_ms": ln_ms, "layernorm_gbs": 512.0 * n / (ln_ms * 1e-3) / 1e9,
                        "block_parallel_ms": blk_ms, "parallel_layer_fused_ms": fused_ms})
