@@ -105,15 +105,18 @@ constexpr int kOffMisc = kOffS32 + kTile * 128 * 4;
 constexpr int kWHalf = 128 * 128;                      // K-half of a 128-row weight block: 128 rows x 128 bytes
 constexpr int kWBlock = 2 * kWHalf;                    // a 128 x 128 bf16 block in shared memory (32 KiB)
 constexpr int kOffWs = ((kOffMisc + 256 + 1023) / 1024) * 1024;   // W_o for the warp-level output projection; W2 (4 blocks) in a feed-forward CTA
-constexpr int kSmemBytes = kOffWs + 4 * kWBlock + 1024;
-static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
+constexpr int kSmemBytes = kOffWs + kWBlock + 1024;              // layers: W_o
+constexpr int kSmemBytesBlock = kOffWs + 4 * kWBlock + 1024;     // blocks: room for W2 in the feed-forward-stage CTAs
+static_assert(kSmemBytesBlock <= 232448, "shared memory budget of one CTA");
 static_assert(kWCol0 + 4 * kWCols <= kTmemCols && kColW1 + 4 * kWCols <= kTmemCols && 6 * kTile <= kWCol0 + kWCols &&
               kColD2 + kTile <= kWCol0 + kWCols, "tensor memory budget of one CTA");
 static_assert((kOffX % 1024) == 0 && (kOffHp % 1024) == 0 && (kTileOp % 1024) == 0, "operand tiles are 1024-byte aligned");
 // Every CTA allocates all of its SM's tensor memory, so two CTAs must never share an SM (the second one's
 // allocation would wait for the first, which waits for the second's levels): the launch asks for more than half
 // of an SM's shared memory, which rules that out.
+// (Blocks ask for more: only then is the rest of the SM's 256 KiB, which the gathers use as L1, given up.)
 constexpr int kLaunchSmemBytes = kSmemBytes > 120 * 1024 ? kSmemBytes : 120 * 1024;
+static_assert(kSmemBytesBlock > 120 * 1024, "one CTA per SM in block mode too");
 
 enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdKv = 2, kCmdKvThenQkv = 3, kCmdFfn1 = 4, kCmdFfn2 = 5 };
 
@@ -247,7 +250,8 @@ __device__ __forceinline__ bool wait_counter(const int32_t* counter, int target,
     return true;
 }
 
-template <int LPH, int MAXN>
+// BLOCK: the whole Transformer block (attention-stage and feed-forward-stage CTAs) instead of attention layers.
+template <int LPH, int MAXN, bool BLOCK>
 __global__ void __launch_bounds__(kThreads, 1)
 levelised_kernel(LevParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -298,8 +302,8 @@ levelised_kernel(LevParams p) {
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
-    const bool ffn_stage = p.block != 0 && (layer & 1) != 0;
-    const int wl = p.block ? layer >> 1 : layer;         // whose weights and K | V table this CTA works with
+    const bool ffn_stage = BLOCK && (layer & 1) != 0;
+    const int wl = BLOCK ? layer >> 1 : layer;         // whose weights and K | V table this CTA works with
     if (warp < 8 && ffn_stage) {
         // W_k, W_v as everywhere; W1's four blocks of 128 hidden units in tensor memory; W2 in shared memory as
         // four 128 x 128 blocks (block c = hidden units 128c .. 128c+127) in the swizzled K-major layout
@@ -463,7 +467,7 @@ levelised_kernel(LevParams p) {
         // arrivals on the layer below's counter for a level of n_level nodes (one per CTA that owns a tile of it)
         // (a feed-forward stage always fills 16-node tiles)
         auto prev_target = [&](int n_level) {
-            const int t = (p.block && !ffn_stage) ? (n_level + kTile - 1) / kTile : tiles_of(n_level, prev_ctas);
+            const int t = (BLOCK && !ffn_stage) ? (n_level + kTile - 1) / kTile : tiles_of(n_level, prev_ctas);
             return t < prev_ctas ? t : prev_ctas;
         };
 
@@ -732,7 +736,7 @@ levelised_kernel(LevParams p) {
                             // (as a block's attention stage: the level below is complete when the feed-forward stage has
                             // refreshed its K | V rows)
                             if (go && last_nonempty >= 0)
-                                go = p.block ? wait_counter(p.arrive + (size_t)(layer + 1) * p.n_levels + last_nonempty, last_participants_ffn, p.abort_word, counter_limit)
+                                go = BLOCK ? wait_counter(p.arrive + (size_t)(layer + 1) * p.n_levels + last_nonempty, last_participants_ffn, p.abort_word, counter_limit)
                                              : wait_counter(my_arrive + last_nonempty, last_participants, p.abort_word, counter_limit);
                             if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
                             if (go && (l & 255) == 0 && ld_acquire(p.abort_word) != 0) go = false;
@@ -963,7 +967,7 @@ levelised_kernel(LevParams p) {
                     // (as a block's attention stage there is no refresh here: the feed-forward stage does it, from the
                     // block's output rows)
                     if (tid == 0) {
-                        if (!p.block) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
+                        if (!BLOCK) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
                         else if (pre_ok) post(kCmdQkv, buf ^ 1);
                     }
                     const int node_v = misc->node[slot];
@@ -993,7 +997,7 @@ levelised_kernel(LevParams p) {
                             }
                         }
                     }
-                    if (!p.block) {
+                    if (!BLOCK) {
                     if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
                     tc_fence_after();
@@ -1051,7 +1055,7 @@ levelised_kernel(LevParams p) {
             if (n_l > 0) {
                 last_nonempty = l;
                 last_participants = tiles < nctas ? tiles : nctas;
-                if (p.block) {      // the feed-forward stage always fills 16-node tiles
+                if (BLOCK) {      // the feed-forward stage always fills 16-node tiles
                     const int t1 = (n_l + kTile - 1) / kTile;
                     last_participants_ffn = t1 < ctas_of(layer + 1) ? t1 : ctas_of(layer + 1);
                 }
@@ -1079,17 +1083,23 @@ int g_sm_count[64] = {};
 int g_coop[64] = {};
 bool g_dev_known[64] = {};
 
-template <int LPH, int MAXN>
-dg4_status launch(const LevParams& p, int grid, cudaStream_t st) {
-    auto kern = levelised_kernel<LPH, MAXN>;
-    DG4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kLaunchSmemBytes));
+template <int LPH, int MAXN, bool BLOCK>
+dg4_status launch_mode(const LevParams& p, int grid, cudaStream_t st) {
+    auto kern = levelised_kernel<LPH, MAXN, BLOCK>;
+    const int smem = p.block ? kSmemBytesBlock : kLaunchSmemBytes;
+    DG4_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesBlock));
     int per_sm = 0;
-    DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kLaunchSmemBytes));
+    DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem));
     if (per_sm != 1) DG4_FAIL(DG4_ERR_CUDA, "the levelised kernel needs exactly one CTA per SM on this device (got %d)", per_sm);
     void* args[] = {(void*)&p};
-    DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, kLaunchSmemBytes, st));
+    DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem, st));
     dg4i_count_launch();
     return DG4_OK;
+}
+
+template <int LPH, int MAXN>
+dg4_status launch(const LevParams& p, int grid, cudaStream_t st) {
+    return p.block ? launch_mode<LPH, MAXN, true>(p, grid, st) : launch_mode<LPH, MAXN, false>(p, grid, st);
 }
 
 template <int MAXN>
