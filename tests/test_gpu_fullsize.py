@@ -183,6 +183,41 @@ def test_config4_full_size_levelised_whole_circuit():
     assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
 
 
+def test_config4_full_size_block_level_by_level_whole_circuit():
+    """All 1 010 000 rows of the 501-level workload after one whole Transformer block in level order (the persistent
+    kernel with attention-stage and feed-forward-stage CTAs), against the checker run on the whole circuit."""
+    w = synth.workload(4)
+    g = w.graph()
+    gr = dg4.dg4_graph_create(g.row_ptr, g.col_idx, g.level, w.hops, 0)
+    dsc = dg4.desc(w.heads, dg4.DG4_BF16, w.scale)
+    xb = w.x_bf16_bits()
+    wq_bits, wq = bf16_weights(w.w_qkv_f32(0))
+    wo_bits, wo = bf16_weights(w.w_o_f32(0))
+    w1_bits, w1 = bf16_weights(synth.normal_f32(44, 1, (512, 128), 0.08))
+    w2_bits, w2 = bf16_weights(synth.normal_f32(44, 2, (128, 512), 0.08))
+    b1 = synth.normal_f32(44, 3, (512,), 0.3).astype(np.float32)
+    b2 = synth.normal_f32(44, 4, (128,), 0.3).astype(np.float32)
+    gam = (synth.normal_f32(44, 5, (128,), 0.2) + 1.0).astype(np.float32)
+    bet = synth.normal_f32(44, 6, (128,), 0.2).astype(np.float32)
+    dv = lambda a: torch.from_numpy(a).cuda()
+    ws = torch.empty(dg4.dg4_layer_workspace_bytes(gr, dsc), dtype=torch.uint8, device="cuda")
+    h = dev_bf16(xb).clone()
+    launches = dg4.dg4_launch_count()
+    dg4.dg4_block_fwd_levelised(gr, dsc, h, dev_bf16(wq_bits), dev_bf16(wo_bits), dv(gam), dv(bet), dev_bf16(w1_bits), dv(b1),
+                                dev_bf16(w2_bits), dv(b2), dv(gam), dv(bet), 1e-5, ws)
+    torch.cuda.synchronize()
+    assert dg4.dg4_graph_poll_status(gr) == 0 and dg4.dg4_launch_count() - launches == 1
+    ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, w.hops)
+    lptr, lnodes = orc.level_buckets(g.level)
+    want = orc.block_levelised(f64_of_bits(xb), wq, wo, gam, bet, w1, b1, w2, b2, gam, bet, ptr, idx, lptr, lnodes, w.heads,
+                               w.scale, eps=1e-5, rounding="bf16")
+    err = rel_row_err(host_f64_of_bf16(h), want)
+    drift = drift_by_level_decile(g.level, err)
+    _report("levelised_drift.txt", [f"cfg4 whole circuit, one block level by level: max row error {err.max():.3e}; "
+                                    "per tenth of the levels: " + " ".join(f"{d:.2e}" for d in drift)])
+    assert err.max() <= BF16_ROW_TOL, (err.max(), int(err.argmax()))
+
+
 def test_config5_full_size_levelised_every_step():
     """The 10 050 000-node, 17 357-level workload in the launch the benchmark times.  (1) The wavefront call, run
     twice, and three successive single-layer calls agree bit for bit.  (2) Layer 1: every row is recomputed by the
