@@ -261,3 +261,19 @@ def test_block_calls_reject_bad_arguments():
     with pytest.raises(dg4.Dg4Error) as e:
         dg4.dg4_ffn_fwd(g, dg4.desc(4, dg4.DG4_F32, 0.25), x, *dev, EPS, x)
     assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+    # several blocks in one call: block count and workspace size are checked on the host, nothing is launched
+    blk = (torch.zeros(384, 128, dtype=torch.bfloat16, device="cuda"), torch.zeros(128, 128, dtype=torch.bfloat16, device="cuda"),
+           dev[4], dev[5]) + tuple(dev)
+    ws = torch.empty(dg4.dg4_blocks_workspace_bytes(g, dsc, 2), dtype=torch.uint8, device="cuda")
+    launches = dg4.dg4_launch_count()
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_blocks_fwd_levelised(g, dsc, x, [blk] * 9, EPS, ws)
+    assert e.value.status == dg4.DG4_ERR_UNSUPPORTED
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_blocks_fwd_levelised(g, dsc, x, [blk] * 3, EPS, ws)           # workspace sized for two blocks
+    assert e.value.status == dg4.DG4_ERR_INVALID_ARG
+    with pytest.raises(dg4.Dg4Error) as e:
+        dg4.dg4_blocks_fwd_levelised(g, dsc, x, [blk[:6] + (dev[2][:, :256],) + blk[7:]] * 2, EPS, ws[1:])   # misaligned workspace
+    assert e.value.status == dg4.DG4_ERR_INVALID_ARG
+    assert dg4.dg4_launch_count() == launches
+    assert dg4.dg4_blocks_workspace_bytes(g, dsc, 0) == 0 and dg4.dg4_blocks_workspace_bytes(g, dsc, 9) == 0
