@@ -47,8 +47,13 @@
 // dealt alternately to an attention stage -- the tile described above without step 4 -- and a feed-forward stage,
 // which keeps W1 in tensor memory and W2 in shared memory and turns the attention stage's rows of a level into
 // the block's output rows (LayerNorm, two transposed products with bias / ReLU between them, residual, LayerNorm)
-// and refreshes the level's K | V rows from THOSE.  The two stages hand each level to one another through the
-// same counters the layers of a wavefront use.
+// and refreshes the level's K | V rows from THOSE.  With the fixed-width table both stages take the same 16-node
+// tiles, so the kernel is launched as clusters of two -- an attention-stage CTA and the feed-forward-stage CTA of
+// the same tiles -- and a tile's rows go from one to the other on chip: the feed-forward CTA reads them out of its
+// partner's shared memory as soon as the partner's arrival on a barrier in ITS shared memory says they are there
+// (no trip through global memory, no wait for the rest of the level).  The way back is a level's worth: the
+// attention stage of the next level waits for the feed-forward stage's counter of this one, as the layers of a
+// wavefront wait for theirs.
 //
 // Several layers run as a wavefront: layer k+1 may process level l as soon as layer k has finished level l
 // (its inputs are that level's new rows) and layer k+1 itself has finished the levels below l.  CTAs are dealt
@@ -122,6 +127,8 @@ enum : int32_t { kCmdExit = 0, kCmdQkv = 1, kCmdKv = 2, kCmdKvThenQkv = 3, kCmdF
 
 struct Misc {
     uint64_t mma0, mma1, mma2, drain;
+    uint64_t pair_rows;                    // feed-forward CTA of a pair: the attention CTA's rows of the next tile are in ITS shared memory
+    uint64_t pair_taken;                   // attention CTA of a pair: the feed-forward CTA has read them
     uint64_t cmd_bar;                      // the workers' next order for the issuing thread is in `cmd`
     int32_t cmd, cmd_buf;
     uint32_t tmem_base;
@@ -157,6 +164,8 @@ struct LevParams {
     // Several blocks: n_layers == 2 x blocks, "layer" 2k is block k's attention stage, 2k+1 its feed-forward stage,
     // and the stages of all blocks form one wavefront.
     int32_t block;
+    int32_t paired;                        // launched as clusters of two: CTA 2j (attention stage) and 2j+1 (feed-forward stage)
+                                           // take the same tiles, and the rows go from one to the other on chip
     float eps;
     const float* ln1_gamma[DG4I_MAX_LAYERS]; const float* ln1_beta[DG4I_MAX_LAYERS];
     const __nv_bfloat16* W1[DG4I_MAX_LAYERS];              // [512, 128]
@@ -236,6 +245,32 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// ---- the two CTAs of a cluster (a block's attention stage and its feed-forward stage, paired tile by tile) ----
+__device__ __forceinline__ uint32_t in_cta(uint32_t smem_addr, uint32_t rank) {      // the same address in the cluster's CTA `rank`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_in_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_from_cluster(uint32_t bar, uint32_t parity, uint32_t limit) {   // bounded, suspended
+    const uint32_t tries = (limit >> 4) + 1u;
+    for (uint32_t i = 0; i < tries; ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(kRelaxedWaitNs) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void ld_cluster_v4(uint32_t cluster_addr, uint32_t* r) {
+    asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // barrier among the eight worker warps only (the issuing warp never joins it)
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 
@@ -279,6 +314,8 @@ levelised_kernel(LevParams p) {
         mbar_init(bar0, 1);
         mbar_init(bar2, 1);
         mbar_init(smem_u32(&misc->mma1), 1);
+        mbar_init(smem_u32(&misc->pair_rows), 1);
+        mbar_init(smem_u32(&misc->pair_taken), 1);
         mbar_init(smem_u32(&misc->drain), 1);
         mbar_init(smem_u32(&misc->cmd_bar), 1);
         misc->cmd = kCmdExit;
@@ -302,6 +339,8 @@ levelised_kernel(LevParams p) {
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
     // half a row (128 bytes) of every block of its layer.
+    const bool paired = BLOCK && p.paired != 0;
+    if (paired) cluster_sync_all();        // the partner's barriers are initialised before anything arrives on them
     const bool ffn_stage = BLOCK && (layer & 1) != 0;
     const int wl = BLOCK ? layer >> 1 : layer;         // whose weights and K | V table this CTA works with
     if (warp < 8 && ffn_stage) {
@@ -513,7 +552,7 @@ levelised_kernel(LevParams p) {
             // epilogues that read tensor memory; the two views meet in shared memory.
             const uint32_t bar1 = smem_u32(&misc->mma1);
             const uint32_t sAct = base + kOffAct, sS32 = base + kOffS32;
-            uint32_t ph1 = 0;
+            uint32_t ph1 = 0, ph_rows = 0;
             float g1[8], be1[8], g2[8], be2[8], bo[8], bh[4];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -548,7 +587,7 @@ levelised_kernel(LevParams p) {
                 for (int tile = bid; tile < tiles; tile += nctas) {
                     const int r = tile * kTile + slot;
                     const int v = r < n_l ? p.level_nodes[first + r] : -1;
-                    if (!waited) {                     // the attention stage has stored this level's rows
+                    if (!paired && !waited) {          // the attention stage has stored this level's rows
                         if (tid == 0) {
                             bool go = misc->failed == 0;
                             if (go) go = wait_counter(prev_arrive + l, prev_target(n_l), p.abort_word, counter_limit);
@@ -561,7 +600,21 @@ levelised_kernel(LevParams p) {
                     }
                     // ---- first LayerNorm, rows into the operand tile
                     float x[8];
-                    {
+                    if (paired) {
+                        // the partner CTA has just finished the same tile: its rows are read out of its shared memory
+                        if (tid == 0) {
+                            bool go = misc->failed == 0 && mbar_wait_from_cluster(smem_u32(&misc->pair_rows), ph_rows, p.poll_limit);
+                            if (!go && ld_acquire(p.abort_word) == 0) give_up(p);
+                            misc->go = go ? 1 : 0;
+                        }
+                        worker_sync();
+                        if (!misc->go) { alive = false; break; }
+                        mbar_wait_from_cluster(smem_u32(&misc->pair_rows), ph_rows, p.poll_limit);   // complete: acquires for this thread
+                        ph_rows ^= 1u;
+                        Piece a;
+                        ld_cluster_v4(in_cta(sHp + operand_piece(slot, sub), 0), a.w);
+                        Elem<true>::unpack(a, x);
+                    } else {
                         const Piece a = load_input(v);
                         Elem<true>::unpack(a, x);
                     }
@@ -571,7 +624,10 @@ levelised_kernel(LevParams p) {
                     if (sub == 0) misc->node[slot] = v;
                     fence_proxy_async_smem();
                     worker_sync();
-                    if (tid == 0) post(kCmdFfn1, 0);
+                    if (tid == 0) {
+                        post(kCmdFfn1, 0);
+                        if (paired) mbar_arrive_in_cluster(in_cta(smem_u32(&misc->pair_taken), 0));   // every lane has its rows
+                    }
                     // ---- hidden units: + b1, ReLU, bf16, into the four activation tiles (operand layout)
                     if (!mbar_wait_relaxed(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph0 ^= 1u;
@@ -659,6 +715,8 @@ levelised_kernel(LevParams p) {
         } else {
         bool pro_ready = false;      // the Q | K | V product of this CTA's next tile has been issued (rows in buffer `buf`)
         int buf = 0;
+        bool rows_out = false;       // paired: a tile's rows are in sHp for the partner
+        uint32_t ph_taken = 0;
 
         for (int l = 0; l < p.n_levels && alive; ++l) {
             const int first = lp0;
@@ -931,6 +989,10 @@ levelised_kernel(LevParams p) {
                     // at N = 16 is longer than the product itself)
                     const bool pre_ok = pre_early || (want_pre && misc->pre_ok != 0);
                     if (pre_ok && !pre_early) xpre = load_input(v_pre);
+                    if (paired && rows_out) {          // the partner has read the previous tile's rows out of sHp
+                        if (!mbar_wait_from_cluster(smem_u32(&misc->pair_taken), ph_taken, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
+                        ph_taken ^= 1u;
+                    }
                     {
                         float acc_o[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
@@ -969,9 +1031,12 @@ levelised_kernel(LevParams p) {
                     if (tid == 0) {
                         if (!BLOCK) post(pre_ok ? kCmdKvThenQkv : kCmdKv, buf ^ 1);
                         else if (pre_ok) post(kCmdQkv, buf ^ 1);
+                        // (paired: the rows stay on chip -- the partner reads them out of this CTA's shared memory)
+                        if (paired) mbar_arrive_in_cluster(in_cta(smem_u32(&misc->pair_rows), 1));
                     }
+                    rows_out = true;
                     const int node_v = misc->node[slot];
-                    {
+                    if (!paired) {
                         uint32_t w4[4];
                         ld_shared_v4(sHp + operand_piece(slot, sub), w4);
                         if (node_v >= 0) st_global_v4((char*)p.H + (size_t)node_v * p.ldh * 2 + sub * 16, w4);
@@ -1035,7 +1100,8 @@ levelised_kernel(LevParams p) {
                 // ---- this CTA's part of (layer, level l) is in global memory: arrive on its counter (release)
                 // (by a thread that does not poll: the release waits for the CTA's outstanding stores, and the pollers
                 // should already be watching the next level's counters meanwhile)
-                if (tid == 64) red_release_add(my_arrive + l, 1);
+                // (the attention CTA of a pair has handed its rows over on chip; nobody reads its counter)
+                if (tid == 64 && !paired) red_release_add(my_arrive + l, 1);
             } else if (!pro_ready && l + 1 < p.n_levels && bid < tiles_next) {
                 // ---- no tile in this level but one in the next: bring that tile up while there is nothing else to do
                 if (tid == 32) {
@@ -1075,6 +1141,7 @@ levelised_kernel(LevParams p) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
+    if (paired) cluster_sync_all();        // neither CTA of a pair leaves while the other may still touch its shared memory
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1091,6 +1158,35 @@ dg4_status launch_mode(const LevParams& p, int grid, cudaStream_t st) {
     int per_sm = 0;
     DG4_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem));
     if (per_sm != 1) DG4_FAIL(DG4_ERR_CUDA, "the levelised kernel needs exactly one CTA per SM on this device (got %d)", per_sm);
+    if (BLOCK && p.paired) {
+        // clusters of two: CTA 2j runs an attention stage, CTA 2j+1 the feed-forward stage of the same tiles
+        LevParams q = p;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(grid & ~1));
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attrs[2];
+        attrs[0].id = cudaLaunchAttributeCooperative;
+        attrs[0].val.cooperative = 1;
+        attrs[1].id = cudaLaunchAttributeClusterDimension;
+        attrs[1].val.clusterDim.x = 2; attrs[1].val.clusterDim.y = 1; attrs[1].val.clusterDim.z = 1;
+        cfg.attrs = attrs;
+        cfg.numAttrs = 2;
+        int clusters = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg);
+        if (e == cudaSuccess && clusters * 2 >= (grid & ~1)) {
+            DG4_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, q));
+            dg4i_count_launch();
+            return DG4_OK;
+        }
+        cudaGetLastError();
+        q.paired = 0;                      // not all pairs can be resident together: plain cooperative launch
+        void* args2[] = {(void*)&q};
+        DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args2, smem, st));
+        dg4i_count_launch();
+        return DG4_OK;
+    }
     void* args[] = {(void*)&p};
     DG4_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem, st));
     dg4i_count_launch();
@@ -1153,7 +1249,7 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
     p.n_levels = g->n_levels; p.n_layers = n_layers;
     p.residual = (desc->flags & DG4_FLAG_RESIDUAL) ? 1 : 0; p.scale = desc->scale;
     p.abort_word = sync; p.arrive = sync + 16; p.status = status; p.poll_limit = dg4i_poll_limit();
-    p.block = 0; p.eps = 0.f;
+    p.block = 0; p.paired = 0; p.eps = 0.f;
     for (int k = 0; k < DG4I_MAX_LAYERS; ++k) {
         p.ln1_gamma[k] = p.ln1_beta[k] = p.b1[k] = p.b2[k] = p.ln2_gamma[k] = p.ln2_beta[k] = nullptr;
         p.W1[k] = p.W2[k] = nullptr;
@@ -1162,6 +1258,8 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         // two kinds of CTA per block, dealt round-robin: attention stage ("layer" 2k) and feed-forward stage (2k+1)
         if (g_sm_count[dev] < 2 * n_layers) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer SMs than stages");
         p.block = 1; p.n_layers = 2 * n_layers; p.eps = block[0].eps; p.residual = 1;
+        // with the fixed-width table both stages take the same 16-node tiles, so CTA 2j and CTA 2j+1 can be paired
+        p.paired = (!g->wide && (g_sm_count[dev] & ~1) >= 2 * 2 * n_layers) ? 1 : 0;
         for (int k = 0; k < n_layers; ++k) {
             p.ln1_gamma[k] = block[k].ln1_gamma; p.ln1_beta[k] = block[k].ln1_beta; p.W1[k] = block[k].W1; p.b1[k] = block[k].b1;
             p.W2[k] = block[k].W2; p.b2[k] = block[k].b2; p.ln2_gamma[k] = block[k].ln2_gamma; p.ln2_beta[k] = block[k].ln2_beta;
