@@ -47,8 +47,8 @@
 // dealt alternately to an attention stage -- the tile described above without step 4 -- and a feed-forward stage,
 // which keeps W1 in tensor memory and W2 in shared memory and turns the attention stage's rows of a level into
 // the block's output rows (LayerNorm, two transposed products with bias / ReLU between them, residual, LayerNorm)
-// and refreshes the level's K | V rows from THOSE.  With the fixed-width table both stages take the same 16-node
-// tiles, so the kernel is launched as clusters of two -- an attention-stage CTA and the feed-forward-stage CTA of
+// and refreshes the level's K | V rows from THOSE.  Both stages take the same tiles, so the kernel is launched as
+// clusters of two -- an attention-stage CTA and the feed-forward-stage CTA of
 // the same tiles -- and a tile's rows go from one to the other on chip: the feed-forward CTA reads them out of its
 // partner's shared memory as soon as the partner's arrival on a barrier in ITS shared memory says they are there
 // (no trip through global memory, no wait for the rest of the level).  The way back is a level's worth: the
@@ -504,11 +504,7 @@ levelised_kernel(LevParams p) {
         };
         auto tiles_of = [&](int n_level, int ctas) { const int t = per_tile(n_level, ctas); return (n_level + t - 1) / t; };
         // arrivals on the layer below's counter for a level of n_level nodes (one per CTA that owns a tile of it)
-        // (a feed-forward stage always fills 16-node tiles)
-        auto prev_target = [&](int n_level) {
-            const int t = (BLOCK && !ffn_stage) ? (n_level + kTile - 1) / kTile : tiles_of(n_level, prev_ctas);
-            return t < prev_ctas ? t : prev_ctas;
-        };
+        auto prev_target = [&](int n_level) { const int t = tiles_of(n_level, prev_ctas); return t < prev_ctas ? t : prev_ctas; };
 
         // this lane's piece of node v's input row (zero for an empty slot) into input buffer b, both layouts
         auto stage_input = [&](int b, const Piece& x) {
@@ -581,12 +577,15 @@ levelised_kernel(LevParams p) {
             for (int l = 0; l < p.n_levels && alive; ++l) {
                 const int first = p.level_ptr[l];
                 const int n_l = p.level_ptr[l + 1] - first;
-                const int tiles = (n_l + kTile - 1) / kTile;
+                // the same tiles as the attention stage (with cone lists: T_l nodes in the first T_l slots; the other
+                // slots, which held replicas there, are empty here)
+                const int T_l = per_tile(n_l, nctas);
+                const int tiles = n_l > 0 ? (n_l + T_l - 1) / T_l : 0;
                 if (n_l <= 0 || bid >= tiles) continue;
                 bool waited = false;
                 for (int tile = bid; tile < tiles; tile += nctas) {
-                    const int r = tile * kTile + slot;
-                    const int v = r < n_l ? p.level_nodes[first + r] : -1;
+                    const int r = tile * T_l + slot;
+                    const int v = (slot < T_l && r < n_l) ? p.level_nodes[first + r] : -1;
                     if (!paired && !waited) {          // the attention stage has stored this level's rows
                         if (tid == 0) {
                             bool go = misc->failed == 0;
@@ -1121,8 +1120,8 @@ levelised_kernel(LevParams p) {
             if (n_l > 0) {
                 last_nonempty = l;
                 last_participants = tiles < nctas ? tiles : nctas;
-                if (BLOCK) {      // the feed-forward stage always fills 16-node tiles
-                    const int t1 = (n_l + kTile - 1) / kTile;
+                if (BLOCK) {      // the feed-forward stage takes the same tiles
+                    const int t1 = tiles_of(n_l, ctas_of(layer + 1));
                     last_participants_ffn = t1 < ctas_of(layer + 1) ? t1 : ctas_of(layer + 1);
                 }
             }
@@ -1258,8 +1257,8 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         // two kinds of CTA per block, dealt round-robin: attention stage ("layer" 2k) and feed-forward stage (2k+1)
         if (g_sm_count[dev] < 2 * n_layers) DG4_FAIL(DG4_ERR_UNSUPPORTED, "fewer SMs than stages");
         p.block = 1; p.n_layers = 2 * n_layers; p.eps = block[0].eps; p.residual = 1;
-        // with the fixed-width table both stages take the same 16-node tiles, so CTA 2j and CTA 2j+1 can be paired
-        p.paired = (!g->wide && (g_sm_count[dev] & ~1) >= 2 * 2 * n_layers) ? 1 : 0;
+        // both stages take the same tiles, so CTA 2j and CTA 2j+1 can be paired
+        p.paired = ((g_sm_count[dev] & ~1) >= 2 * 2 * n_layers) ? 1 : 0;
         for (int k = 0; k < n_layers; ++k) {
             p.ln1_gamma[k] = block[k].ln1_gamma; p.ln1_beta[k] = block[k].ln1_beta; p.W1[k] = block[k].W1; p.b1[k] = block[k].b1;
             p.W2[k] = block[k].W2; p.b2[k] = block[k].b2; p.ln2_gamma[k] = block[k].ln2_gamma; p.ln2_beta[k] = block[k].ln2_beta;
