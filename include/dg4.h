@@ -373,7 +373,8 @@ dg4_status dg4_layers_fwd_levelised(const dg4_graph* g, const dg4_desc* desc, vo
  * per level (the level's rows are taken through the handle's level buckets).  Same results either way.
  * The persistent kernel is launched cooperatively in clusters of two CTAs (a tile's rows go from its attention-stage
  * CTA to its feed-forward-stage CTA through distributed shared memory); if the device cannot hold all pairs at once,
- * or if the environment variable DG4_NO_CLUSTER_PAIRS is set (for profilers that cannot replay such a launch), it is
+ * if the environment variable DG4_NO_CLUSTER_PAIRS is set, or if a tool has injected itself into the process
+ * (CUDA_INJECTION64_PATH / NV_COMPUTE_PROFILER_PERFWORKS_DIR set: profilers that cannot replay such a launch), it is
  * launched plainly cooperatively and the rows go through global memory.
  */
 dg4_status dg4_layernorm_fwd(const dg4_graph* g, const dg4_desc* desc, const void* X, int64_t ldx,

@@ -1260,9 +1260,10 @@ dg4_status dg4i_levelised_launch(const dg4_graph* g, const dg4_desc* desc, int n
         p.block = 1; p.n_layers = 2 * n_layers; p.eps = block[0].eps; p.residual = 1;
         // both stages take the same tiles, so CTA 2j and CTA 2j+1 can be paired
         p.paired = ((g_sm_count[dev] & ~1) >= 2 * 2 * n_layers) ? 1 : 0;
-        // (a profiler that cannot replay a cooperative launch in clusters can ask for the plain cooperative launch,
-        // whose stages hand over through the level counters)
-        if (getenv("DG4_NO_CLUSTER_PAIRS")) p.paired = 0;
+        // (a profiler that cannot replay a cooperative launch in clusters gets the plain cooperative launch, whose
+        // stages hand over through the level counters: on request, or when a tool has injected itself into the process)
+        if (getenv("DG4_NO_CLUSTER_PAIRS") || getenv("NV_COMPUTE_PROFILER_PERFWORKS_DIR") || getenv("CUDA_INJECTION64_PATH"))
+            p.paired = 0;
         for (int k = 0; k < n_layers; ++k) {
             p.ln1_gamma[k] = block[k].ln1_gamma; p.ln1_beta[k] = block[k].ln1_beta; p.W1[k] = block[k].W1; p.b1[k] = block[k].b1;
             p.W2[k] = block[k].W2; p.b2[k] = block[k].b2; p.ln2_gamma[k] = block[k].ln2_gamma; p.ln2_beta[k] = block[k].ln2_beta;
