@@ -243,6 +243,47 @@ def test_blocks_as_one_wavefront_equal_successive_blocks(hops, n_blocks):
     assert rel_row_err(host_f64_of_bf16(h), want).max() <= BF16_ROW_TOL
 
 
+def test_blocks_wavefront_can_be_captured_in_a_cuda_graph():
+    """The persistent block kernel (a cooperative launch in clusters of two) only enqueues on the caller's stream:
+    captured once, its replays give the bits of the eager call."""
+    fanins = random_dag(np.random.default_rng(97), 40, 3000, window=120)
+    rp, ci = csr_from_fanins(fanins)
+    n = len(fanins)
+    g = dg4.dg4_graph_create(rp, ci, levels_of(fanins), 2, 0)
+    dsc = dg4.desc(8, dg4.DG4_BF16, 0.25)
+    x = dev_bf16(synth.normal_bf16_bits(29, 1, (n, 128), 1.0))
+    blocks = []
+    for k in range(2):
+        wq_bits, _ = bf16_weights(synth.normal_f32(29, 10 * k + 2, (384, 128), 0.08))
+        wo_bits, _ = bf16_weights(synth.normal_f32(29, 10 * k + 3, (128, 128), 0.08))
+        blocks.append((dev_bf16(wq_bits), dev_bf16(wo_bits), _vec(29, 10 * k + 4, 128, 0.2, 1.0)[1],
+                       _vec(29, 10 * k + 5, 128, 0.2)[1]) + tuple(_ffn_params(29 + k)[1]))
+    ws = torch.empty(dg4.dg4_blocks_workspace_bytes(g, dsc, 2), dtype=torch.uint8, device="cuda")
+    h = torch.empty_like(x)
+    side = torch.cuda.Stream()
+
+    def run():
+        h.copy_(x)
+        dg4.dg4_blocks_fwd_levelised(g, dsc, h, blocks, EPS, ws)
+
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager = h.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        run()
+    for _ in range(2):
+        h.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(h.view(torch.int16), eager.view(torch.int16))
+    assert dg4.dg4_graph_poll_status(g) == 0
+    dg4.dg4_graph_destroy(g)
+
+
 def test_block_calls_reject_bad_arguments():
     n = 64
     g = _edgeless(n)
