@@ -127,7 +127,10 @@ int64_t dg4_launch_count(void);
  *
  * Allocates device memory and returns when the handle is complete; not for use inside a captured region.  Its
  * uploads and kernels run on a stream of their own: the call neither waits for nor delays work the caller has in
- * flight on other streams (cones of more than two hops are the exception: that path synchronises the device).
+ * flight on other streams (cones of more than two hops are the exception: that path synchronises the device).  The
+ * two small results it needs on the host (the size of the lists, the level offsets) are written by a kernel into
+ * pinned, mapped host memory owned by the library, so they do not queue behind a large device-to-host copy
+ * either.
  * Errors: INVALID_ARG, NOT_SORTED, BAD_DEGREE, BAD_LEVEL, UNSUPPORTED, ALLOC, CUDA.
  */
 dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, const int32_t* col_idx,

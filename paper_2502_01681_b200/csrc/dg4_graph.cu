@@ -403,6 +403,43 @@ dg4_status device_pool(int dev, cudaMemPool_t* out) {
     return DG4_OK;
 }
 
+// Small device-to-host read-backs of graph creation.  A kernel writes the words into pinned host memory that the
+// device has mapped, and the host copies them out after the stream has drained: a copy-engine transfer of the same
+// few bytes would queue behind whatever large device-to-host copy the caller has in flight on another stream and
+// hold graph creation up for its whole length.  One staging buffer per process, grown on demand, taken in turn.
+__global__ void publish_words_kernel(const int32_t* __restrict__ src, int32_t* dst, int64_t count) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < count; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+std::mutex g_stage_mu;
+int32_t* g_stage = nullptr;
+int64_t g_stage_words = 0;
+dg4_status read_words(int32_t* host_dst, const int32_t* dev_src, int64_t count, cudaStream_t st, const char* what) {
+    if (count <= 0) return DG4_OK;
+    std::lock_guard<std::mutex> lock(g_stage_mu);
+    if (g_stage_words < count) {
+        if (g_stage) cudaFreeHost(g_stage);
+        g_stage = nullptr;
+        g_stage_words = 0;
+        const int64_t words = 2 * count > 4096 ? 2 * count : 4096;
+        void* mem = nullptr;
+        cudaError_t e = cudaHostAlloc(&mem, (size_t)words * 4, cudaHostAllocPortable | cudaHostAllocMapped);
+        if (e != cudaSuccess) { cudaGetLastError(); DG4_FAIL(DG4_ERR_ALLOC, "pinned staging buffer of %lld bytes: %s", (long long)words * 4, cudaGetErrorString(e)); }
+        g_stage = (int32_t*)mem;
+        g_stage_words = words;
+    }
+    int32_t* dev_view = nullptr;
+    cudaError_t e = cudaHostGetDevicePointer((void**)&dev_view, g_stage, 0);
+    if (e != cudaSuccess) { cudaGetLastError(); DG4_FAIL(DG4_ERR_CUDA, "%s failed: %s", what, cudaGetErrorString(e)); }
+    const int blocks = (int)((count + 255) / 256 < 64 ? (count + 255) / 256 : 64);
+    publish_words_kernel<<<blocks, 256, 0, st>>>(dev_src, dev_view, count);
+    dg4i_count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess || (e = cudaStreamSynchronize(st)) != cudaSuccess)
+        DG4_FAIL(DG4_ERR_CUDA, "%s failed: %s", what, cudaGetErrorString(e));
+    memcpy(host_dst, g_stage, (size_t)count * 4);
+    return DG4_OK;
+}
+
 template <typename T>
 dg4_status dalloc(T** p, int64_t count, cudaMemPool_t pool, cudaStream_t st) {
     if (count < 1) count = 1;
@@ -561,8 +598,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     } else {
         if ((s = dg4i_graph_device_pass(g, st, true)) != DG4_OK) return fail(s);
         int32_t total = 0;
-        if ((ce = cudaMemcpyAsync(&total, g->nbr_ptr + n, 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "read of neighbourhood total");
-        if ((ce = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ce, "neighbourhood sizes");
+        if ((s = read_words(&total, g->nbr_ptr + n, 1, st, "read of neighbourhood total")) != DG4_OK) return fail(s);
         g->n_nbr = total;
         TRY_ALLOC(g->nbr_idx, g->n_nbr);
         TRY_ALLOC(g->nbr_pad, n * g->pad_width);
@@ -573,8 +609,7 @@ extern "C" dg4_status dg4_graph_create(int32_t n_nodes, const int32_t* row_ptr, 
     g->h_level_ptr = (int32_t*)malloc(((size_t)g->n_levels + 1) * sizeof(int32_t));
     if (!g->h_level_ptr) { dg4_set_error("host allocation failed"); return fail(DG4_ERR_ALLOC); }
     if (g->wide && (ce = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(ce, "graph prep");
-    if ((ce = cudaMemcpyAsync(g->h_level_ptr, g->level_ptr, ((size_t)g->n_levels + 1) * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "read of level_ptr");
-    if ((ce = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(ce, "graph prep");
+    if ((s = read_words(g->h_level_ptr, g->level_ptr, (int64_t)g->n_levels + 1, st, "read of level_ptr")) != DG4_OK) return fail(s);
     *out = g;
     return DG4_OK;
 }

@@ -617,6 +617,62 @@ def test_stream_ordered_destroy_and_pooled_create():
     dg4.dg4_graph_destroy(gr)
 
 
+def test_graph_create_from_several_host_threads_under_a_read_back():
+    """Graph creation fetches its small results through one staging buffer taken in turn: handles created from
+    four host threads at once, of different sizes, while a large device-to-host copy is in flight on another
+    stream, all hold the oracle's lists and level buckets, and the host's copy of the level offsets is whole."""
+    import threading
+    cases = [(2, 40), (3, 40), (2, 7), (4, 40)]
+    graphs = [synth.workload(c, s).graph() for c, s in cases]
+    big = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
+    host = torch.empty(64 << 20, dtype=torch.int32).pin_memory()
+    side = torch.cuda.Stream()
+    made, errors = [None] * len(cases), []
+
+    def create(i):
+        try:
+            made[i] = dg4.dg4_graph_create(graphs[i].row_ptr, graphs[i].col_idx, graphs[i].level, 2, 0)
+        except Exception as e:                                 # reported by the main thread
+            errors.append(e)
+
+    for rep in range(2):
+        with torch.cuda.stream(side):
+            host.copy_(big, non_blocking=True)
+        threads = [threading.Thread(target=create, args=(i,)) for i in range(len(cases))]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+        torch.cuda.synchronize()
+        assert not errors
+        for i, g in enumerate(graphs):
+            ptr, idx = orc.neighbourhood(g.row_ptr, g.col_idx, 2)
+            lptr, lnodes = orc.level_buckets(g.level)
+            assert made[i].info.n_nbr == len(idx) and made[i].info.n_levels == len(lptr) - 1
+            assert (dg4.dg4_graph_export(made[i], dg4.DG4_ARR_NBR_PTR) == ptr).all()
+            assert (dg4.dg4_graph_export(made[i], dg4.DG4_ARR_LEVEL_PTR) == lptr).all()
+            assert (dg4.dg4_graph_export(made[i], dg4.DG4_ARR_LEVEL_NODES) == lnodes).all()
+            # the host's copy of the level offsets drives the one-launch-group-per-level order: same bits as the
+            # persistent kernel's order only if every offset arrived
+            dsc = dg4.desc(8, dg4.DG4_BF16, 0.25, residual=True)
+            by_level = dg4.desc(8, dg4.DG4_BF16, 0.25, residual=True, level_launches=True)
+            ws = torch.empty(dg4.dg4_layer_workspace_bytes(made[i], dsc), dtype=torch.uint8, device="cuda")
+            xb = synth.normal_bf16_bits(31, i, (g.n, 128), 1.0)
+            wq_bits, wq = bf16_weights(synth.normal_f32(31, 50, (384, 128), 0.08))
+            wo_bits, wo = bf16_weights(synth.normal_f32(31, 51, (128, 128), 0.08))
+            h_a, h_b = dev_bf16(xb).clone(), dev_bf16(xb).clone()
+            dg4.dg4_layer_fwd_levelised(made[i], dsc, h_a, dev_bf16(wq_bits), dev_bf16(wo_bits), ws)
+            dg4.dg4_layer_fwd_levelised(made[i], by_level, h_b, dev_bf16(wq_bits), dev_bf16(wo_bits), ws)
+            torch.cuda.synchronize()
+            assert dg4.dg4_graph_poll_status(made[i]) == 0
+            assert rel_row_err(host_f64_of_bf16(h_a), host_f64_of_bf16(h_b)).max() <= BF16_ROW_TOL
+            if i == 0 and rep == 0:
+                want = orc.layer_levelised(f64_of_bits(xb), wq, wo, ptr, idx, lptr, lnodes, 8, 0.25, residual=True,
+                                           rounding="bf16")
+                assert rel_row_err(host_f64_of_bf16(h_b), want).max() <= BF16_ROW_TOL
+            dg4.dg4_graph_destroy(made[i])
+
+
 @pytest.mark.parametrize("mode", ["parallel", "levelised"])
 def test_forward_calls_can_be_captured_in_a_cuda_graph(mode):
     """The forward calls only enqueue work on the caller's stream (no allocation, no synchronisation), so a stack
