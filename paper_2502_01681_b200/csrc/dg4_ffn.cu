@@ -92,15 +92,11 @@ __device__ __forceinline__ uint16_t bf16_bits(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
 }
-// max(0, lo) and max(0, hi) rounded to bf16 in one conversion, stored as two 16-bit values
-__device__ __forceinline__ void relu_pack_store2(uint32_t addr_lo, uint32_t addr_hi, float lo, float hi) {
-    asm volatile(
-        "{\n\t.reg .b32 pk;\n\t.reg .b16 l, h;\n\t"
-        "cvt.rn.relu.bf16x2.f32 pk, %3, %2;\n\t"
-        "mov.b32 {l, h}, pk;\n\t"
-        "st.shared.b16 [%0], l;\n\t"
-        "st.shared.b16 [%1], h;\n\t}"
-        ::"r"(addr_lo), "r"(addr_hi), "f"(lo), "f"(hi) : "memory");
+// max(0, lo) and max(0, hi) rounded to bf16 in one conversion (lo in the low half)
+__device__ __forceinline__ uint32_t relu_pack(float lo, float hi) {
+    uint32_t pk;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %2, %1;" : "=r"(pk) : "f"(lo), "f"(hi));
+    return pk;
 }
 // barrier (and barrier with an OR reduction) among the eight worker warps only
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
@@ -166,7 +162,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
 
     // W1 into tensor memory: hidden unit `ln` of block q in lane `ln`, two consecutive inputs per 32-bit column
     // (the bytes as they lie in global memory); each worker thread copies half a row (128 bytes) of every block.
-    float b1v[4] = {0.f, 0.f, 0.f, 0.f};
+    float b1v[4][4] = {};                                // b1 of the hidden units this thread holds after a fragment load
     if (warp < 8) {
         for (int q = 0; q < 4; ++q) {
             const uint4* src = reinterpret_cast<const uint4*>(p.W1 + (size_t)(q * 128 + ln) * 128 + cg * 64);
@@ -176,7 +172,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 const uint32_t r[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
                 tmem_st_32x8(tmem + lane_base + (uint32_t)(kColW1 + q * 64 + cg * 32 + c * 8), r);
             }
-            b1v[q] = p.b1[q * 128 + ln];
+#pragma unroll
+            for (int m = 0; m < 4; ++m) b1v[q][m] = p.b1[q * 128 + q4 * 32 + 8 * m + (lane >> 2)];
         }
         tmem_st_wait();
     }
@@ -236,9 +233,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
             __threadfence_block();
             *reinterpret_cast<volatile int32_t*>(&misc->posted) = misc->posted + 1;
         };
-        uint32_t a2_base[8];                             // where this thread's hidden unit lies in rows cg*64 + (0..7)
-#pragma unroll
-        for (int k = 0; k < 8; ++k) a2_base[k] = sA2 + operand_offset(cg * 64 + k, ln) - (uint32_t)(k * 128);
+        // The accumulator of a first product holds hidden units in lanes and rows in columns; the operand of the
+        // second product wants rows with their hidden units contiguous.  A fragment load followed by a transposing
+        // matrix store does that 8 rows x 32 hidden units at a time: thread 8m + j passes the address of row
+        // cg*64 + 8c + j, hidden units q4*32 + 8m .. +7 (16 bytes; the swizzle depends on j only).
+        const uint32_t a2_addr = sA2 + operand_offset(cg * 64 + (lane & 7), q4 * 32 + 8 * (lane >> 3));
         uint32_t ph_g1 = 0, ph_g2 = 0;
         bool failed = false;
         if (first_tile < p.n_tiles) failed |= !mbar_wait(bar_w, 0, p.poll_limit);
@@ -283,8 +282,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 ph_g1 ^= 1u;
                 tc_fence_after();
                 uint32_t d[64];
-                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64), d);
-                tmem_ld_32x32(tmem + lane_base + (uint32_t)(kColD1 + cg * 64 + 32), d + 32);
+                tmem_ld_16x256b_x8(tmem + lane_base + (uint32_t)(kColD1 + cg * 64), d);                  // lanes +0..15
+                tmem_ld_16x256b_x8(tmem + lane_base + (16u << 16) + (uint32_t)(kColD1 + cg * 64), d + 32);  // lanes +16..31
                 tmem_ld_wait();
                 tc_fence_before();
                 if (!LISTED && q == 0 && tid == 0) bulk_wait_read0();   // the previous tile's store has read the staging buffer
@@ -294,13 +293,18 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);
                     ph_g2 ^= 1u;
                 }
-                // rows cg*64 + j: element `ln` of row j lies at a2_base[j & 7] + 128 j (the swizzle depends on j & 7
-                // only, because cg*64 is a multiple of 8); two rows per conversion, ReLU folded into it
-                const float bq = b1v[q];
+                // d[32u + 4c + 2h + e]: hidden unit q4*32 + 8(2u + h) + lane/4, row cg*64 + 8c + 2(lane%4) + e; bias and
+                // ReLU folded into the conversion, then eight rows of 32 hidden units per store
 #pragma unroll
-                for (int j = 0; j < 64; j += 2)
-                    relu_pack_store2(a2_base[j & 7] + (uint32_t)(j * 128), a2_base[(j + 1) & 7] + (uint32_t)((j + 1) * 128),
-                                     __uint_as_float(d[j]) + bq, __uint_as_float(d[j + 1]) + bq);
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t m[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int i = 32 * (k >> 1) + 4 * c + 2 * (k & 1);
+                        m[k] = relu_pack(__uint_as_float(d[i]) + b1v[q][k], __uint_as_float(d[i + 1]) + b1v[q][k]);
+                    }
+                    stmatrix_x4_trans(a2_addr + (uint32_t)(c * 1024), m);
+                }
                 fence_proxy_async_smem();
                 worker_sync();
                 if (tid == 0) release_product();             // G2(q)

@@ -10,6 +10,7 @@ kernels, so the rows must agree well inside the bf16 tolerance used throughout t
 
 Collected last on purpose: a failure here cannot hide the result of any other test in a fail-fast run."""
 import ctypes
+import gc
 
 import numpy as np
 import pytest
@@ -60,6 +61,7 @@ def test_static_scratch_layer_matches_regular_layer_twice():
         # From the second call on a device nothing is taken from the device heap or from the framework's
         # allocator.  (The very first call may: the driver may instantiate the library image, and with it the
         # 32 MiB array, only then -- which is why that call belongs at start-up.)
+        gc.collect()          # tensors of earlier tests that only a collection frees must not be freed in between
         free0, _ = torch.cuda.mem_get_info()
         stats0 = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
         for _ in range(3):
