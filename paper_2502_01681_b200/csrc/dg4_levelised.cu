@@ -185,6 +185,32 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t* r) {
 __device__ __forceinline__ void st_shared_b16(uint32_t addr, uint16_t v) {
     asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
 }
+// NB accumulators (lanes = 128 output features, 16 columns = the tile's nodes, kTile columns apart) into the staging
+// rows as bf16: the warp reads its 32 lanes x 8 nodes as m16n8 fragments and writes, per accumulator, one transposing
+// matrix store -- 8 nodes x 32 features, 16 bytes (8 features) per node and matrix.  `taddr`: the first accumulator
+// at this warp's lanes and columns; `st_addr`: thread 8m + j passes staging row j of the warp's 8 nodes at
+// features 8m of the warp's 32.
+__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo, uint32_t hi) {
+    uint32_t pk;
+    asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pk) : "f"(__uint_as_float(lo)), "f"(__uint_as_float(hi)));
+    return pk;
+}
+template <int NB>
+__device__ __forceinline__ void accumulators_to_stage(uint32_t taddr, uint32_t st_addr) {
+    uint32_t r[NB][8];
+#pragma unroll
+    for (int blk = 0; blk < NB; ++blk) {
+        tmem_ld_16x256b_x1(taddr + (uint32_t)(blk * kTile), r[blk]);
+        tmem_ld_16x256b_x1(taddr + (16u << 16) + (uint32_t)(blk * kTile), r[blk] + 4);
+    }
+    tmem_ld_wait();
+#pragma unroll
+    for (int blk = 0; blk < NB; ++blk) {
+        const uint32_t m[4] = {pack_bf16x2(r[blk][0], r[blk][1]), pack_bf16x2(r[blk][2], r[blk][3]),
+                               pack_bf16x2(r[blk][4], r[blk][5]), pack_bf16x2(r[blk][6], r[blk][7])};
+        stmatrix_x4_trans(st_addr + (uint32_t)(blk * 256), m);
+    }
+}
 __device__ __forceinline__ void st_global_v4(void* p, const uint32_t* r) {
     asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
 }
@@ -336,6 +362,8 @@ levelised_kernel(LevParams p) {
     static_assert(kWorkers / 32 / 4 * 8 == kTile, "epilogue: every warp reads 8 node columns of its lane quadrant");
     const int q4 = warp & 3, cg = warp >> 2;             // TMEM lane quadrant of the warp; which half of the columns it takes
     const int feat = q4 * 32 + lane;                     // output feature (TMEM lane) this thread holds
+    // where this thread points a transposing matrix store of its warp's 8 nodes x 32 features (see accumulators_to_stage)
+    const uint32_t stage_frag = sSt + (uint32_t)((cg * 8 + (lane & 7)) * kStageRow + (q4 * 32 + 8 * (lane >> 3)) * 2);
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     // The weights stay in tensor memory for the whole kernel: row `feat` of every block in lane `feat`, two
     // consecutive bf16 of the row per 32-bit column (the bytes as they lie in global memory).  Each thread copies
@@ -681,20 +709,7 @@ levelised_kernel(LevParams p) {
                     if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
                     tc_fence_after();
-                    {
-                        uint32_t d[2][8];
-#pragma unroll
-                        for (int blk = 0; blk < 2; ++blk)
-                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int blk = 0; blk < 2; ++blk) {
-                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
-#pragma unroll
-                            for (int nn = 0; nn < 8; ++nn)
-                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
-                        }
-                    }
+                    accumulators_to_stage<2>(tmem + lane_base + (uint32_t)(kTile * kAccK2 + cg * 8), stage_frag);
                     tc_fence_before();
                     worker_sync();
                     if (v >= 0) {
@@ -768,18 +783,7 @@ levelised_kernel(LevParams p) {
                         if (!mbar_wait_relaxed(bar0, ph0, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                         ph0 ^= 1u;
                         tc_fence_after();
-                        uint32_t d[3][8];
-#pragma unroll
-                        for (int blk = 0; blk < 3; ++blk)
-                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccQ + blk) + cg * 8), d[blk]);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int blk = 0; blk < 3; ++blk) {
-                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
-#pragma unroll
-                            for (int nn = 0; nn < 8; ++nn)
-                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
-                        }
+                        accumulators_to_stage<3>(tmem + lane_base + (uint32_t)(kTile * kAccQ + cg * 8), stage_frag);
                         tc_fence_before();
                     };
                     if (pro_ready) epilogue_qkv();
@@ -1066,20 +1070,7 @@ levelised_kernel(LevParams p) {
                     if (!mbar_wait_relaxed(bar2, ph2, p.poll_limit) && tid == 0) { give_up(p); misc->failed = 1; }
                     ph2 ^= 1u;
                     tc_fence_after();
-                    {
-                        uint32_t d[2][8];
-#pragma unroll
-                        for (int blk = 0; blk < 2; ++blk)
-                            tmem_ld_32x8(tmem + lane_base + (uint32_t)(kTile * (kAccK2 + blk) + cg * 8), d[blk]);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int blk = 0; blk < 2; ++blk) {
-                            const uint32_t off = (uint32_t)(blk * 256 + feat * 2);
-#pragma unroll
-                            for (int nn = 0; nn < 8; ++nn)
-                                st_shared_b16(sSt + (uint32_t)((cg * 8 + nn) * kStageRow) + off, bf16_bits(__uint_as_float(d[blk][nn])));
-                        }
-                    }
+                    accumulators_to_stage<2>(tmem + lane_base + (uint32_t)(kTile * kAccK2 + cg * 8), stage_frag);
                     tc_fence_before();
                     worker_sync();
                     if (node_v >= 0) {

@@ -113,6 +113,12 @@ __device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, uint32_t* r) 
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+// The same fragment layout for one group of 8 columns: r[0], r[1] = columns 2(t%4), +1 of lane (lane base + t/4),
+// r[2], r[3] = the same columns of lane (lane base + t/4 + 8).
+__device__ __forceinline__ void tmem_ld_16x256b_x1(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x1.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+}
 // Four 8 x 8 matrices of 16-bit elements, each stored transposed: thread t holds of matrix i (register r[i]) the
 // elements 2(t%4), +1 of its row t/4; column j of matrix i goes, as 16 contiguous bytes, to the shared-memory
 // address that thread 8i + j passes.
