@@ -8,9 +8,9 @@
 //   * W1 stays in TENSOR memory for the whole kernel (4 blocks of 128 hidden units x 128 inputs = 4 x 64 columns)
 //     and is the A operand of the first product, computed TRANSPOSED per block q of 128 hidden units:
 //         D1^T[hidden, row] = W1_q (tensor memory) * X^T (the X tile in shared memory, K-major, as B operand);
-//   * the epilogue of block q (thread = hidden unit, registers = rows) adds b1, applies the ReLU, rounds to
-//     bf16 and scatters the values into shared memory as the K-major, 128-byte-swizzled A operand of the
-//     second product: A2[row, hidden of block q];
+//   * the epilogue of block q reads the accumulator as m16n8 fragments, adds b1, applies the ReLU, rounds to bf16
+//     and writes the values with transposing matrix stores (8 rows x 32 hidden units each) into shared memory as
+//     the K-major, 128-byte-swizzled A operand of the second product: A2[row, hidden of block q];
 //   * second product, accumulated over the four blocks: D2[row, out] += A2 * W2_q^T with W2 resident in shared
 //     memory (4 chunks of 128 outputs x 128 hidden units, 128 KiB, loaded once by TMA);
 //   * final epilogue (thread = row, two threads per row): + b2 + the X row (still in shared memory), mean and
