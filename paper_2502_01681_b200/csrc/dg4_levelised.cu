@@ -190,7 +190,7 @@ __device__ __forceinline__ void st_shared_b16(uint32_t addr, uint16_t v) {
 // matrix store -- 8 nodes x 32 features, 16 bytes (8 features) per node and matrix.  `taddr`: the first accumulator
 // at this warp's lanes and columns; `st_addr`: thread 8m + j passes staging row j of the warp's 8 nodes at
 // features 8m of the warp's 32.
-__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo, uint32_t hi) {
+__device__ __forceinline__ uint32_t pack_bf16x2_of_bits(uint32_t lo, uint32_t hi) {   // fp32 bit patterns in, as tcgen05.ld delivers them
     uint32_t pk;
     asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pk) : "f"(__uint_as_float(lo)), "f"(__uint_as_float(hi)));
     return pk;
@@ -206,8 +206,8 @@ __device__ __forceinline__ void accumulators_to_stage(uint32_t taddr, uint32_t s
     tmem_ld_wait();
 #pragma unroll
     for (int blk = 0; blk < NB; ++blk) {
-        const uint32_t m[4] = {pack_bf16x2(r[blk][0], r[blk][1]), pack_bf16x2(r[blk][2], r[blk][3]),
-                               pack_bf16x2(r[blk][4], r[blk][5]), pack_bf16x2(r[blk][6], r[blk][7])};
+        const uint32_t m[4] = {pack_bf16x2_of_bits(r[blk][0], r[blk][1]), pack_bf16x2_of_bits(r[blk][2], r[blk][3]),
+                               pack_bf16x2_of_bits(r[blk][4], r[blk][5]), pack_bf16x2_of_bits(r[blk][6], r[blk][7])};
         stmatrix_x4_trans(st_addr + (uint32_t)(blk * 256), m);
     }
 }
