@@ -85,12 +85,10 @@ __device__ __forceinline__ void st_shared_f2(uint32_t addr, float a, float b) {
 __device__ __forceinline__ void ld_shared_f2(uint32_t addr, float& a, float& b) {
     asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
 }
-__device__ __forceinline__ uint16_t bf16_bits(float x) {
-    __nv_bfloat16 h = __float2bfloat16_rn(x);
-    return *reinterpret_cast<uint16_t*>(&h);
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {   // both rounded to nearest even in one conversion
+    uint32_t pk;
+    asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(pk) : "f"(lo), "f"(hi));
+    return pk;
 }
 // max(0, lo) and max(0, hi) rounded to bf16 in one conversion (lo in the low half)
 __device__ __forceinline__ uint32_t relu_pack(float lo, float hi) {
@@ -372,6 +370,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 const float mean = 0.5f * (m + mo);
                 const float var = (m2 + m2o + 32.0f * (m - mo) * (m - mo)) * (1.0f / 128.0f);
                 const float rstd = rsqrtf(var + p.eps);
+                const float nmr = -mean * rstd;              // (y - mean) rstd as one fused multiply-add per element
                 const float4* gv = reinterpret_cast<const float4*>(p.gamma + cg * 64);
                 const float4* bv = reinterpret_cast<const float4*>(p.beta + cg * 64);
 #pragma unroll
@@ -379,10 +378,10 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     const float4 ga = __ldg(gv + 2 * c), gb = __ldg(gv + 2 * c + 1);
                     const float4 ba = __ldg(bv + 2 * c), bb = __ldg(bv + 2 * c + 1);
                     uint32_t w[4];
-                    w[0] = pack_bf16((y[c * 8 + 0] - mean) * rstd * ga.x + ba.x, (y[c * 8 + 1] - mean) * rstd * ga.y + ba.y);
-                    w[1] = pack_bf16((y[c * 8 + 2] - mean) * rstd * ga.z + ba.z, (y[c * 8 + 3] - mean) * rstd * ga.w + ba.w);
-                    w[2] = pack_bf16((y[c * 8 + 4] - mean) * rstd * gb.x + bb.x, (y[c * 8 + 5] - mean) * rstd * gb.y + bb.y);
-                    w[3] = pack_bf16((y[c * 8 + 6] - mean) * rstd * gb.z + bb.z, (y[c * 8 + 7] - mean) * rstd * gb.w + bb.w);
+                    w[0] = pack_bf16(fmaf(fmaf(y[c * 8 + 0], rstd, nmr), ga.x, ba.x), fmaf(fmaf(y[c * 8 + 1], rstd, nmr), ga.y, ba.y));
+                    w[1] = pack_bf16(fmaf(fmaf(y[c * 8 + 2], rstd, nmr), ga.z, ba.z), fmaf(fmaf(y[c * 8 + 3], rstd, nmr), ga.w, ba.w));
+                    w[2] = pack_bf16(fmaf(fmaf(y[c * 8 + 4], rstd, nmr), gb.x, bb.x), fmaf(fmaf(y[c * 8 + 5], rstd, nmr), gb.y, bb.y));
+                    w[3] = pack_bf16(fmaf(fmaf(y[c * 8 + 6], rstd, nmr), gb.z, bb.z), fmaf(fmaf(y[c * 8 + 7], rstd, nmr), gb.w, bb.w));
                     st_shared_v4(sA2 + (uint32_t)(cg * kHalf) + sw128_offset(ln, c), w);
                 }
             }
