@@ -418,7 +418,7 @@ def run_ours(args, w):
     # runs 3 parallel + 3 levelised layers and reads the result back into pinned memory.  Steps are pipelined
     # the way a serving loop would be: while step i computes, the host validates and uploads circuit i+1 on a
     # second stream, and the result of step i-1 drains on a third one.
-    e2e_steps = max(2, min(8, args.steps))      # enough steps for the three-stage pipeline's fill and drain to amortise
+    e2e_steps = max(2, min(16, args.steps))     # as many as the timed steps (at most 16): the three-stage pipeline's fill and drain amortise over them
     h2d = x_host.numel() * 2 + (g.row_ptr.nbytes + g.col_idx.nbytes + g.level.nbytes)
     d2h = out_host.numel() * 2 * (1 if args.no_levelised else 2)      # the parallel and the levelised result
     up, down = torch.cuda.Stream(), torch.cuda.Stream()
