@@ -16,7 +16,9 @@
 //   * final epilogue (thread = row, two threads per row): + b2 + the X row (still in shared memory), mean and
 //     variance of the row combined from the two half-rows, gamma / beta, bf16, staged in shared memory and
 //     written with a TMA store (the last tile is clipped by the tensor map).
-//   The X tile of the next tile is prefetched by TMA while the current one is processed.
+//   The X tile of the next tile is prefetched by TMA while the current one is processed.  Inside a tile the eight
+//   worker warps never wait for one another: each arrives on an mbarrier when it has read the accumulator or
+//   written its part of the operand, and the warp that issues the products waits on those.
 // Every CTA loads its own tiles (no load is shared across CTAs).  Every wait is bounded; after a timeout the kernel records DG4_ERR_TIMEOUT and
 // the CTA leaves its tile loop.
 #include "dg4_internal.h"
@@ -43,9 +45,9 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr int kColD1 = 0, kColD2 = 128, kColW1 = 256, kTmemCols = 512;
 
 struct Misc {
-    uint64_t bar_w, bar_x[2], bar_g1, bar_g2, bar_drain;
+    uint64_t bar_w, bar_x[2], bar_g1, bar_g2, bar_d1free, bar_a2full, bar_drain;
     uint32_t tmem_base;
-    int32_t posted;            // products the workers have released to the issuing thread so far (monotone)
+    int32_t posted;            // tiles whose rows have landed, as told to the issuing thread so far (monotone)
     int32_t stop;              // the workers are leaving: no further products
 };
 
@@ -134,6 +136,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         mbar_init(bar_x[1], 1);
         mbar_init(bar_g1, 1);
         mbar_init(bar_g2, 1);
+        mbar_init(smem_u32(&misc->bar_d1free), kWorkers / 32);     // one arrival per worker warp
+        mbar_init(smem_u32(&misc->bar_a2full), kWorkers / 32);
         mbar_init(smem_u32(&misc->bar_drain), 1);
         misc->posted = 0;
         misc->stop = 0;
@@ -184,28 +188,45 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
 
     if (warp == 8) {
         // ------------------------------------------------------------------ the issuing thread
-        // The order of the products is fixed (per tile: G1(0) G1(1) G2(0) G1(2) G2(1) G1(3) G2(2) G2(3)), so the
-        // workers only release them one by one: `posted` counts the releases.  Issuing a product keeps the issuing
-        // thread busy for about as long as the tensor pipe needs to execute it, which is why no worker does it.
+        // The order of the products is fixed (per tile: G1(0) G1(1) G2(0) G1(2) G2(1) G1(3) G2(2) G2(3)).  A tile's first
+        // product waits for the word that its rows have landed (`posted`); every other first product for all eight
+        // worker warps to have read the accumulator D1 (bar_d1free), every second product for all of them to have
+        // written their part of the activation buffer (bar_a2full): the warps arrive on those barriers and go on, none
+        // waits for another.  Issuing a product keeps the issuing thread busy for about as long as the tensor pipe
+        // needs to execute it, which is why no worker does it.
         if (lane == 0) {
             int consumed = 0;
             bool leave = false;
             const uint32_t token_limit = p.poll_limit < (1u << 28) ? p.poll_limit << 2 : p.poll_limit;
+            const uint32_t bar_d1free = smem_u32(&misc->bar_d1free), bar_a2full = smem_u32(&misc->bar_a2full);
+            uint32_t ph_d1 = 0, ph_a2 = 0;
             int it = 0;
             for (int tile = first_tile; tile < p.n_tiles && !leave; tile += (int)gridDim.x, ++it) {
                 const uint64_t dX = smem_desc_sw128(sX + (it & 1) * kTileBytes);
                 for (int step = 0; step < 8 && !leave; ++step) {
-                    uint32_t polls = 0;
-                    while (*reinterpret_cast<volatile int32_t*>(&misc->posted) <= consumed) {
-                        if (*reinterpret_cast<volatile int32_t*>(&misc->stop) != 0 || ++polls > token_limit) { leave = true; break; }
-                        if (polls > 256) __nanosleep(20);
+                    const bool first_product = (step == 0) || (step == 1) || (step == 3) || (step == 5);
+                    if (step == 0) {
+                        uint32_t polls = 0;
+                        while (*reinterpret_cast<volatile int32_t*>(&misc->posted) <= consumed) {
+                            if (*reinterpret_cast<volatile int32_t*>(&misc->stop) != 0 || ++polls > token_limit) { leave = true; break; }
+                            if (polls > 256) __nanosleep(20);
+                        }
+                        if (leave || *reinterpret_cast<volatile int32_t*>(&misc->stop) != 0) { leave = true; break; }
+                        ++consumed;
+                        __threadfence_block();
+                        if (it > 0) {                    // block 3 of the tile before is out of D1 (long since: its second product was issued)
+                            if (!mbar_wait(bar_d1free, ph_d1, token_limit)) { leave = true; break; }
+                            ph_d1 ^= 1u;
+                        }
+                    } else if (first_product) {
+                        if (!mbar_wait(bar_d1free, ph_d1, token_limit)) { leave = true; break; }
+                        ph_d1 ^= 1u;
+                    } else {
+                        if (!mbar_wait(bar_a2full, ph_a2, token_limit)) { leave = true; break; }
+                        ph_a2 ^= 1u;
                     }
-                    if (leave || *reinterpret_cast<volatile int32_t*>(&misc->stop) != 0) { leave = true; break; }
-                    ++consumed;
-                    __threadfence_block();
                     tc_fence_after();
                     // steps 0, 1, 3, 5 are first products of blocks 0..3; steps 2, 4, 6, 7 second products of blocks 0..3
-                    const bool first_product = (step == 0) || (step == 1) || (step == 3) || (step == 5);
                     const int q = first_product ? (step + 1) / 2 : (step == 7 ? 3 : step / 2 - 1);
                     if (first_product) {             // D1^T = W1_q * X^T
 #pragma unroll
@@ -227,7 +248,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
         }
     } else {
         // ------------------------------------------------------------------ the eight worker warps
-        auto release_product = [&]() {               // one worker thread, after the barrier that made the operands visible
+        const uint32_t bar_d1free = smem_u32(&misc->bar_d1free), bar_a2full = smem_u32(&misc->bar_a2full);
+        auto release_product = [&]() {               // one worker thread: the rows of a tile have landed
             __threadfence_block();
             *reinterpret_cast<volatile int32_t*>(&misc->posted) = misc->posted + 1;
         };
@@ -284,9 +306,12 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                 tmem_ld_16x256b_x8(tmem + lane_base + (16u << 16) + (uint32_t)(kColD1 + cg * 64), d + 32);  // lanes +16..31
                 tmem_ld_wait();
                 tc_fence_before();
-                if (!LISTED && q == 0 && tid == 0) bulk_wait_read0();   // the previous tile's store has read the staging buffer
-                worker_sync();                               // every thread holds its part of D1^T
-                if (tid == 0 && q < 3) release_product();    // G1(q + 1)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_d1free);      // this warp holds its part of D1^T: G1(q + 1) may overwrite it
+                if (!LISTED && q == 0) {                     // the previous tile's store has read the staging buffer
+                    if (tid == 0) bulk_wait_read0();
+                    worker_sync();
+                }
                 if (q > 0) {                                 // the previous block's second product has read the buffer
                     failed |= !mbar_wait(bar_g2, ph_g2, p.poll_limit);
                     ph_g2 ^= 1u;
@@ -304,8 +329,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CU
                     stmatrix_x4_trans(a2_addr + (uint32_t)(c * 1024), m);
                 }
                 fence_proxy_async_smem();
-                worker_sync();
-                if (tid == 0) release_product();             // G2(q)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_a2full);      // this warp's part of the operand is written: G2(q)
             }
             // The next tile's rows were requested a tile ago and have landed: its first product may run under this
             // tile's final epilogue (its accumulator is free: every worker has read block 3's before the last barrier).
